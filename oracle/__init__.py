@@ -1,0 +1,159 @@
+"""TEST INFRASTRUCTURE: ctypes front-end of the fp64 CPU oracle (``nsp_oracle.c``).
+
+Only tests, the smoke check and the benchmark's CPU-baseline / reference legs import this package. It never
+imports the CUDA package and shares nothing with it. All arithmetic lives in the C file; this module only
+compiles it with gcc, marshals numpy arrays and reshapes results.
+
+Conventions (identical to the C file header): packed ragged token-major tensors, bf16 inputs passed as
+``uint16`` bit patterns (or ``float64`` arrays for finite-difference checks), float64 outputs.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "nsp_oracle.c"
+_LIB = _HERE / "liboracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile the oracle with gcc (-O2, OpenMP). Rebuilds when the source is newer than the library."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-fno-fast-math", str(_SRC), "-o", str(tmp), "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(str(_LIB))
+        _lib.orc_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().orc_num_threads())
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _dt(a) -> int:
+    if a.dtype == np.uint16:
+        return 0
+    if a.dtype == np.float64:
+        return 1
+    raise TypeError("oracle inputs are uint16 (bf16 bits) or float64")
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError(f"oracle {what} failed with code {rc}")
+
+
+def layout_sizes(cu, hq, hkv, D):
+    cu, hq, hkv = _i32(cu), _i32(hq), _i32(hkv)
+    L = np.diff(cu).astype(np.int64)
+    return int((L * hq).sum() * D), int((L * hkv).sum() * D), int((L * hq).sum())
+
+
+def attn_fwd(q, k, v, cu, hq, hkv, D, scale):
+    """Full forward. Returns (O [q_elems] f64, LSE [lse_elems] f64)."""
+    lib = _load()
+    cu, hq, hkv = _i32(cu), _i32(hq), _i32(hkv)
+    qe, _, le = layout_sizes(cu, hq, hkv, D)
+    O = np.zeros(qe, np.float64)
+    LSE = np.zeros(le, np.float64)
+    dt = _dt(q)
+    rc = lib.orc_attn_fwd(_p(q), _p(k), _p(v), ctypes.c_int(dt), _p(cu), _p(hq), _p(hkv), ctypes.c_int(len(hq)),
+                          ctypes.c_int(D), ctypes.c_double(scale), _p(O), _p(LSE))
+    _check(rc, "attn_fwd")
+    return O, LSE
+
+
+def attn_bwd(q, k, v, d_o, cu, hq, hkv, D, scale, rows=None):
+    """Full backward (or, with rows=[(seg,row),...], the sums restricted to those query rows).
+
+    Returns (dQ, dK, dV) as flat float64 arrays in the packed layout.
+    """
+    lib = _load()
+    cu, hq, hkv = _i32(cu), _i32(hq), _i32(hkv)
+    qe, kve, _ = layout_sizes(cu, hq, hkv, D)
+    dQ = np.zeros(qe, np.float64)
+    dK = np.zeros(kve, np.float64)
+    dV = np.zeros(kve, np.float64)
+    if rows is None:
+        rs = ri = None
+        n = 0
+    else:
+        rows = np.asarray(rows, dtype=np.int32).reshape(-1, 2)
+        rs, ri = _i32(rows[:, 0]), _i32(rows[:, 1])
+        n = len(rs)
+    rc = lib.orc_attn_bwd(_p(q), _p(k), _p(v), _p(d_o), ctypes.c_int(_dt(q)), _p(cu), _p(hq), _p(hkv),
+                          ctypes.c_int(len(hq)), ctypes.c_int(D), ctypes.c_double(scale), _p(rs), _p(ri),
+                          ctypes.c_int64(n), _p(dQ), _p(dK), _p(dV))
+    _check(rc, "attn_bwd")
+    return dQ, dK, dV
+
+
+def attn_rows(q, k, v, d_o, cu, hq, hkv, D, scale, samples):
+    """O, LSE, dQ for sampled (seg, q head, row) triples. d_o may be None (then dQ is None)."""
+    lib = _load()
+    cu, hq, hkv = _i32(cu), _i32(hq), _i32(hkv)
+    samples = np.asarray(samples, dtype=np.int32).reshape(-1, 3)
+    n = len(samples)
+    ss, sh, sr = _i32(samples[:, 0]), _i32(samples[:, 1]), _i32(samples[:, 2])
+    O = np.zeros((n, D), np.float64)
+    LSE = np.zeros(n, np.float64)
+    dQ = np.zeros((n, D), np.float64) if d_o is not None else None
+    rc = lib.orc_attn_rows(_p(q), _p(k), _p(v), _p(d_o), ctypes.c_int(_dt(q)), _p(cu), _p(hq), _p(hkv),
+                           ctypes.c_int(len(hq)), ctypes.c_int(D), ctypes.c_double(scale), ctypes.c_int64(n), _p(ss),
+                           _p(sh), _p(sr), _p(O), _p(LSE), _p(dQ))
+    _check(rc, "attn_rows")
+    return O, LSE, dQ
+
+
+def attn_cols(q, k, v, d_o, cu, hq, hkv, D, scale, samples):
+    """dK, dV for sampled (seg, kv head, column) triples under the full dO."""
+    lib = _load()
+    cu, hq, hkv = _i32(cu), _i32(hq), _i32(hkv)
+    samples = np.asarray(samples, dtype=np.int32).reshape(-1, 3)
+    n = len(samples)
+    ss, sh, sc = _i32(samples[:, 0]), _i32(samples[:, 1]), _i32(samples[:, 2])
+    dK = np.zeros((n, D), np.float64)
+    dV = np.zeros((n, D), np.float64)
+    rc = lib.orc_attn_cols(_p(q), _p(k), _p(v), _p(d_o), ctypes.c_int(_dt(q)), _p(cu), _p(hq), _p(hkv),
+                           ctypes.c_int(len(hq)), ctypes.c_int(D), ctypes.c_double(scale), ctypes.c_int64(n), _p(ss),
+                           _p(sh), _p(sc), _p(dK), _p(dV))
+    _check(rc, "attn_cols")
+    return dK, dV
+
+
+def plan_tiles(cu, hq, hkv, bm=128, bn=128, pass_=0):
+    """Sorted tile work list as an int32 array [n_items, 4] = (seg, head, tile, cost)."""
+    lib = _load()
+    cu, hq, hkv = _i32(cu), _i32(hq), _i32(hkv)
+    n = ctypes.c_int64(0)
+    rc = lib.orc_plan_tiles(_p(cu), _p(hq), _p(hkv), ctypes.c_int(len(hq)), ctypes.c_int(bm), ctypes.c_int(bn),
+                            ctypes.c_int(pass_), None, ctypes.c_int64(0), ctypes.byref(n))
+    _check(rc, "plan_tiles(size)")
+    out = np.zeros((max(n.value, 1), 4), np.int32)
+    rc = lib.orc_plan_tiles(_p(cu), _p(hq), _p(hkv), ctypes.c_int(len(hq)), ctypes.c_int(bm), ctypes.c_int(bn),
+                            ctypes.c_int(pass_), _p(out), ctypes.c_int64(n.value), ctypes.byref(n))
+    _check(rc, "plan_tiles")
+    return out[: n.value]
