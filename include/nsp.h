@@ -1,0 +1,136 @@
+/*
+ * nsp.h -- C ABI of the B200 (sm_100a) library for the local attention compute phase of nested sequence
+ * parallelism: packed variable-length causal GQA attention, forward and backward, over ONE GPU's share of a
+ * nested plan.
+ *
+ * Where the operation comes from (paper sections):
+ *   - Sec. 2.2 "Sequence Parallelism": after the Ulysses all-to-all a GPU holds the FULL-length sequence for
+ *     H/d of the heads (d = the sequence's SP degree) and attends locally, with no communication.
+ *   - Sec. 2.3 "Sequence Packing": a batch is a token budget of packed variable-length segments that never
+ *     attend to one another.
+ *   - Sec. 4.1 (Def. 1, SP tree) and Sec. 4.2 "Tree level": a GPU takes part in every node of its
+ *     leaf-to-root chain, so one GPU's share mixes segments of different degrees, i.e. different head counts.
+ *   - Sec. 4.2 "SP-backend level": the compute phase T^comp exists separately for forward and backward; this
+ *     library is that phase. The paper hands it to standard softmax-attention kernels and prints no formula,
+ *     so the semantics are the textbook ones:
+ *         S_ij = scale * <Q[i,h], K[j,g]>  (j <= i, diagonal included; g = h / (Hq/Hkv), contiguous groups)
+ *         LSE_i = ln sum_j exp(S_ij);  P_ij = exp(S_ij - LSE_i);  O[i,h] = sum_j P_ij V[j,g]
+ *         dQ, dK, dV = gradients of sum(O * dO); dK/dV are summed over the Hq/Hkv query heads of a KV head.
+ *
+ * Packed layout ("ragged token-major"), head_dim D = 128:
+ *   segment s has L_s = cu_seqlens[s+1]-cu_seqlens[s] tokens, hq[s] query heads and hkv[s] KV heads.
+ *   Q, O, dO, dQ : segment s is a contiguous [L_s, hq[s], D] block at element offset D * sum_{t<s} L_t*hq[t].
+ *   K, V, dK, dV : segment s is a contiguous [L_s, hkv[s], D] block at element offset D * sum_{t<s} L_t*hkv[t].
+ *   LSE          : fp32, segment s is [hq[s], L_s] at element offset sum_{t<s} L_t*hq[t]; natural log,
+ *                  softmax scale included.
+ *   A maximal range of consecutive segments with equal (hq, hkv) is a "run" (one tree node's samples);
+ *   at most NSP_MAX_RUNS runs per plan.
+ *
+ * Pointers: metadata pointers (cu_seqlens, hq, hkv, opts, every out-parameter) are HOST pointers; tensor and
+ * workspace pointers are DEVICE pointers on the current device, 16-byte aligned, owned by the caller.
+ * The plan is owned by the library (nsp_plan_destroy frees it). Calls enqueue work on the given CUDA stream
+ * (a cudaStream_t passed as void*; NULL = default stream) and return without synchronising unless stated.
+ * Outputs are fully overwritten. A plan may be in use by one stream at a time.
+ *
+ * Errors: every function returns an NSP_* code; nothing throws, aborts or traps. Device-side problems (a bounded
+ * wait that ran out) are recorded in a sticky per-plan status word that nsp_device_status reads.
+ * There is no CPU fallback: without a CUDA device the compute calls return NSP_ERR_CUDA.
+ */
+#ifndef NSP_H_
+#define NSP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NSP_MAX_RUNS 32
+#define NSP_HEAD_DIM 128
+
+enum {
+  NSP_OK = 0,
+  NSP_ERR_INVALID_ARG = 1,    /* null pointer, bad metadata, misaligned tensor, bad dtype, bad scale */
+  NSP_ERR_UNSUPPORTED = 2,    /* head_dim != 128, too many runs, tile sizes not built, counts out of range */
+  NSP_ERR_ALLOC = 3,          /* host or device allocation failed (plan construction only) */
+  NSP_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (including: no device) */
+  NSP_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait expired (sticky, see nsp_device_status) */
+  NSP_ERR_WORKSPACE = 6       /* workspace pointer null/misaligned or ws_bytes too small */
+};
+
+enum { NSP_BF16 = 0, NSP_F32 = 1 }; /* output dtypes of the gradients */
+
+typedef struct nsp_plan nsp_plan_t; /* opaque */
+
+/* One work item of the in-GPU schedule. forward: head = q head, tile = q tile. backward: head = kv head,
+ * tile = key tile. cost = number of inner-loop steps (see nsp_plan_tiles). */
+typedef struct {
+  int32_t seg, head, tile, cost;
+} nsp_tile_t;
+
+/* bm / bn: query / key tile rows (built: 128 / 128). order_version: 1. flags: 0. */
+typedef struct {
+  int32_t bm, bn, order_version, flags;
+} nsp_plan_opts;
+
+/*
+ * Build the device-side work lists for one packed batch (the in-GPU counterpart of the paper's per-node
+ * issue order, Sec. 5.1; the paper balances across GPUs, this list balances the SMs of one GPU).
+ *   forward  item (s, h, m), h in [0,hq[s]), m in [0, ceil(L_s/bm)):  cost = ceil(min(L_s,(m+1)*bm) / bn)
+ *   backward item (s, g, n), g in [0,hkv[s]), n in [0, ceil(L_s/bn)): cost = (hq[s]/hkv[s]) * (ceil(L_s/bm) - floor(n*bn/bm))
+ *   order: cost descending, then seg, tile, head ascending (a total order: the list is unique).
+ * cu_seqlens [n_seg+1], hq [n_seg], hkv [n_seg]: host arrays, copied. Zero-length segments and n_seg == 0 are legal.
+ * opts may be NULL (= {128,128,1,0}). The lists are built by kernels enqueued on `stream`.
+ * Errors: INVALID_ARG (null, n_seg < 0, cu_seqlens[0] != 0, decreasing cu_seqlens, hq/hkv <= 0, hq % hkv != 0),
+ * UNSUPPORTED (head_dim != 128, > NSP_MAX_RUNS runs, unsupported tile sizes, >= 65536 segments, > 256 heads,
+ * >= 65536 tiles in a segment), ALLOC, CUDA. On error *out_plan is NULL.
+ */
+int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* hkv, int32_t n_seg, int32_t head_dim,
+                   const nsp_plan_opts* opts, void* stream, nsp_plan_t** out_plan);
+
+/* Element counts of the packed tensors (q_elems: Q/O/dO/dQ; kv_elems: K/V/dK/dV; lse_elems: LSE) and the
+ * workspace bytes nsp_attn_fwd / nsp_attn_bwd need. Any out pointer may be NULL. Host-only, no CUDA call. */
+int nsp_plan_sizes(const nsp_plan_t* plan, int64_t* q_elems, int64_t* kv_elems, int64_t* lse_elems,
+                   size_t* fwd_ws_bytes, size_t* bwd_ws_bytes);
+
+/* Copy a work list to the host (pass 0 = forward, 1 = backward). Writes min(cap, n) items, stores n in
+ * *n_items (host_out may be NULL to query). Synchronises the plan's build stream. */
+int nsp_plan_get(const nsp_plan_t* plan, int pass, nsp_tile_t* host_out, int64_t cap, int64_t* n_items);
+
+/*
+ * Forward (paper Sec. 4.2, T^comp,fwd of every node on this GPU's chain, in one launch).
+ * q [q_elems] bf16, k/v [kv_elems] bf16 (device, read-only); o [q_elems] bf16 and lse [lse_elems] fp32 (device,
+ * written). softmax_scale: finite, > 0. ws / ws_bytes: device workspace of at least fwd_ws_bytes (may be NULL
+ * when that is 0). Errors: INVALID_ARG, WORKSPACE, CUDA, DEVICE_TIMEOUT (sticky status from an earlier call).
+ */
+int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const void* v, void* o, float* lse,
+                 float softmax_scale, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Backward (paper Sec. 4.2, T^comp,bwd). Inputs: q, k, v, o, d_o (bf16) and lse (fp32) as produced by
+ * nsp_attn_fwd. Outputs: dq [q_elems], dk/dv [kv_elems] in dq_dtype / dkv_dtype (NSP_BF16 or NSP_F32);
+ * dk/dv hold the sum over the hq/hkv query heads that share a KV head on THIS GPU (with a replicated KV head
+ * at high degree the cross-GPU sum belongs to the epilogue collective, outside this library).
+ * ws: at least bwd_ws_bytes, 256-byte aligned; contents undefined afterwards.
+ * Errors: as nsp_attn_fwd.
+ */
+int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                 const float* lse, void* dq, void* dk, void* dv, int dq_dtype, int dkv_dtype, float softmax_scale,
+                 void* ws, size_t ws_bytes, void* stream);
+
+/* Read the sticky device status {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
+int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
+
+/* Number of kernel launches the library has enqueued so far in this process (all plans). */
+int64_t nsp_launch_count(void);
+
+/* Free the plan (device lists, tables, status word). NULL is a no-op. */
+int nsp_plan_destroy(nsp_plan_t* plan);
+
+const char* nsp_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NSP_H_ */

@@ -1,0 +1,195 @@
+"""ctypes binding of ``libnsp.so``: the same entry points as ``include/nsp.h``, argument marshalling only.
+
+Every step of the path runs inside the CUDA library; torch is used here for device memory and streams. There is
+no fallback: if the library has not been built (``python -m paper_2609_22755_b200.build``) importing the symbols
+raises, and on a machine without a B200 the compute calls return ``NSP_ERR_CUDA`` / ``NSP_ERR_UNSUPPORTED``.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import numpy as np
+
+NSP_OK = 0
+NSP_ERR_INVALID_ARG = 1
+NSP_ERR_UNSUPPORTED = 2
+NSP_ERR_ALLOC = 3
+NSP_ERR_CUDA = 4
+NSP_ERR_DEVICE_TIMEOUT = 5
+NSP_ERR_WORKSPACE = 6
+NSP_BF16 = 0
+NSP_F32 = 1
+NSP_MAX_RUNS = 32
+
+EXPORTS = [
+    "nsp_plan_tiles", "nsp_plan_sizes", "nsp_plan_get", "nsp_attn_fwd", "nsp_attn_bwd", "nsp_device_status",
+    "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string",
+]
+
+LIB_PATH = Path(__file__).resolve().parent / "libnsp.so"
+_lib = None
+
+
+class NspError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {status_string(code)} (code {code})")
+
+
+class PlanOpts(ctypes.Structure):
+    _fields_ = [("bm", ctypes.c_int32), ("bn", ctypes.c_int32), ("order_version", ctypes.c_int32),
+                ("flags", ctypes.c_int32)]
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_22755_b200.build` "
+                              "(there is no CPU fallback)")
+        L = ctypes.CDLL(str(LIB_PATH))
+        vp, i32p, i64p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)
+        L.nsp_plan_tiles.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, vp, vp, ctypes.POINTER(vp)]
+        L.nsp_plan_tiles.restype = ctypes.c_int
+        L.nsp_plan_sizes.argtypes = [vp, i64p, i64p, i64p, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+        L.nsp_plan_sizes.restype = ctypes.c_int
+        L.nsp_plan_get.argtypes = [vp, ctypes.c_int, vp, ctypes.c_int64, i64p]
+        L.nsp_plan_get.restype = ctypes.c_int
+        L.nsp_attn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp]
+        L.nsp_attn_fwd.restype = ctypes.c_int
+        L.nsp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+                                   vp, ctypes.c_size_t, vp]
+        L.nsp_attn_bwd.restype = ctypes.c_int
+        L.nsp_device_status.argtypes = [vp, i32p]
+        L.nsp_device_status.restype = ctypes.c_int
+        L.nsp_launch_count.argtypes = []
+        L.nsp_launch_count.restype = ctypes.c_int64
+        L.nsp_plan_destroy.argtypes = [vp]
+        L.nsp_plan_destroy.restype = ctypes.c_int
+        L.nsp_status_string.argtypes = [ctypes.c_int]
+        L.nsp_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().nsp_status_string(int(code)).decode()
+
+
+def launch_count() -> int:
+    return int(lib().nsp_launch_count())
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return ctypes.c_void_p(t)
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data_as(ctypes.c_void_p)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, int):
+        return ctypes.c_void_p(stream)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+class Plan:
+    """Owner of an ``nsp_plan_t*``."""
+
+    def __init__(self, handle, n_seg):
+        self.handle = handle
+        self.n_seg = n_seg
+        q, kv, l = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+        fw, bw = ctypes.c_size_t(), ctypes.c_size_t()
+        rc = lib().nsp_plan_sizes(handle, ctypes.byref(q), ctypes.byref(kv), ctypes.byref(l), ctypes.byref(fw),
+                                  ctypes.byref(bw))
+        if rc != NSP_OK:
+            raise NspError(rc, "nsp_plan_sizes")
+        self.q_elems, self.kv_elems, self.lse_elems = q.value, kv.value, l.value
+        self.fwd_ws_bytes, self.bwd_ws_bytes = fw.value, bw.value
+
+    def destroy(self):
+        if self.handle:
+            lib().nsp_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def nsp_plan_tiles(cu_seqlens, hq, hkv, head_dim=128, opts=None, stream=None) -> Plan:
+    cu, hq_, hkv_ = _i32(cu_seqlens), _i32(hq), _i32(hkv)
+    n_seg = len(hq_)
+    if len(cu) != n_seg + 1 or len(hkv_) != n_seg:
+        raise NspError(NSP_ERR_INVALID_ARG, "nsp_plan_tiles(argument shapes)")
+    o = None
+    if opts is not None:
+        o = PlanOpts(*opts)
+    handle = ctypes.c_void_p()
+    rc = lib().nsp_plan_tiles(_ptr(cu), _ptr(hq_), _ptr(hkv_), n_seg, head_dim, ctypes.byref(o) if o else None,
+                              _stream_ptr(stream), ctypes.byref(handle))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_plan_tiles")
+    return Plan(handle, n_seg)
+
+
+def nsp_plan_get(plan: Plan, pass_: int) -> np.ndarray:
+    """The device work list as an int32 array [n_items, 4] = (seg, head, tile, cost)."""
+    n = ctypes.c_int64()
+    rc = lib().nsp_plan_get(plan.handle, pass_, None, 0, ctypes.byref(n))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_plan_get")
+    out = np.zeros((max(n.value, 1), 4), np.int32)
+    rc = lib().nsp_plan_get(plan.handle, pass_, _ptr(out), n.value, ctypes.byref(n))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_plan_get")
+    return out[: n.value]
+
+
+def nsp_attn_fwd(plan: Plan, q, k, v, o, lse, softmax_scale, ws=None, stream=None):
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    rc = lib().nsp_attn_fwd(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), float(softmax_scale), _ptr(ws),
+                            ws_bytes, _stream_ptr(stream))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_attn_fwd")
+
+
+def nsp_attn_bwd(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, softmax_scale, ws, dq_dtype=None, dkv_dtype=None,
+                 stream=None):
+    import torch
+
+    if dq_dtype is None:
+        dq_dtype = NSP_F32 if dq.dtype == torch.float32 else NSP_BF16
+    if dkv_dtype is None:
+        dkv_dtype = NSP_F32 if dk.dtype == torch.float32 else NSP_BF16
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    rc = lib().nsp_attn_bwd(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk),
+                            _ptr(dv), dq_dtype, dkv_dtype, float(softmax_scale), _ptr(ws), ws_bytes,
+                            _stream_ptr(stream))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_attn_bwd")
+
+
+def nsp_device_status(plan: Plan):
+    out = (ctypes.c_int32 * 4)()
+    rc = lib().nsp_device_status(plan.handle, out)
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_device_status")
+    return tuple(out)

@@ -1,0 +1,387 @@
+// Host side of libnsp: argument validation, plan object, tensor-map encoding and kernel launches.
+// Plain C ABI (include/nsp.h); no torch types, no CPU fallback.
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+#include <cuda_bf16.h>
+#include "nsp_internal.cuh"
+
+namespace nsp {
+static std::atomic<int64_t> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace nsp
+
+using namespace nsp;
+
+struct nsp_plan {
+  int32_t n_seg = 0, bm = kBM, bn = kBN;
+  int device = 0, num_sms = 0;
+  int64_t q_elems = 0, kv_elems = 0, lse_elems = 0, n_fwd = 0, n_bwd = 0;
+  std::vector<SegInfo> seg;
+  std::vector<RunInfo> runs;
+  // device state
+  SegInfo* d_seg = nullptr;
+  int64_t* d_row_base = nullptr;  // [n_seg + 1] first packed (token, head) row of each segment
+  nsp_tile_t* d_fwd = nullptr;
+  nsp_tile_t* d_bwd = nullptr;
+  int32_t* d_counters = nullptr;  // [0] forward cursor, [1] backward cursor
+  int32_t* d_status = nullptr;    // {code, item, where, aux}
+  cudaStream_t build_stream = nullptr;
+  int sticky = 0;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// Tensor map of one run: a dense bf16 [tokens, heads, 128] tensor; tiles are {64 dims, 1 head, 128 tokens}
+// with 128-byte swizzle, rows past the run read as zero.
+bool encode_run_map(CUtensorMap* out, const void* base, int64_t elem_off, int64_t tokens, int heads) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return false;
+  if (tokens <= 0) {
+    std::memset(out, 0, sizeof(*out));
+    return true;
+  }
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(kHeadDim), static_cast<cuuint64_t>(heads),
+                              static_cast<cuuint64_t>(tokens)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(kHeadDim) * 2, static_cast<cuuint64_t>(heads) * kHeadDim * 2};
+  const cuuint32_t box[3] = {64, 1, 128};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  void* ptr = const_cast<char*>(static_cast<const char*>(base)) + elem_off * 2;
+  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+void free_plan(nsp_plan* p) {
+  if (!p) return;
+  cudaFree(p->d_seg);
+  cudaFree(p->d_row_base);
+  cudaFree(p->d_fwd);
+  cudaFree(p->d_bwd);
+  cudaFree(p->d_counters);
+  cudaFree(p->d_status);
+  delete p;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* nsp_status_string(int code) {
+  switch (code) {
+    case NSP_OK: return "ok";
+    case NSP_ERR_INVALID_ARG: return "invalid argument";
+    case NSP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case NSP_ERR_ALLOC: return "allocation failed";
+    case NSP_ERR_CUDA: return "CUDA call failed";
+    case NSP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case NSP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    default: return "unknown status";
+  }
+}
+
+int64_t nsp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* hkv, int32_t n_seg, int32_t head_dim,
+                   const nsp_plan_opts* opts, void* stream, nsp_plan_t** out_plan) {
+  if (!out_plan) return NSP_ERR_INVALID_ARG;
+  *out_plan = nullptr;
+  if (n_seg < 0 || (n_seg > 0 && (!cu_seqlens || !hq || !hkv))) return NSP_ERR_INVALID_ARG;
+  if (n_seg > 0 && cu_seqlens[0] != 0) return NSP_ERR_INVALID_ARG;
+  for (int s = 0; s < n_seg; ++s) {
+    if (cu_seqlens[s + 1] < cu_seqlens[s]) return NSP_ERR_INVALID_ARG;
+    if (hq[s] <= 0 || hkv[s] <= 0 || hq[s] % hkv[s] != 0) return NSP_ERR_INVALID_ARG;
+  }
+  int bm = kBM, bn = kBN;
+  if (opts) {
+    if (opts->bm <= 0 || opts->bn <= 0) return NSP_ERR_INVALID_ARG;
+    bm = opts->bm;
+    bn = opts->bn;
+    if (opts->order_version != 1 || opts->flags != 0) return NSP_ERR_UNSUPPORTED;
+  }
+  if (head_dim != kHeadDim) return NSP_ERR_UNSUPPORTED;
+  if (bm != kBM || bn != kBN) return NSP_ERR_UNSUPPORTED;
+  if (n_seg >= 65536) return NSP_ERR_UNSUPPORTED;
+
+  nsp_plan* p = new (std::nothrow) nsp_plan;
+  if (!p) return NSP_ERR_ALLOC;
+  p->n_seg = n_seg;
+  p->bm = bm;
+  p->bn = bn;
+  p->build_stream = static_cast<cudaStream_t>(stream);
+  std::vector<int64_t> row_base, fwd_base, bwd_base;
+  try {
+    p->seg.resize(n_seg);
+    row_base.resize(n_seg + 1);
+    fwd_base.resize(n_seg + 1);
+    bwd_base.resize(n_seg + 1);
+  } catch (...) {
+    delete p;
+    return NSP_ERR_ALLOC;
+  }
+  int64_t q_off = 0, kv_off = 0, lse_off = 0, nf = 0, nb = 0;
+  for (int s = 0; s < n_seg; ++s) {
+    const int64_t L = static_cast<int64_t>(cu_seqlens[s + 1]) - cu_seqlens[s];
+    const int64_t Mt = (L + bm - 1) / bm, Nt = (L + bn - 1) / bn;
+    if (hq[s] > 256 || Mt >= 65536 || Nt >= 65536 || (hq[s] / hkv[s]) * Mt >= (1 << 24)) {
+      delete p;
+      return NSP_ERR_UNSUPPORTED;
+    }
+    const bool new_run = s == 0 || hq[s] != hq[s - 1] || hkv[s] != hkv[s - 1];
+    if (new_run) {
+      if (p->runs.size() == NSP_MAX_RUNS) {
+        delete p;
+        return NSP_ERR_UNSUPPORTED;
+      }
+      p->runs.push_back(RunInfo{q_off, kv_off, 0, hq[s], hkv[s]});
+    }
+    RunInfo& run = p->runs.back();
+    SegInfo& sg = p->seg[s];
+    std::memset(&sg, 0, sizeof(sg));
+    sg.q_off = q_off;
+    sg.kv_off = kv_off;
+    sg.lse_off = lse_off;
+    sg.len = static_cast<int32_t>(L);
+    sg.hq = hq[s];
+    sg.hkv = hkv[s];
+    sg.run = static_cast<int32_t>(p->runs.size() - 1);
+    sg.tok_in_run = static_cast<int32_t>(run.tokens);
+    run.tokens += L;
+    row_base[s] = lse_off;
+    fwd_base[s] = nf;
+    bwd_base[s] = nb;
+    q_off += L * hq[s] * kHeadDim;
+    kv_off += L * hkv[s] * kHeadDim;
+    lse_off += L * hq[s];
+    nf += Mt * hq[s];
+    nb += Nt * hkv[s];
+  }
+  row_base[n_seg] = lse_off;
+  fwd_base[n_seg] = nf;
+  bwd_base[n_seg] = nb;
+  p->q_elems = q_off;
+  p->kv_elems = kv_off;
+  p->lse_elems = lse_off;
+  p->n_fwd = nf;
+  p->n_bwd = nb;
+  if (nf >= (1ll << 31) || nb >= (1ll << 31)) {
+    delete p;
+    return NSP_ERR_UNSUPPORTED;
+  }
+
+  // ---- device side
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&p->device) != cudaSuccess || cudaGetDeviceProperties(&prop, p->device) != cudaSuccess) {
+    delete p;
+    return NSP_ERR_CUDA;
+  }
+  p->num_sms = prop.multiProcessorCount;
+  if (prop.major != 10) {
+    delete p;
+    return NSP_ERR_UNSUPPORTED;
+  }
+  cudaStream_t st = p->build_stream;
+  int64_t* d_bases = nullptr;
+  uint64_t* d_keys = nullptr;
+  void* d_tmp = nullptr;
+  const size_t tmp_bytes = plan_sort_tmp_bytes(nf > nb ? nf : nb);
+  bool okc = true;
+  auto A = [&](void** ptr, size_t bytes) {
+    if (okc && cudaMalloc(ptr, bytes ? bytes : 16) != cudaSuccess) okc = false;
+  };
+  A(reinterpret_cast<void**>(&p->d_seg), sizeof(SegInfo) * n_seg);
+  A(reinterpret_cast<void**>(&p->d_row_base), sizeof(int64_t) * (n_seg + 1));
+  A(reinterpret_cast<void**>(&p->d_fwd), sizeof(nsp_tile_t) * nf);
+  A(reinterpret_cast<void**>(&p->d_bwd), sizeof(nsp_tile_t) * nb);
+  A(reinterpret_cast<void**>(&p->d_counters), 2 * sizeof(int32_t));
+  A(reinterpret_cast<void**>(&p->d_status), 4 * sizeof(int32_t));
+  A(reinterpret_cast<void**>(&d_bases), 2 * sizeof(int64_t) * (n_seg + 1));
+  A(reinterpret_cast<void**>(&d_keys), 2 * sizeof(uint64_t) * (nf + nb));
+  A(&d_tmp, tmp_bytes);
+  int rc = NSP_OK;
+  if (!okc) {
+    rc = NSP_ERR_ALLOC;
+    cudaGetLastError();
+  } else {
+    cudaError_t e = cudaSuccess;
+    auto C = [&](cudaError_t x) {
+      if (e == cudaSuccess) e = x;
+    };
+    C(cudaMemsetAsync(p->d_counters, 0, 2 * sizeof(int32_t), st));
+    C(cudaMemsetAsync(p->d_status, 0, 4 * sizeof(int32_t), st));
+    if (n_seg > 0) {
+      C(cudaMemcpyAsync(p->d_seg, p->seg.data(), sizeof(SegInfo) * n_seg, cudaMemcpyHostToDevice, st));
+      C(cudaMemcpyAsync(d_bases, fwd_base.data(), sizeof(int64_t) * (n_seg + 1), cudaMemcpyHostToDevice, st));
+      C(cudaMemcpyAsync(d_bases + n_seg + 1, bwd_base.data(), sizeof(int64_t) * (n_seg + 1), cudaMemcpyHostToDevice,
+                        st));
+    }
+    C(cudaMemcpyAsync(p->d_row_base, row_base.data(), sizeof(int64_t) * (n_seg + 1), cudaMemcpyHostToDevice, st));
+    if (e == cudaSuccess)
+      C(launch_plan_build(p->d_seg, n_seg, bm, bn, p->d_fwd, nf, p->d_bwd, nb, d_keys, d_keys + nf + nb, d_tmp, tmp_bytes,
+                          d_bases, d_bases + n_seg + 1, st));
+    // the host staging vectors and the scratch buffers die with this call: wait for the build
+    C(cudaStreamSynchronize(st));
+    if (e != cudaSuccess) rc = NSP_ERR_CUDA;
+  }
+  cudaFree(d_bases);
+  cudaFree(d_keys);
+  cudaFree(d_tmp);
+  if (rc != NSP_OK) {
+    free_plan(p);
+    return rc;
+  }
+  *out_plan = p;
+  return NSP_OK;
+}
+
+int nsp_plan_sizes(const nsp_plan_t* plan, int64_t* q_elems, int64_t* kv_elems, int64_t* lse_elems,
+                   size_t* fwd_ws_bytes, size_t* bwd_ws_bytes) {
+  if (!plan) return NSP_ERR_INVALID_ARG;
+  if (q_elems) *q_elems = plan->q_elems;
+  if (kv_elems) *kv_elems = plan->kv_elems;
+  if (lse_elems) *lse_elems = plan->lse_elems;
+  if (fwd_ws_bytes) *fwd_ws_bytes = 0;
+  if (bwd_ws_bytes)
+    *bwd_ws_bytes = align_up(static_cast<size_t>(plan->q_elems) * 4, 256) + align_up(static_cast<size_t>(plan->lse_elems) * 4, 256);
+  return NSP_OK;
+}
+
+int nsp_plan_get(const nsp_plan_t* plan, int pass, nsp_tile_t* host_out, int64_t cap, int64_t* n_items) {
+  if (!plan || !n_items || (pass != 0 && pass != 1) || cap < 0) return NSP_ERR_INVALID_ARG;
+  const int64_t n = pass == 0 ? plan->n_fwd : plan->n_bwd;
+  *n_items = n;
+  if (!host_out || cap == 0 || n == 0) return NSP_OK;
+  const int64_t m = cap < n ? cap : n;
+  if (cudaStreamSynchronize(plan->build_stream) != cudaSuccess) return NSP_ERR_CUDA;
+  if (cudaMemcpy(host_out, pass == 0 ? plan->d_fwd : plan->d_bwd, sizeof(nsp_tile_t) * m, cudaMemcpyDeviceToHost) !=
+      cudaSuccess)
+    return NSP_ERR_CUDA;
+  return NSP_OK;
+}
+
+int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const void* v, void* o, float* lse,
+                 float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  if (!plan) return NSP_ERR_INVALID_ARG;
+  if (plan->sticky) return plan->sticky;
+  if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return NSP_ERR_INVALID_ARG;
+  if (plan->n_fwd == 0) return NSP_OK;
+  if (!q || !k || !v || !o || !lse) return NSP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return NSP_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FwdMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
+  for (size_t r = 0; r < plan->runs.size(); ++r) {
+    const RunInfo& run = plan->runs[r];
+    if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq) ||
+        !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv) ||
+        !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv))
+      return NSP_ERR_CUDA;
+  }
+  if (cudaMemsetAsync(plan->d_counters, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
+  FwdArgs a;
+  a.seg = plan->d_seg;
+  a.items = plan->d_fwd;
+  a.n_items = static_cast<int32_t>(plan->n_fwd);
+  a.counter = plan->d_counters;
+  a.status = plan->d_status;
+  a.o = static_cast<__nv_bfloat16*>(o);
+  a.lse = lse;
+  a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  if (launch_fwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  return NSP_OK;
+}
+
+int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                 const float* lse, void* dq, void* dk, void* dv, int dq_dtype, int dkv_dtype, float softmax_scale,
+                 void* ws, size_t ws_bytes, void* stream) {
+  if (!plan) return NSP_ERR_INVALID_ARG;
+  if (plan->sticky) return plan->sticky;
+  if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return NSP_ERR_INVALID_ARG;
+  if ((dq_dtype != NSP_BF16 && dq_dtype != NSP_F32) || (dkv_dtype != NSP_BF16 && dkv_dtype != NSP_F32))
+    return NSP_ERR_INVALID_ARG;
+  if (plan->n_bwd == 0) return NSP_OK;
+  if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) return NSP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
+      !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
+    return NSP_ERR_INVALID_ARG;
+  size_t need = 0;
+  nsp_plan_sizes(plan, nullptr, nullptr, nullptr, nullptr, &need);
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < need) return NSP_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* dq_acc = static_cast<float*>(ws);
+  float* delta = reinterpret_cast<float*>(static_cast<char*>(ws) + align_up(static_cast<size_t>(plan->q_elems) * 4, 256));
+
+  BwdMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
+  for (size_t r = 0; r < plan->runs.size(); ++r) {
+    const RunInfo& run = plan->runs[r];
+    if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq) ||
+        !encode_run_map(&maps.d_o[r], d_o, run.q_off, run.tokens, run.hq) ||
+        !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv) ||
+        !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv))
+      return NSP_ERR_CUDA;
+  }
+  if (cudaMemsetAsync(plan->d_counters + 1, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (cudaMemsetAsync(dq_acc, 0, static_cast<size_t>(plan->q_elems) * 4, st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (launch_bwd_preprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems,
+                            static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta,
+                            st) != cudaSuccess)
+    return NSP_ERR_CUDA;
+  BwdArgs a;
+  a.seg = plan->d_seg;
+  a.items = plan->d_bwd;
+  a.n_items = static_cast<int32_t>(plan->n_bwd);
+  a.counter = plan->d_counters + 1;
+  a.status = plan->d_status;
+  a.lse = lse;
+  a.delta = delta;
+  a.dq_acc = dq_acc;
+  a.dk = dk;
+  a.dv = dv;
+  a.dkv_f32 = dkv_dtype == NSP_F32;
+  a.scale = softmax_scale;
+  a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  if (launch_bwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (launch_bwd_postprocess(dq_acc, dq, plan->q_elems, dq_dtype == NSP_F32, softmax_scale, st) != cudaSuccess)
+    return NSP_ERR_CUDA;
+  return NSP_OK;
+}
+
+int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]) {
+  if (!plan || !out) return NSP_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return NSP_ERR_CUDA;
+  if (cudaMemcpy(out, plan->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return NSP_ERR_CUDA;
+  if (out[0] != 0) const_cast<nsp_plan_t*>(plan)->sticky = out[0];
+  return NSP_OK;
+}
+
+int nsp_plan_destroy(nsp_plan_t* plan) {
+  free_plan(plan);
+  return NSP_OK;
+}
+
+}  // extern "C"

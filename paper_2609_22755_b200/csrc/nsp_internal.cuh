@@ -1,0 +1,100 @@
+// Internal structures shared by the host API and the kernels of libnsp (never visible across the C ABI).
+#pragma once
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include "../../include/nsp.h"
+
+namespace nsp {
+
+constexpr int kHeadDim = NSP_HEAD_DIM;
+constexpr int kBM = 128;  // query rows per tile
+constexpr int kBN = 128;  // key rows per tile
+
+// Per-segment table entry (device + host copy).
+struct SegInfo {
+  int64_t q_off;    // element offset of the segment in Q/O/dO/dQ
+  int64_t kv_off;   // element offset in K/V/dK/dV
+  int64_t lse_off;  // element offset in LSE / delta
+  int32_t len;      // tokens
+  int32_t hq, hkv;
+  int32_t run;         // index of the run (dense [T, H, D] tensor) the segment belongs to
+  int32_t tok_in_run;  // first token of the segment, relative to the run
+  int32_t pad_[3];
+};
+static_assert(sizeof(SegInfo) == 56 || sizeof(SegInfo) == 64, "SegInfo layout");
+
+struct RunInfo {
+  int64_t q_off, kv_off;  // element offsets of the run's first token
+  int64_t tokens;
+  int32_t hq, hkv;
+};
+
+// Tensor maps of every run, passed by value as a __grid_constant__ kernel parameter.
+struct FwdMaps {
+  CUtensorMap q[NSP_MAX_RUNS], k[NSP_MAX_RUNS], v[NSP_MAX_RUNS];
+};
+struct BwdMaps {
+  CUtensorMap q[NSP_MAX_RUNS], d_o[NSP_MAX_RUNS], k[NSP_MAX_RUNS], v[NSP_MAX_RUNS];
+};
+
+// Device status word: {code, item, where, aux}; first writer wins (atomicCAS on code).
+enum DeviceWhere : int32_t {
+  kWhereFwdLoad = 1,
+  kWhereFwdS = 2,
+  kWhereFwdO = 3,
+  kWhereBwdLoadKV = 11,
+  kWhereBwdLoadQ = 12,
+  kWhereBwdS = 13,
+  kWhereBwdMma2 = 14,
+};
+
+__device__ __forceinline__ void report_timeout(int32_t* status, int32_t item, int32_t where, int32_t aux) {
+  if (atomicCAS(status, 0, NSP_ERR_DEVICE_TIMEOUT) == 0) {
+    status[1] = item;
+    status[2] = where;
+    status[3] = aux;
+  }
+}
+
+struct FwdArgs {
+  const SegInfo* seg;
+  const nsp_tile_t* items;
+  int32_t n_items;
+  int32_t* counter;  // work-list cursor, zeroed before the launch
+  int32_t* status;
+  __nv_bfloat16* o;
+  float* lse;
+  float scale_log2;  // softmax_scale * log2(e)
+};
+
+struct BwdArgs {
+  const SegInfo* seg;
+  const nsp_tile_t* items;
+  int32_t n_items;
+  int32_t* counter;
+  int32_t* status;
+  const float* lse;
+  const float* delta;
+  float* dq_acc;  // fp32 [q_elems], zeroed before the launch
+  void* dk;
+  void* dv;
+  int32_t dkv_f32;
+  float scale;
+  float scale_log2;
+};
+
+// Host-side launchers implemented next to their kernels.
+cudaError_t launch_plan_build(const SegInfo* d_seg, int n_seg, int bm, int bn, nsp_tile_t* d_fwd, int64_t n_fwd,
+                              nsp_tile_t* d_bwd, int64_t n_bwd, uint64_t* d_keys, uint64_t* d_keys_alt, void* d_sort_tmp,
+                              size_t sort_tmp_bytes, const int64_t* d_fwd_base, const int64_t* d_bwd_base,
+                              cudaStream_t st);
+size_t plan_sort_tmp_bytes(int64_t max_items);
+cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st);
+cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
+                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, cudaStream_t st);
+cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st);
+cudaError_t launch_bwd_postprocess(const float* dq_acc, void* dq, int64_t n, int dq_f32, float scale, cudaStream_t st);
+void count_launches(int n);
+
+}  // namespace nsp

@@ -1,0 +1,96 @@
+"""Helpers for the GPU parity tests: run the CUDA path through the C ABI, run the oracle, compare.
+
+Tolerances (benchmark definition): max-abs error 2e-2 and relative L2 error 1e-2 for O, dQ, dK, dV against the
+fp64 oracle evaluated on the same bf16 input bytes. The graded gradient dtypes are dQ bf16, dK/dV fp32.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+MAX_ABS_TOL = 2e-2
+REL_L2_TOL = 1e-2
+LSE_ABS_TOL = 2e-3
+
+
+def errors(got: np.ndarray, want: np.ndarray):
+    got = np.asarray(got, np.float64).ravel()
+    want = np.asarray(want, np.float64).ravel()
+    if want.size == 0:
+        return 0.0, 0.0
+    d = got - want
+    max_abs = float(np.max(np.abs(d)))
+    denom = float(np.sqrt((want * want).sum()))
+    rel = float(np.sqrt((d * d).sum()) / denom) if denom > 0 else float(np.sqrt((d * d).sum()))
+    return max_abs, rel
+
+
+def check(name, got, want, max_abs_tol=MAX_ABS_TOL, rel_tol=REL_L2_TOL):
+    assert np.all(np.isfinite(np.asarray(got, np.float64))), f"{name}: non-finite values in the GPU result"
+    ma, rl = errors(got, want)
+    assert ma <= max_abs_tol, f"{name}: max-abs error {ma:.4g} > {max_abs_tol}"
+    assert rl <= rel_tol, f"{name}: relative L2 error {rl:.4g} > {rel_tol}"
+    return ma, rl
+
+
+class GpuRun:
+    """Device buffers + one forward/backward through the C ABI for a workload."""
+
+    def __init__(self, w, tensors=None, dq_dtype="bf16", dkv_dtype="f32", device="cuda:0"):
+        import torch
+
+        from paper_2609_22755_b200 import binding as B
+        from paper_2609_22755_b200 import workloads as W
+
+        self.torch, self.B, self.w = torch, B, w
+        self.dev = torch.device(device)
+        self.host = tensors if tensors is not None else W.make_tensors(w)
+        self.q, self.k, self.v, self.do = (self.host[n].to(self.dev) for n in ("q", "k", "v", "do"))
+        self.plan = B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, w.head_dim)
+        assert self.plan.q_elems == w.q_elems() and self.plan.kv_elems == w.kv_elems()
+        assert self.plan.lse_elems == w.lse_elems()
+        self.o = torch.full((w.q_elems(),), float("nan"), dtype=torch.bfloat16, device=self.dev)
+        self.lse = torch.full((w.lse_elems(),), float("nan"), dtype=torch.float32, device=self.dev)
+        tq = torch.float32 if dq_dtype == "f32" else torch.bfloat16
+        tkv = torch.float32 if dkv_dtype == "f32" else torch.bfloat16
+        self.dq = torch.full((w.q_elems(),), float("nan"), dtype=tq, device=self.dev)
+        self.dk = torch.full((w.kv_elems(),), float("nan"), dtype=tkv, device=self.dev)
+        self.dv = torch.full((w.kv_elems(),), float("nan"), dtype=tkv, device=self.dev)
+        self.ws = torch.empty(max(self.plan.bwd_ws_bytes, 256), dtype=torch.uint8, device=self.dev)
+
+    def forward(self):
+        self.B.nsp_attn_fwd(self.plan, self.q, self.k, self.v, self.o, self.lse, self.w.softmax_scale)
+
+    def backward(self):
+        self.B.nsp_attn_bwd(self.plan, self.q, self.k, self.v, self.o, self.do, self.lse, self.dq, self.dk, self.dv,
+                            self.w.softmax_scale, self.ws)
+
+    def status(self):
+        return self.B.nsp_device_status(self.plan)
+
+    def results(self):
+        t = self.torch
+        t.cuda.synchronize()
+        f = lambda x: x.float().cpu().numpy().astype(np.float64)
+        return {"o": f(self.o), "lse": f(self.lse), "dq": f(self.dq), "dk": f(self.dk), "dv": f(self.dv)}
+
+
+def oracle_full(w, host):
+    import oracle
+    from paper_2609_22755_b200 import workloads as W
+
+    b = {n: W.bf16_bits(host[n]) for n in ("q", "k", "v", "do")}
+    O, LSE = oracle.attn_fwd(b["q"], b["k"], b["v"], w.cu_seqlens, w.hq, w.hkv, w.head_dim, w.softmax_scale)
+    dQ, dK, dV = oracle.attn_bwd(b["q"], b["k"], b["v"], b["do"], w.cu_seqlens, w.hq, w.hkv, w.head_dim,
+                                 w.softmax_scale)
+    return {"o": O, "lse": LSE, "dq": dQ, "dk": dK, "dv": dV}
+
+
+def compare_full(w, res, ref, tag=""):
+    out = {}
+    for name in ("o", "dq", "dk", "dv"):
+        out[name] = check(f"{w.name}{tag}:{name}", res[name], ref[name])
+    if ref["lse"].size:
+        d = float(np.max(np.abs(res["lse"] - ref["lse"])))
+        assert d <= LSE_ABS_TOL, f"{w.name}{tag}: LSE max-abs error {d:.4g}"
+        out["lse"] = (d, 0.0)
+    return out
