@@ -86,15 +86,15 @@ def attn_fwd(q, k, v, cu, hq, hkv, D, scale):
     return O, LSE
 
 
-def attn_bwd(q, k, v, d_o, cu, hq, hkv, D, scale, rows=None):
+def attn_bwd(q, k, v, d_o, cu, hq, hkv, D, scale, rows=None, want_dq=True):
     """Full backward (or, with rows=[(seg,row),...], the sums restricted to those query rows).
 
-    Returns (dQ, dK, dV) as flat float64 arrays in the packed layout.
+    Returns (dQ, dK, dV) as flat float64 arrays in the packed layout (dQ is None when want_dq is False).
     """
     lib = _load()
     cu, hq, hkv = _i32(cu), _i32(hq), _i32(hkv)
     qe, kve, _ = layout_sizes(cu, hq, hkv, D)
-    dQ = np.zeros(qe, np.float64)
+    dQ = np.zeros(qe, np.float64) if want_dq else None
     dK = np.zeros(kve, np.float64)
     dV = np.zeros(kve, np.float64)
     if rows is None:

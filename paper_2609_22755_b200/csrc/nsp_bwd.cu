@@ -14,6 +14,8 @@
 //     dV  += P^T dO                               A = P^T (bf16, TMEM), B = dO  MN-major
 //     dK  += dS^T Q                               A = dS^T (shared, K-major), B = Q MN-major
 //     dQ_m = dS K                                 A = dS^T read MN-major, B = K MN-major   -> TMEM (over S^T)
+// For the first q tile of a segment (rows 0..127, where P is O(1)) P^T and dS^T are split into hi + lo bf16
+// parts and every product is issued twice; this keeps dK/dV/dQ inside the 2e-2 max-abs tolerance.
 // dK and dV accumulate in TMEM over the whole item, in a fixed order (heads ascending, tiles ascending), so
 // the reduction over the query heads of a group is deterministic. dQ tiles are added to an fp32 accumulator
 // in global memory with vector reductions.
@@ -36,8 +38,10 @@ struct BwdSmem {
   uint8_t q[2][kHalfTileBytes];
   uint8_t d_o[2][kHalfTileBytes];
   uint8_t ds[2][kHalfTileBytes];  // dS^T, [key row][query col], split in two 64-column halves
+  uint8_t ds_lo[2][kHalfTileBytes];  // bf16 residual of dS^T (first q tile of a segment only)
   float lse[128];                 // LSE * log2(e) of the current q tile (+inf for rows past the segment)
   float delta[128];
+  float part[4][128];             // per-quadrant partial sums of the exact delta (first q tile only)
   uint64_t bar_kv, bar_qdo, bar_s, bar_m2;
   uint32_t tmem_base;
   int32_t item_idx;
@@ -73,7 +77,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   const uint32_t tS = s.tmem_base, tDP = tS + 128, tDK = tS + 256, tDV = tS + 384;
   const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
   const uint32_t k_addr = smem_u32(s.k[0]), v_addr = smem_u32(s.v[0]), q_addr = smem_u32(s.q[0]),
-                 do_addr = smem_u32(s.d_o[0]), ds_addr = smem_u32(s.ds[0]);
+                 do_addr = smem_u32(s.d_o[0]), ds_addr = smem_u32(s.ds[0]), dsl_addr = smem_u32(s.ds_lo[0]);
   constexpr uint32_t idesc_kk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
   constexpr uint32_t idesc_kn = make_idesc_bf16(128, 128, 0, 1);  // A K-major (or TMEM), B MN-major
   constexpr uint32_t idesc_nn = make_idesc_bf16(128, 128, 1, 1);  // A MN-major, B MN-major
@@ -153,13 +157,41 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         else
           s.delta[tid - 128] = valid ? a.delta[idx] : 0.f;
       }
-      __syncthreads();
       bool okw = mbar_wait(&s.bar_s, ph_s);
       ph_s ^= 1;
-      okw = __all_sync(0xffffffffu, okw);
-      if (okw) {
+      if (!okw && lane == 0) report_timeout(a.status, it, kWhereBwdS, t);
+      ok = __syncthreads_and(ok && okw);  // also publishes s.lse / s.delta
+      if (!ok) break;
+      {
         tc_fence_after_sync();
         const bool diag = (m == n);
+        // First q tile of a segment: P and dS are O(1) there and their bf16 rounding dominates the error of
+        // dK/dV/dQ, so they are fed to the tensor core as hi + lo bf16 pairs (two MMAs per product), and
+        // delta_i is recomputed as sum_j P_ij dP_ij in fp32 (all keys of these rows lie in this key tile)
+        // instead of taking it from the bf16-rounded O.
+        const bool hilo = (m == 0);
+        if (hilo) {
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const int col0 = half * 64 + c * 32;
+            uint32_t sv[32], dpv[32];
+            tmem_ld32(tS + lane_off + col0, sv);
+            tmem_ld32(tDP + lane_off + col0, dpv);
+            tmem_wait_ld();
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+              float p = ex2f(fmaf(__uint_as_float(sv[x]), a.scale_log2, -s.lse[col0 + x]));
+              if (col0 + x < r) p = 0.f;
+              float v = p * __uint_as_float(dpv[x]);
+#pragma unroll
+              for (int sft = 16; sft > 0; sft >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sft);
+              if (lane == 0) s.part[quad][col0 + x] = v;
+            }
+          }
+          __syncthreads();
+          if (tid < 128) s.delta[tid] = (s.part[0][tid] + s.part[1][tid]) + (s.part[2][tid] + s.part[3][tid]);
+          __syncthreads();
+        }
 #pragma unroll
         for (int c = 0; c < 2; ++c) {  // 32 query columns at a time
           const int col0 = half * 64 + c * 32;
@@ -167,7 +199,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           tmem_ld32(tS + lane_off + col0, sv);
           tmem_ld32(tDP + lane_off + col0, dpv);
           tmem_wait_ld();
-          uint32_t pp[16], dsp[16];
+          uint32_t pp[16], dsp[16], ppl[16], dspl[16];
 #pragma unroll
           for (int x = 0; x < 32; x += 2) {
             float p0 = ex2f(fmaf(__uint_as_float(sv[x]), a.scale_log2, -s.lse[col0 + x]));
@@ -178,47 +210,75 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             }
             const float d0 = p0 * (__uint_as_float(dpv[x]) - s.delta[col0 + x]);
             const float d1 = p1 * (__uint_as_float(dpv[x + 1]) - s.delta[col0 + x + 1]);
-            pp[x >> 1] = pack_bf16x2(p0, p1);
-            dsp[x >> 1] = pack_bf16x2(d0, d1);
+            const uint32_t ph = pack_bf16x2(p0, p1), dh = pack_bf16x2(d0, d1);
+            pp[x >> 1] = ph;
+            dsp[x >> 1] = dh;
+            if (hilo) {
+              ppl[x >> 1] = pack_bf16x2(p0 - __uint_as_float(ph << 16), p1 - __uint_as_float(ph & 0xffff0000u));
+              dspl[x >> 1] = pack_bf16x2(d0 - __uint_as_float(dh << 16), d1 - __uint_as_float(dh & 0xffff0000u));
+            }
           }
-          // P^T (bf16 pairs) goes over S^T columns this warp has already read: packed columns
-          // [64*half, 64*half+32) hold query columns [64*half, 64*half+64).
-          tmem_st16(tS + lane_off + half * 64 + c * 16, pp);
+          // P^T (bf16 pairs) goes over S^T columns this warp has already read: for query columns
+          // [col0, col0+32) the hi parts take packed columns [col0, col0+16), the lo parts [col0+16, col0+32).
+          tmem_st16(tS + lane_off + col0, pp);
+          if (hilo) tmem_st16(tS + lane_off + col0 + 16, ppl);
           // dS^T row r, columns col0 .. col0+31 -> four 16-byte chunks of the swizzled half tile
           uint8_t* base = s.ds[half] + r * 128;
+          uint8_t* base_lo = s.ds_lo[half] + r * 128;
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             const int chunk = (c * 4 + ch) ^ (r & 7);
             *reinterpret_cast<uint4*>(base + chunk * 16) =
                 make_uint4(dsp[ch * 4 + 0], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
+            if (hilo)
+              *reinterpret_cast<uint4*>(base_lo + chunk * 16) =
+                  make_uint4(dspl[ch * 4 + 0], dspl[ch * 4 + 1], dspl[ch * 4 + 2], dspl[ch * 4 + 3]);
           }
         }
         tmem_wait_st();
         fence_proxy_async_smem();
-      } else if (lane == 0) {
-        report_timeout(a.status, it, kWhereBwdS, t);
       }
-      ok = ok && okw;
       tc_fence_before_sync();
-      ok = __syncthreads_and(ok);
-      if (!ok) break;
+      __syncthreads();
       // ---- step 2: dV += P^T dO, dK += dS^T Q, dQ = dS K
       if (tid == 0) {
         tc_fence_after_sync();
+        const bool hilo = (m == 0);
+        // packed P^T column of K-step kk (16 query columns): see the store above
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          umma_ts(tDV, tS + (kk >> 2) * 64 + (kk & 3) * 8, make_smem_desc_sw128(do_addr + kk * 2048, kHalfTileBytes, 1024), idesc_kn,
-                  (t > 0 || kk > 0));
+          umma_ts(tDV, tS + (kk >> 1) * 32 + (kk & 1) * 8, make_smem_desc_sw128(do_addr + kk * 2048, kHalfTileBytes, 1024),
+                  idesc_kn, (t > 0 || kk > 0));
+        if (hilo) {
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            umma_ts(tDV, tS + (kk >> 1) * 32 + 16 + (kk & 1) * 8,
+                    make_smem_desc_sw128(do_addr + kk * 2048, kHalfTileBytes, 1024), idesc_kn, 1);
+        }
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t off = (kk >> 2) * kHalfTileBytes + (kk & 3) * 32;
           umma_ss(tDK, make_smem_desc_sw128(ds_addr + off, 16, 1024),
                   make_smem_desc_sw128(q_addr + kk * 2048, kHalfTileBytes, 1024), idesc_kn, (t > 0 || kk > 0));
         }
+        if (hilo) {
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (kk >> 2) * kHalfTileBytes + (kk & 3) * 32;
+            umma_ss(tDK, make_smem_desc_sw128(dsl_addr + off, 16, 1024),
+                    make_smem_desc_sw128(q_addr + kk * 2048, kHalfTileBytes, 1024), idesc_kn, 1);
+          }
+        }
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           umma_ss(tS, make_smem_desc_sw128(ds_addr + kk * 2048, kHalfTileBytes, 1024),
                   make_smem_desc_sw128(k_addr + kk * 2048, kHalfTileBytes, 1024), idesc_nn, kk > 0);
+        if (hilo) {
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            umma_ss(tS, make_smem_desc_sw128(dsl_addr + kk * 2048, kHalfTileBytes, 1024),
+                    make_smem_desc_sw128(k_addr + kk * 2048, kHalfTileBytes, 1024), idesc_nn, 1);
+        }
         umma_commit(&s.bar_m2);
       }
       okw = mbar_wait(&s.bar_m2, ph_m2);

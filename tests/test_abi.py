@@ -1,0 +1,93 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares, and rejects bad
+arguments before touching a device. No compute call is made here."""
+import ctypes
+import re
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2609_22755_b200 import build
+
+    build.build_library()
+    from paper_2609_22755_b200 import binding
+
+    return binding
+
+
+def test_header_symbols_are_exported(B):
+    header = (ROOT / "include" / "nsp.h").read_text()
+    declared = set(re.findall(r"\b(nsp_[a-z_]+)\s*\(", header))
+    assert {"nsp_plan_tiles", "nsp_attn_fwd", "nsp_attn_bwd"} <= declared
+    lib = ctypes.CDLL(str(B.LIB_PATH))
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} is declared in include/nsp.h but not exported"
+    assert declared == set(B.EXPORTS)
+
+
+def test_status_strings(B):
+    assert B.status_string(B.NSP_OK) == "ok"
+    for code in range(1, 7):
+        assert B.status_string(code) not in ("ok", "unknown status")
+    assert B.status_string(99) == "unknown status"
+
+
+def _plan_rc(B, cu, hq, hkv, head_dim=128, opts=None, null=None):
+    cu, hq, hkv = (np.asarray(x, np.int32) for x in (cu, hq, hkv))
+    handle = ctypes.c_void_p()
+    o = B.PlanOpts(*opts) if opts else None
+    args = [B._ptr(cu), B._ptr(hq), B._ptr(hkv)]
+    if null is not None:
+        args[null] = None
+    rc = B.lib().nsp_plan_tiles(*args, len(hq), head_dim, ctypes.byref(o) if o else None, None, ctypes.byref(handle))
+    if rc == B.NSP_OK:
+        B.lib().nsp_plan_destroy(handle)
+    else:
+        assert not handle.value
+    return rc
+
+
+def test_plan_argument_validation(B):
+    good = ([0, 4, 9], [4, 4], [2, 2])
+    assert _plan_rc(B, [1, 4, 9], good[1], good[2]) == B.NSP_ERR_INVALID_ARG  # cu_seqlens[0] != 0
+    assert _plan_rc(B, [0, 9, 4], good[1], good[2]) == B.NSP_ERR_INVALID_ARG  # decreasing
+    assert _plan_rc(B, good[0], [4, 0], good[2]) == B.NSP_ERR_INVALID_ARG  # hq <= 0
+    assert _plan_rc(B, good[0], good[1], [2, -1]) == B.NSP_ERR_INVALID_ARG  # hkv <= 0
+    assert _plan_rc(B, good[0], [4, 3], good[2]) == B.NSP_ERR_INVALID_ARG  # hq % hkv != 0
+    for null in (0, 1, 2):
+        assert _plan_rc(B, *good, null=null) == B.NSP_ERR_INVALID_ARG
+    assert _plan_rc(B, *good, head_dim=64) == B.NSP_ERR_UNSUPPORTED
+    assert _plan_rc(B, *good, opts=(64, 128, 1, 0)) == B.NSP_ERR_UNSUPPORTED  # tile size not built
+    assert _plan_rc(B, *good, opts=(0, 128, 1, 0)) == B.NSP_ERR_INVALID_ARG
+    assert _plan_rc(B, *good, opts=(128, 128, 2, 0)) == B.NSP_ERR_UNSUPPORTED  # unknown order version
+    assert _plan_rc(B, good[0], [512, 512], good[2]) == B.NSP_ERR_UNSUPPORTED  # > 256 heads
+    # too many runs: alternating head counts
+    n = B.NSP_MAX_RUNS + 1
+    assert _plan_rc(B, np.arange(n + 1) * 8, [4, 8] * (n // 2) + [4], [1] * n) == B.NSP_ERR_UNSUPPORTED
+    rc = B.lib().nsp_plan_tiles(None, None, None, -1, 128, None, None, ctypes.byref(ctypes.c_void_p()))
+    assert rc == B.NSP_ERR_INVALID_ARG
+    rc = B.lib().nsp_plan_tiles(B._ptr(np.zeros(1, np.int32)), None, None, 0, 128, None, None, None)
+    assert rc == B.NSP_ERR_INVALID_ARG  # null out pointer
+
+
+def test_null_plan_is_rejected(B):
+    L = B.lib()
+    assert L.nsp_plan_sizes(None, None, None, None, None, None) == B.NSP_ERR_INVALID_ARG
+    assert L.nsp_attn_fwd(None, None, None, None, None, None, 1.0, None, 0, None) == B.NSP_ERR_INVALID_ARG
+    assert L.nsp_attn_bwd(None, None, None, None, None, None, None, None, None, None, 0, 1, 1.0, None, 0,
+                          None) == B.NSP_ERR_INVALID_ARG
+    assert L.nsp_plan_destroy(None) == B.NSP_OK
+    assert L.nsp_launch_count() >= 0
+
+
+def test_no_device_means_an_error_not_a_fallback(B):
+    import torch
+
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    assert _plan_rc(B, [0, 4, 9], [4, 4], [2, 2]) in (B.NSP_ERR_CUDA, B.NSP_ERR_UNSUPPORTED)

@@ -1,0 +1,279 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded inputs.
+
+Small cases and scaled-down twins compare every element; the full-size benchmark configurations compare
+sampled query rows (O, LSE, dQ), the last key columns (dK, dV under the full dO) and a sparse-dO probe (all of
+dK, dV), each computed independently by the oracle. The tile work lists are compared bit for bit.
+"""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import oracle
+    import parity_util as P
+    from paper_2609_22755_b200 import binding as B
+    from paper_2609_22755_b200 import workloads as W
+
+    B.lib()  # fails loudly if the extension is missing
+    return dict(torch=torch, oracle=oracle, P=P, B=B, W=W)
+
+
+def _full_case(env, w, **kw):
+    P = env["P"]
+    run = P.GpuRun(w, **kw)
+    run.forward()
+    run.backward()
+    assert run.status()[0] == 0
+    res = run.results()
+    ref = P.oracle_full(w, run.host)
+    return P.compare_full(w, res, ref), run, res, ref
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_tile_plan_bit_exact_full_size(env, idx):
+    B, W, oracle = env["B"], env["W"], env["oracle"]
+    w = W.config(idx)
+    plan = B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, w.head_dim)
+    for p in (0, 1):
+        got = B.nsp_plan_get(plan, p)
+        want = oracle.plan_tiles(w.cu_seqlens, w.hq, w.hkv, 128, 128, p)
+        assert got.dtype == np.int32 and got.shape == want.shape
+        assert np.array_equal(got, want)
+    plan.destroy()
+
+
+def test_cfg1_every_element(env):
+    _full_case(env, env["W"].config(1))
+
+
+def test_ragged_tails_every_element(env):
+    # lengths 1, 17, 127, 129, 255, 1000, 3 ..., a zero-length segment, MQA / GQA / MHA runs
+    _full_case(env, env["W"].ragged())
+
+
+def test_bf16_gradients_and_fp32_dq_variants(env):
+    # the dtype arguments of nsp_attn_bwd: fp32 dQ meets the tolerance; bf16 dK/dV are produced and close
+    # (their output rounding alone can exceed 2e-2 where |dV| > 8, so only rel-L2 is asserted for them)
+    W, P = env["W"], env["P"]
+    w = W.custom([300, 77], [8, 8], [2, 2], seed=5)
+    _full_case(env, w, dq_dtype="f32", dkv_dtype="f32")
+    run = P.GpuRun(w, dq_dtype="bf16", dkv_dtype="bf16")
+    run.forward()
+    run.backward()
+    res, ref = run.results(), P.oracle_full(w, run.host)
+    for n in ("dk", "dv"):
+        assert P.errors(res[n], ref[n])[1] <= P.REL_L2_TOL
+
+
+@pytest.mark.parametrize("idx", [2, 3, 4, 5])
+def test_scaled_down_twins_every_element(env, idx):
+    _full_case(env, env["W"].config(idx, twin=True))
+
+
+def test_empty_and_degenerate_batches(env):
+    B, W, P, torch = env["B"], env["W"], env["P"], env["torch"]
+    # no segments at all
+    plan = B.nsp_plan_tiles([0], [], [], 128)
+    assert plan.q_elems == 0 and len(B.nsp_plan_get(plan, 0)) == 0 and len(B.nsp_plan_get(plan, 1)) == 0
+    B.nsp_attn_fwd(plan, None, None, None, None, None, 0.1)
+    B.nsp_attn_bwd(plan, None, None, None, None, None, None, None, None, None, 0.1, None, dq_dtype=0, dkv_dtype=1)
+    plan.destroy()
+    # only zero-length segments
+    plan = B.nsp_plan_tiles([0, 0, 0], [4, 8], [2, 2], 128)
+    assert plan.q_elems == 0 and len(B.nsp_plan_get(plan, 0)) == 0
+    plan.destroy()
+    # 1-token segments: O = V exactly (bf16 copy), dQ = dK = 0 up to rounding, dV = sum of the group's dO
+    w = W.custom([1, 1, 1], [4, 4, 2], [2, 2, 1], seed=3)
+    run = P.GpuRun(w)
+    run.forward()
+    run.backward()
+    res = run.results()
+    v = run.host["v"].float().numpy().astype(np.float64)
+    o = res["o"].reshape(-1, 128)
+    exp_rows = []
+    kvo = 0
+    for s in range(w.n_seg):
+        G = w.hq[s] // w.hkv[s]
+        for h in range(w.hq[s]):
+            exp_rows.append(v[kvo + (h // G) * 128: kvo + (h // G + 1) * 128])
+        kvo += w.hkv[s] * 128
+    assert np.array_equal(o, np.stack(exp_rows))
+    # dS = P (dP - delta) vanishes up to the rounding of P = exp2(s - lse) ~ 1
+    assert np.max(np.abs(res["dq"])) <= 1e-4 and np.max(np.abs(res["dk"])) <= 1e-4
+    do = run.host["do"].float().numpy().astype(np.float64)
+    qo, kvo = w.q_offsets(), w.kv_offsets()
+    for s in range(w.n_seg):
+        G = w.hq[s] // w.hkv[s]
+        want = do[qo[s]:qo[s + 1]].reshape(w.hkv[s], G, 128).sum(axis=1)
+        assert np.max(np.abs(res["dv"][kvo[s]:kvo[s + 1]].reshape(w.hkv[s], 128) - want)) <= 2e-2
+
+
+def test_argument_errors_on_device(env):
+    B, W, P, torch = env["B"], env["W"], env["P"], env["torch"]
+    w = W.config(1)
+    run = P.GpuRun(w)
+    with pytest.raises(B.NspError) as e:
+        B.nsp_attn_fwd(run.plan, run.q, run.k, run.v, run.o, run.lse, -1.0)
+    assert e.value.code == B.NSP_ERR_INVALID_ARG
+    with pytest.raises(B.NspError) as e:
+        B.nsp_attn_fwd(run.plan, run.q[1:], run.k, run.v, run.o, run.lse, 0.1)  # 2-byte offset: misaligned
+    assert e.value.code == B.NSP_ERR_INVALID_ARG
+    with pytest.raises(B.NspError) as e:
+        B.nsp_attn_bwd(run.plan, run.q, run.k, run.v, run.o, run.do, run.lse, run.dq, run.dk, run.dv, 0.1, run.ws[:256])
+    assert e.value.code == B.NSP_ERR_WORKSPACE
+    with pytest.raises(B.NspError) as e:
+        B.nsp_attn_bwd(run.plan, run.q, run.k, run.v, run.o, run.do, run.lse, run.dq, run.dk, run.dv, 0.1, run.ws,
+                       dq_dtype=7)
+    assert e.value.code == B.NSP_ERR_INVALID_ARG
+    assert run.status() == (0, 0, 0, 0)
+
+
+def test_packing_order_invariance_and_reproducibility(env):
+    W, P, torch = env["W"], env["P"], env["torch"]
+    lengths, hq, hkv = [700, 130, 2048, 64], [8, 8, 4, 4], [2, 2, 1, 1]
+    w = W.custom(lengths, hq, hkv, seed=21)
+    run = P.GpuRun(w)
+    run.forward()
+    run.backward()
+    a = run.results()
+    # same inputs again: O, LSE, dK, dV bitwise equal (fixed accumulation order); dQ within tolerance
+    # (its tiles are added to the fp32 accumulator with floating-point reductions in arrival order)
+    run.forward()
+    run.backward()
+    b = run.results()
+    for n in ("o", "lse", "dk", "dv"):
+        assert np.array_equal(a[n], b[n]), n
+    assert P.errors(a["dq"], b["dq"])[0] <= 2e-2
+    # permute the two runs (segments 2,3 first): every segment's results are unchanged
+    qo, kvo, lo = w.q_offsets(), w.kv_offsets(), w.lse_offsets()
+    perm = [2, 3, 0, 1]
+    wp = W.custom([lengths[p] for p in perm], [hq[p] for p in perm], [hkv[p] for p in perm], seed=21)
+    host = {}
+    for name, off in (("q", qo), ("do", qo), ("k", kvo), ("v", kvo)):
+        host[name] = torch.cat([run.host[name][off[p]:off[p + 1]] for p in perm])
+    runp = P.GpuRun(wp, tensors=host)
+    runp.forward()
+    runp.backward()
+    c = runp.results()
+    pqo, pkvo, plo = wp.q_offsets(), wp.kv_offsets(), wp.lse_offsets()
+    for new, p in enumerate(perm):
+        for n, off, poff in (("o", qo, pqo), ("lse", lo, plo), ("dk", kvo, pkvo), ("dv", kvo, pkvo)):
+            assert np.array_equal(a[n][off[p]:off[p + 1]], c[n][poff[new]:poff[new + 1]]), (n, p)
+        assert P.errors(c["dq"][pqo[new]:pqo[new + 1]], a["dq"][qo[p]:qo[p + 1]])[0] <= 2e-2
+
+
+def _sample_rows(w, rng, per_seg):
+    rows = []
+    for s in range(w.n_seg):
+        L = int(w.lengths[s])
+        if L == 0:
+            continue
+        cand = {0, L - 1, min(127, L - 1), min(128, L - 1), L // 2, max(0, L - 129), (L // 128) * 128 - 1 if L >= 128 else 0}
+        cand |= set(int(x) for x in rng.integers(0, L, size=per_seg))
+        for i in sorted(cand):
+            rows.append((s, int(rng.integers(0, w.hq[s])), i))
+    return rows
+
+
+@pytest.mark.parametrize("idx,per_seg,last_cols", [(2, 2, 32), (3, 3, 32), (4, 6, 48), (5, 3, 24)])
+def test_full_size_configs_sampled(env, idx, per_seg, last_cols):
+    """Full benchmark sizes in the launch configuration the benchmark times."""
+    W, P, oracle, torch = env["W"], env["P"], env["oracle"], env["torch"]
+    w = W.config(idx)
+    run = P.GpuRun(w)
+    run.forward()
+    run.backward()
+    assert run.status()[0] == 0
+    torch.cuda.synchronize()
+    bits = {n: W.bf16_bits(run.host[n]) for n in ("q", "k", "v", "do")}
+    rng = np.random.default_rng(100 + idx)
+    D = w.head_dim
+    qo, kvo, lo = w.q_offsets(), w.kv_offsets(), w.lse_offsets()
+    # only the long segments keep the oracle cost bounded: sample rows in the 4 longest + 4 random segments
+    order = np.argsort(-w.lengths)
+    keep = set(order[:4].tolist()) | set(rng.choice(w.n_seg, size=min(4, w.n_seg), replace=False).tolist())
+    rows = [r for r in _sample_rows(w, rng, per_seg) if r[0] in keep]
+    O, LSE, dQ = oracle.attn_rows(bits["q"], bits["k"], bits["v"], bits["do"], w.cu_seqlens, w.hq, w.hkv, D,
+                                  w.softmax_scale, rows)
+    idx_q = np.concatenate([qo[s] + (i * w.hq[s] + h) * D + np.arange(D) for s, h, i in rows])
+    idx_l = np.array([lo[s] + h * w.lengths[s] + i for s, h, i in rows])
+    go = run.o[torch.as_tensor(idx_q, device=run.dev)].float().cpu().numpy()
+    gdq = run.dq[torch.as_tensor(idx_q, device=run.dev)].float().cpu().numpy()
+    glse = run.lse[torch.as_tensor(idx_l, device=run.dev)].cpu().numpy()
+    P.check(f"{w.name}:o[rows]", go, O.ravel())
+    P.check(f"{w.name}:dq[rows]", gdq, dQ.ravel())
+    assert np.max(np.abs(glse - LSE)) <= P.LSE_ABS_TOL
+    # last key columns of the longest and of one short segment, every kv head of it
+    cols = []
+    for s in (int(order[0]), int(order[min(3, w.n_seg - 1)])):
+        L = int(w.lengths[s])
+        for g in range(min(int(w.hkv[s]), 2)):
+            cols += [(s, g, j) for j in range(max(0, L - last_cols), L)]
+    dK, dV = oracle.attn_cols(bits["q"], bits["k"], bits["v"], bits["do"], w.cu_seqlens, w.hq, w.hkv, D,
+                              w.softmax_scale, cols)
+    idx_kv = np.concatenate([kvo[s] + (j * w.hkv[s] + g) * D + np.arange(D) for s, g, j in cols])
+    gdk = run.dk[torch.as_tensor(idx_kv, device=run.dev)].float().cpu().numpy()
+    gdv = run.dv[torch.as_tensor(idx_kv, device=run.dev)].float().cpu().numpy()
+    P.check(f"{w.name}:dk[last cols]", gdk, dK.ravel())
+    P.check(f"{w.name}:dv[last cols]", gdv, dV.ravel())
+    # gradient identities at full size (no oracle run needed): sum_j dK_j = 0, sum_j dV_j = sum of the group's dO
+    s0 = int(order[0])
+    L, Hkv, Hq = int(w.lengths[s0]), int(w.hkv[s0]), int(w.hq[s0])
+    dk0 = run.dk[kvo[s0]:kvo[s0 + 1]].view(L, Hkv, D).double()
+    dv0 = run.dv[kvo[s0]:kvo[s0 + 1]].view(L, Hkv, D).double()
+    do0 = run.do[qo[s0]:qo[s0 + 1]].view(L, Hkv, Hq // Hkv, D).double()
+    scale_ref = float(dk0.abs().sum(dim=0).max())
+    assert float(dk0.sum(dim=0).abs().max()) <= 2e-3 * max(scale_ref, 1.0)
+    want = do0.sum(dim=(0, 2))
+    got = dv0.sum(dim=0)
+    assert float((got - want).abs().max()) <= 2e-3 * float(dv0.abs().sum(dim=0).max())
+
+
+@pytest.mark.parametrize("idx", [4, 5])
+def test_full_size_sparse_dO_probe(env, idx):
+    """dO non-zero on a sparse set of query rows: every element of dK and dV then depends on those rows only,
+    so the oracle can produce ALL of dK/dV of the full-size configuration; dQ must vanish off the rows."""
+    W, P, oracle, torch = env["W"], env["P"], env["oracle"], env["torch"]
+    w = W.config(idx)
+    host = W.make_tensors(w)
+    rng = np.random.default_rng(7 + idx)
+    qo, kvo = w.q_offsets(), w.kv_offsets()
+    D = w.head_dim
+    order = np.argsort(-w.lengths)
+    active = []
+    for s, cnt in ((int(order[0]), 20), (int(order[1]), 8), (int(order[-1]), 4)):
+        L = int(w.lengths[s])
+        pick = {L - 1, 0, min(L - 1, 128)} | set(int(x) for x in rng.integers(0, L, size=cnt))
+        active += [(s, i) for i in sorted(pick)]
+    do = torch.zeros_like(host["do"])
+    for s, i in active:
+        a, b = qo[s] + i * w.hq[s] * D, qo[s] + (i + 1) * w.hq[s] * D
+        do[a:b] = host["do"][a:b]
+    host["do"] = do
+    run = P.GpuRun(w, tensors=host)
+    run.forward()
+    run.backward()
+    assert run.status()[0] == 0
+    bits = {n: W.bf16_bits(host[n]) for n in ("q", "k", "v", "do")}
+    _, dK, dV = oracle.attn_bwd(bits["q"], bits["k"], bits["v"], bits["do"], w.cu_seqlens, w.hq, w.hkv, D,
+                                w.softmax_scale, rows=active, want_dq=False)
+    P.check(f"{w.name}:dk[sparse dO, all]", run.dk.cpu().numpy(), dK)
+    P.check(f"{w.name}:dv[sparse dO, all]", run.dv.cpu().numpy(), dV)
+    del dK, dV
+    gdq = run.dq.float()
+    mask = torch.ones(w.q_elems(), dtype=torch.bool, device=run.dev)
+    for s, i in active:
+        mask[qo[s] + i * w.hq[s] * D: qo[s] + (i + 1) * w.hq[s] * D] = False
+    assert float(gdq[mask].abs().max()) == 0.0
+    rows = [(s, int(rng.integers(0, w.hq[s])), i) for s, i in active]
+    _, _, dQ = oracle.attn_rows(bits["q"], bits["k"], bits["v"], bits["do"], w.cu_seqlens, w.hq, w.hkv, D,
+                                w.softmax_scale, rows)
+    idx_q = np.concatenate([qo[s] + (i * w.hq[s] + h) * D + np.arange(D) for s, h, i in rows])
+    P.check(f"{w.name}:dq[active rows]", gdq[torch.as_tensor(idx_q, device=run.dev)].cpu().numpy(), dQ.ravel())
