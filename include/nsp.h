@@ -122,6 +122,18 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
 /* Read the sticky device status {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
 int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
 
+/* Kernels of the path, for nsp_plan_kernel_ms. */
+enum { NSP_KERNEL_FWD = 0, NSP_KERNEL_BWD_PRE = 1, NSP_KERNEL_BWD_MAIN = 2, NSP_KERNEL_BWD_POST = 3, NSP_KERNEL_COUNT = 4 };
+
+/* Measurement aid (the paper's cost model is fed by offline profiles of the compute phase, Sec. 4.2): when
+ * enabled, every later nsp_attn_fwd / nsp_attn_bwd on this plan brackets each of its kernels with a pair of CUDA
+ * events recorded on the launching stream. Errors: INVALID_ARG (null plan), CUDA. */
+int nsp_plan_set_profiling(nsp_plan_t* plan, int enable);
+
+/* Device time in milliseconds of the most recent launch of kernel `kernel_id` (NSP_KERNEL_*) on this plan.
+ * Waits for that launch to finish. Errors: INVALID_ARG (profiling off, kernel not launched yet, bad id), CUDA. */
+int nsp_plan_kernel_ms(const nsp_plan_t* plan, int kernel_id, float* ms);
+
 /* Number of kernel launches the library has enqueued so far in this process (all plans). */
 int64_t nsp_launch_count(void);
 

@@ -24,8 +24,9 @@ NSP_MAX_RUNS = 32
 
 EXPORTS = [
     "nsp_plan_tiles", "nsp_plan_sizes", "nsp_plan_get", "nsp_attn_fwd", "nsp_attn_bwd", "nsp_device_status",
-    "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string",
+    "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string", "nsp_plan_set_profiling", "nsp_plan_kernel_ms",
 ]
+KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST = 0, 1, 2, 3
 
 LIB_PATH = Path(__file__).resolve().parent / "libnsp.so"
 _lib = None
@@ -68,6 +69,10 @@ def lib() -> ctypes.CDLL:
         L.nsp_launch_count.restype = ctypes.c_int64
         L.nsp_plan_destroy.argtypes = [vp]
         L.nsp_plan_destroy.restype = ctypes.c_int
+        L.nsp_plan_set_profiling.argtypes = [vp, ctypes.c_int]
+        L.nsp_plan_set_profiling.restype = ctypes.c_int
+        L.nsp_plan_kernel_ms.argtypes = [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
+        L.nsp_plan_kernel_ms.restype = ctypes.c_int
         L.nsp_status_string.argtypes = [ctypes.c_int]
         L.nsp_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -193,3 +198,17 @@ def nsp_device_status(plan: Plan):
     if rc != NSP_OK:
         raise NspError(rc, "nsp_device_status")
     return tuple(out)
+
+
+def nsp_plan_set_profiling(plan: Plan, enable: bool):
+    rc = lib().nsp_plan_set_profiling(plan.handle, int(bool(enable)))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_plan_set_profiling")
+
+
+def nsp_plan_kernel_ms(plan: Plan, kernel_id: int) -> float:
+    ms = ctypes.c_float()
+    rc = lib().nsp_plan_kernel_ms(plan.handle, kernel_id, ctypes.byref(ms))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_plan_kernel_ms")
+    return float(ms.value)

@@ -31,6 +31,10 @@ struct nsp_plan {
   int32_t* d_status = nullptr;    // {code, item, where, aux}
   cudaStream_t build_stream = nullptr;
   int sticky = 0;
+  // optional per-kernel timing (CUDA events on the launching stream)
+  bool profiling = false;
+  cudaEvent_t ev[2 * NSP_KERNEL_COUNT] = {};
+  bool ev_valid[NSP_KERNEL_COUNT] = {};
 };
 
 namespace {
@@ -82,7 +86,17 @@ void free_plan(nsp_plan* p) {
   cudaFree(p->d_bwd);
   cudaFree(p->d_counters);
   cudaFree(p->d_status);
+  for (cudaEvent_t e : p->ev)
+    if (e) cudaEventDestroy(e);
   delete p;
+}
+
+// Record the start / stop event of kernel `id` when profiling is on.
+void prof_mark(const nsp_plan* plan, int id, int stop, cudaStream_t st) {
+  if (!plan->profiling) return;
+  nsp_plan* p = const_cast<nsp_plan*>(plan);
+  cudaEventRecord(p->ev[2 * id + stop], st);
+  if (stop) p->ev_valid[id] = true;
 }
 
 }  // namespace
@@ -311,7 +325,9 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  prof_mark(plan, NSP_KERNEL_FWD, 0, st);
   if (launch_fwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  prof_mark(plan, NSP_KERNEL_FWD, 1, st);
   return NSP_OK;
 }
 
@@ -347,10 +363,12 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   }
   if (cudaMemsetAsync(plan->d_counters + 1, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
   if (cudaMemsetAsync(dq_acc, 0, static_cast<size_t>(plan->q_elems) * 4, st) != cudaSuccess) return NSP_ERR_CUDA;
+  prof_mark(plan, NSP_KERNEL_BWD_PRE, 0, st);
   if (launch_bwd_preprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems,
                             static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta,
                             st) != cudaSuccess)
     return NSP_ERR_CUDA;
+  prof_mark(plan, NSP_KERNEL_BWD_PRE, 1, st);
   BwdArgs a;
   a.seg = plan->d_seg;
   a.items = plan->d_bwd;
@@ -365,9 +383,13 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.dkv_f32 = dkv_dtype == NSP_F32;
   a.scale = softmax_scale;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  prof_mark(plan, NSP_KERNEL_BWD_MAIN, 0, st);
   if (launch_bwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  prof_mark(plan, NSP_KERNEL_BWD_MAIN, 1, st);
+  prof_mark(plan, NSP_KERNEL_BWD_POST, 0, st);
   if (launch_bwd_postprocess(dq_acc, dq, plan->q_elems, dq_dtype == NSP_F32, softmax_scale, st) != cudaSuccess)
     return NSP_ERR_CUDA;
+  prof_mark(plan, NSP_KERNEL_BWD_POST, 1, st);
   return NSP_OK;
 }
 
@@ -376,6 +398,26 @@ int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]) {
   if (cudaDeviceSynchronize() != cudaSuccess) return NSP_ERR_CUDA;
   if (cudaMemcpy(out, plan->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return NSP_ERR_CUDA;
   if (out[0] != 0) const_cast<nsp_plan_t*>(plan)->sticky = out[0];
+  return NSP_OK;
+}
+
+int nsp_plan_set_profiling(nsp_plan_t* plan, int enable) {
+  if (!plan) return NSP_ERR_INVALID_ARG;
+  if (enable && !plan->ev[0]) {
+    for (cudaEvent_t& e : plan->ev)
+      if (cudaEventCreate(&e) != cudaSuccess) return NSP_ERR_CUDA;
+  }
+  plan->profiling = enable != 0;
+  if (!enable)
+    for (bool& v : plan->ev_valid) v = false;
+  return NSP_OK;
+}
+
+int nsp_plan_kernel_ms(const nsp_plan_t* plan, int kernel_id, float* ms) {
+  if (!plan || !ms || kernel_id < 0 || kernel_id >= NSP_KERNEL_COUNT) return NSP_ERR_INVALID_ARG;
+  if (!plan->profiling || !plan->ev_valid[kernel_id]) return NSP_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(plan->ev[2 * kernel_id + 1]) != cudaSuccess) return NSP_ERR_CUDA;
+  if (cudaEventElapsedTime(ms, plan->ev[2 * kernel_id], plan->ev[2 * kernel_id + 1]) != cudaSuccess) return NSP_ERR_CUDA;
   return NSP_OK;
 }
 
