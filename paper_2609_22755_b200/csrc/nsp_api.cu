@@ -383,6 +383,10 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.dkv_f32 = dkv_dtype == NSP_F32;
   a.scale = softmax_scale;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  {
+    const char* dbg = std::getenv("NSP_DEBUG_FLAGS");
+    a.debug_flags = dbg ? std::atoi(dbg) : 0;
+  }
   prof_mark(plan, NSP_KERNEL_BWD_MAIN, 0, st);
   if (launch_bwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_MAIN, 1, st);

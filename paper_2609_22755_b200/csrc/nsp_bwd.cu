@@ -169,8 +169,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         // dK/dV/dQ, so they are fed to the tensor core as hi + lo bf16 pairs (two MMAs per product), and
         // delta_i is recomputed as sum_j P_ij dP_ij in fp32 (all keys of these rows lie in this key tile)
         // instead of taking it from the bf16-rounded O.
-        const bool hilo = (m == 0);
-        if (hilo) {
+        const bool exact_delta = (m == 0) && (a.debug_flags & 2) == 0;
+        const bool hilo = (m == 0) && (a.debug_flags & 1) == 0;
+        if (exact_delta) {
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             const int col0 = half * 64 + c * 32;
@@ -243,7 +244,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       // ---- step 2: dV += P^T dO, dK += dS^T Q, dQ = dS K
       if (tid == 0) {
         tc_fence_after_sync();
-        const bool hilo = (m == 0);
+        const bool hilo = (m == 0) && (a.debug_flags & 1) == 0;
         // packed P^T column of K-step kk (16 query columns): see the store above
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)

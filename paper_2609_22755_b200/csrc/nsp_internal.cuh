@@ -82,6 +82,7 @@ struct BwdArgs {
   int32_t dkv_f32;
   float scale;
   float scale_log2;
+  int32_t debug_flags;  // experiments only: bit 0 = no hi/lo split, bit 1 = no exact delta
 };
 
 // Host-side launchers implemented next to their kernels.
