@@ -36,6 +36,7 @@ struct FwdMaps {
 };
 struct BwdMaps {
   CUtensorMap q[NSP_MAX_RUNS], d_o[NSP_MAX_RUNS], k[NSP_MAX_RUNS], v[NSP_MAX_RUNS];
+  CUtensorMap dq[NSP_MAX_RUNS];  // fp32 dQ accumulator, tiles {32 dims, 1 head, 128 tokens}
 };
 
 // Device status word: {code, item, where, aux}; first writer wins (atomicCAS on code).
@@ -47,6 +48,15 @@ enum DeviceWhere : int32_t {
   kWhereBwdLoadQ = 12,
   kWhereBwdS = 13,
   kWhereBwdMma2 = 14,
+  kWhereBwdSmemAlign = 15,
+  kWhereBwdQEmpty = 16,
+  kWhereBwdDqEmpty = 17,
+  kWhereBwdPReady = 18,
+  kWhereBwdLdEmpty = 19,
+  kWhereBwdDqFull = 20,
+  kWhereBwdDp = 21,
+  kWhereBwdStaged = 22,
+  kWhereBwdDelta = 23,
 };
 
 __device__ __forceinline__ void report_timeout(int32_t* status, int32_t item, int32_t where, int32_t aux) {
