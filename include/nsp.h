@@ -119,6 +119,28 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
                  const float* lse, void* dq, void* dk, void* dv, int dq_dtype, int dkv_dtype, float softmax_scale,
                  void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * (No counterpart in the paper: an addition for callers that are not allowed to allocate.)
+ * nsp_attn_bwd without a caller-provided workspace. Some callers cannot supply one: an executor that handed all
+ * device memory to its own planner or caching pool at start-up has no way to obtain a transient q-sized fp32
+ * buffer mid-iteration, because cudaMalloc would synchronise the device, may fail once the pool owns the memory,
+ * and is banned inside some schedulers. For them the scratch (fp32 dQ accumulator + delta) is a fixed array of
+ * NSP_STATIC_WS_BYTES inside the library image; every GPU that loads the library holds that much memory until exit.
+ * Arguments, outputs and results are those of nsp_attn_bwd (same kernels); inputs and outputs are still the caller's.
+ * Limit: plans whose bwd_ws_bytes (see nsp_plan_sizes; roughly 4 * q_elems + 4 * lse_elems bytes) exceed
+ * NSP_STATIC_WS_BYTES are rejected with NSP_ERR_WORKSPACE and nothing is enqueued.
+ * This call makes no cudaMalloc / cudaFree and calls no allocating routine. The first call on each device looks up
+ * the array's device address (cudaGetSymbolAddress, with that device current); make that first call before any
+ * stream capture begins. The array is shared by all calls and keeps the previous call's contents: the
+ * accumulator part is cleared on `stream` at the start of each call, and two calls whose device work overlaps
+ * (other streams or host threads) race on it -- serialise them.
+ * Errors: INVALID_ARG, WORKSPACE (batch too large), CUDA, DEVICE_TIMEOUT, as nsp_attn_bwd.
+ */
+#define NSP_STATIC_WS_BYTES (32u * 1024u * 1024u)
+int nsp_attn_bwd_static(const nsp_plan_t* plan, const void* q, const void* k, const void* v, const void* o,
+                        const void* d_o, const float* lse, void* dq, void* dk, void* dv, int dq_dtype, int dkv_dtype,
+                        float softmax_scale, void* stream);
+
 /* Read the sticky device status {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
 int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
 

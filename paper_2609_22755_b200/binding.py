@@ -25,7 +25,9 @@ NSP_MAX_RUNS = 32
 EXPORTS = [
     "nsp_plan_tiles", "nsp_plan_sizes", "nsp_plan_get", "nsp_attn_fwd", "nsp_attn_bwd", "nsp_device_status",
     "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string", "nsp_plan_set_profiling", "nsp_plan_kernel_ms",
+    "nsp_attn_bwd_static",
 ]
+NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
 KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST = 0, 1, 2, 3
 
 LIB_PATH = Path(__file__).resolve().parent / "libnsp.so"
@@ -63,6 +65,9 @@ def lib() -> ctypes.CDLL:
         L.nsp_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_float,
                                    vp, ctypes.c_size_t, vp]
         L.nsp_attn_bwd.restype = ctypes.c_int
+        L.nsp_attn_bwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int,
+                                          ctypes.c_float, vp]
+        L.nsp_attn_bwd_static.restype = ctypes.c_int
         L.nsp_device_status.argtypes = [vp, i32p]
         L.nsp_device_status.restype = ctypes.c_int
         L.nsp_launch_count.argtypes = []
@@ -212,3 +217,20 @@ def nsp_plan_kernel_ms(plan: Plan, kernel_id: int) -> float:
     if rc != NSP_OK:
         raise NspError(rc, "nsp_plan_kernel_ms")
     return float(ms.value)
+
+
+def nsp_attn_bwd_static(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, softmax_scale, dq_dtype=None, dkv_dtype=None,
+                        stream=None):
+    """nsp_attn_bwd for callers that may not allocate: no workspace argument, the scratch is a fixed array inside
+    the library (at most NSP_STATIC_WS_BYTES; larger batches raise NSP_ERR_WORKSPACE). Calls sharing a device
+    must not overlap. Make the first call on a device outside any stream capture."""
+    import torch
+
+    if dq_dtype is None:
+        dq_dtype = NSP_F32 if dq.dtype == torch.float32 else NSP_BF16
+    if dkv_dtype is None:
+        dkv_dtype = NSP_F32 if dk.dtype == torch.float32 else NSP_BF16
+    rc = lib().nsp_attn_bwd_static(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq),
+                                   _ptr(dk), _ptr(dv), dq_dtype, dkv_dtype, float(softmax_scale), _stream_ptr(stream))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_attn_bwd_static")
