@@ -122,7 +122,7 @@ def reference_arm(args, rank, world):
     """The oracle as it stands, timed on the host cores; each step is one bounded sample of the workload."""
     if rank != 0:
         return
-    w = W.config(args.config)
+    w = W.profile_case() if args.config == 0 else W.config(args.config)
     vals = []
     for _ in range(args.warmup):
         run_oracle_sample(w)
@@ -150,7 +150,9 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=4, help="benchmark configuration 1..5 (default: the nested-plan shard)")
+    ap.add_argument("--config", type=int, default=4,
+                    help="benchmark configuration 1..5 (default 4: the nested-plan shard); 0 = the scaled-down nested "
+                         "case used for profiler captures")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile-mode", action="store_true",
@@ -185,7 +187,10 @@ def main():
         torch.cuda.synchronize()
 
     # one shard per GPU: same configuration, its own seed (lengths and values)
-    w = W.config(args.config, seed=(args.config - 1) + 1000 * rank)
+    if args.config == 0:
+        w = W.profile_case()
+    else:
+        w = W.config(args.config, seed=(args.config - 1) + 1000 * rank)
     host = W.make_tensors(w)
     host = {k: v.pin_memory() for k, v in host.items()}
     eng = NspAttention(w, device=f"cuda:{local_rank}")

@@ -30,7 +30,9 @@ EXPORTS = [
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
 KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST = 0, 1, 2, 3
 
-LIB_PATH = Path(__file__).resolve().parent / "libnsp.so"
+import os
+
+LIB_PATH = Path(os.environ.get("NSP_LIBRARY", Path(__file__).resolve().parent / "libnsp.so"))
 _lib = None
 
 

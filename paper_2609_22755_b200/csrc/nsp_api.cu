@@ -210,6 +210,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     nf += Mt * hq[s];
     nb += Nt * hkv[s];
   }
+  for (int s = 0; s < n_seg; ++s) p->seg[s].run_tokens = static_cast<int32_t>(p->runs[p->seg[s].run].tokens);
   row_base[n_seg] = lse_off;
   fwd_base[n_seg] = nf;
   bwd_base[n_seg] = nb;

@@ -20,7 +20,8 @@ struct SegInfo {
   int32_t hq, hkv;
   int32_t run;         // index of the run (dense [T, H, D] tensor) the segment belongs to
   int32_t tok_in_run;  // first token of the segment, relative to the run
-  int32_t pad_[3];
+  int32_t run_tokens;  // tokens of the whole run (extent of its tensor maps)
+  int32_t pad_[2];
 };
 static_assert(sizeof(SegInfo) == 56 || sizeof(SegInfo) == 64, "SegInfo layout");
 
@@ -57,6 +58,8 @@ enum DeviceWhere : int32_t {
   kWhereBwdDp = 21,
   kWhereBwdStaged = 22,
   kWhereBwdDelta = 23,
+  kWhereBwdDsReady = 24,
+  kWhereBwdItemBarrier = 25,
 };
 
 __device__ __forceinline__ void report_timeout(int32_t* status, int32_t item, int32_t where, int32_t aux) {

@@ -140,6 +140,15 @@ def config(idx: int, seed: int | None = None, twin: bool = False) -> Workload:
     raise ValueError("config index must be 1..5")
 
 
+def profile_case(seed: int = 3) -> Workload:
+    """A scaled-down nested shard for profiler captures: one 65,536-token segment at degree 8 (4q/1kv) plus a
+    degree-1 tail (32q/4kv) filling 8,192 tokens. About 0.7 GB on the device (more than L2), a few hundred
+    milliseconds of kernels even under a multi-pass capture."""
+    short = lognormal_lengths(seed, 8192, 2048, 1.2, 64, 16384)
+    return _mk("nested_profile_case_64k", [65536] + short, [4] + [32] * len(short), [1] + [4] * len(short), seed,
+               "one 65,536-token segment (4q/1kv) + degree-1 tail (32q/4kv) filling 8,192 tokens")
+
+
 def ragged(seed: int = 11) -> Workload:
     """Lengths that are not multiples of 16 or of any tile, a 1-token and a zero-length segment, three runs."""
     lengths = [1, 17, 0, 127, 129, 255, 1000, 3, 384]
