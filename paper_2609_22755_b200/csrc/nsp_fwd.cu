@@ -1,16 +1,20 @@
 // Forward: packed variable-length causal GQA attention on tcgen05 tensor cores.
 //
-// One persistent CTA (128 threads, two CTAs resident per SM) pops work items (segment, q head, q tile) from the
-// longest-first list with an atomic cursor. For an item it keeps the 128 x 128 Q tile in shared memory and
-// walks the key tiles 0 .. diagonal:
-//     S = Q K^T        tcgen05.mma, both operands K-major in 128B-swizzled shared memory (TMA-staged)
-//     online softmax   one thread per query row: tcgen05.ld S, exp2 with the scale folded in, row max/sum
-//     P -> TMEM        bf16 pairs written over S (tcgen05.st)
-//     O += P V         tcgen05.mma with A = P from TMEM, B = V (MN-major) from shared memory
-// O stays in TMEM for the whole item and is rescaled in place only when the running maximum grows by more
-// than 2^8 (the stale reference maximum is exact in the final normalisation because the same reference is
-// used for the row sum). Only the diagonal tile is masked; tiles above the diagonal are never visited.
-// The two CTAs of an SM overlap one CTA's softmax with the other's MMAs.
+// One persistent CTA per SM (384 threads) pops work items (segment, q head, q tile) from the longest-first
+// list TWO at a time. Neighbouring items of the list are the same (segment, q tile) for consecutive q heads, so
+// when they share a KV head (GQA) the CTA runs them as a pair "A/B" over the SAME K/V tiles: every K/V tile is
+// fetched once for 256 query rows, and the tensor pipe alternates between the two while their softmax
+// warpgroups work (otherwise the two items run one after the other with warpgroup B idle).
+//     S_x  = Q_x K_j^T      tcgen05.mma SS (both K-major, 128B-swizzled smem staged by TMA)       -> TMEM S_x
+//     P_x  = exp2(S_x*c - m)  one thread per query row (tcgen05.ld), bf16 pairs written over S_x  (tcgen05.st)
+//     O_x += P_x V_j        tcgen05.mma TS (A = P_x from TMEM, B = V MN-major from smem)          -> TMEM O_x
+// Issue order of the single MMA thread: PV_A(j), S_A(j+1), PV_B(j), S_B(j+1): S of the next key tile is already
+// running while the other half's softmax is still working. TMEM: S_A, S_B, O_A, O_B = 4 x 128 columns.
+// Roles: warps 0-3 softmax of A, warps 4-7 softmax of B, warp 8 TMA producer (Q pair, two-stage K and V rings),
+// warp 9 MMA issuer; register budgets are set per warpgroup with setmaxnreg.
+// O stays in TMEM for the whole item and is rescaled in place only when the running maximum grows by more than
+// 2^8 (the stale reference maximum is exact in the final normalisation because the same reference is used for
+// the row sum). Only the diagonal tile is masked; tiles above the diagonal are never visited.
 #include <cuda_bf16.h>
 #include "nsp_internal.cuh"
 #include "sm100_ptx.cuh"
@@ -18,33 +22,63 @@
 namespace nsp {
 namespace {
 
-constexpr int kFwdThreads = 128;
+constexpr int kFwdThreads = 384;
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;  // one [128 rows x 64 cols] bf16 sub-tile
 constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;
-constexpr uint32_t kFwdTmemCols = 256;  // S/P: columns [0,128), O: columns [128,256)
+constexpr uint32_t kFwdTmemCols = 512;  // S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512)
+constexpr int kFwdRegsSoftmax = 216, kFwdRegsAux = 72;  // 2*216 + 72 = 504 = 3 * 168, the launch-time allocation
 
 struct FwdSmem {
-  uint8_t q[2][kHalfTileBytes];
-  uint8_t k[2][kHalfTileBytes];
-  uint8_t v[2][kHalfTileBytes];
-  uint64_t bar_q, bar_k, bar_v, bar_s, bar_o;
+  uint8_t q[2][2][kHalfTileBytes];  // [A/B][64-column half]
+  uint8_t k[2][2][kHalfTileBytes];  // [stage][half]
+  uint8_t v[2][2][kHalfTileBytes];  // [stage][half]
+  uint64_t bar_q;
+  uint64_t bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
+  uint64_t bar_s_full[2];   // [A/B] S_x of a key tile is in TMEM
+  uint64_t bar_p_ready[2];  // [A/B] 128 softmax threads: P_x written (and O_x rescaled if needed)
+  uint64_t bar_pv_done[2];  // [A/B] O_x += P_x V has completed
   uint32_t tmem_base;
-  int32_t item_idx;
+  int32_t item_idx[2];
+  int32_t abort;
+};
+static_assert(sizeof(FwdSmem) <= 232448, "shared memory budget (227 KB)");
+constexpr size_t kFwdSmemBytes = sizeof(FwdSmem);
+
+template <int N>
+__device__ __forceinline__ void fwd_setmaxnreg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void fwd_setmaxnreg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+// What one pop of the work list turned into: one or two rounds, each with item A and (in a joint round) item B.
+struct FwdRound {
+  nsp_tile_t a, b;
+  int joint;
 };
 
-constexpr size_t kFwdSmemBytes = sizeof(FwdSmem) + 1024;  // + slack for manual 1024-byte alignment
-
-__global__ void __launch_bounds__(kFwdThreads, 2) fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  FwdSmem& s = *reinterpret_cast<FwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
+__global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  FwdSmem& s = *reinterpret_cast<FwdSmem*>(smem_raw);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
+  if ((smem_u32(smem_raw) & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
+    if (tid == 0) report_timeout(a.status, -1, kWhereFwdSmemAlign, 0);
+    return;
+  }
   if (tid == 0) {
     mbar_init(&s.bar_q, 1);
-    mbar_init(&s.bar_k, 1);
-    mbar_init(&s.bar_v, 1);
-    mbar_init(&s.bar_s, 1);
-    mbar_init(&s.bar_o, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&s.bar_k_full[i], 1);
+      mbar_init(&s.bar_k_empty[i], 1);
+      mbar_init(&s.bar_v_full[i], 1);
+      mbar_init(&s.bar_v_empty[i], 1);
+      mbar_init(&s.bar_s_full[i], 1);
+      mbar_init(&s.bar_p_ready[i], 128);
+      mbar_init(&s.bar_pv_done[i], 1);
+    }
+    s.abort = 0;
     fence_mbar_init();
   }
   if (warp == 0) {
@@ -55,195 +89,297 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_kernel(const __grid_consta
   __syncthreads();
   tc_fence_after_sync();
 
-  const uint32_t tS = s.tmem_base;
-  const uint32_t tO = s.tmem_base + 128;
-  const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
-  const uint32_t q_addr = smem_u32(s.q[0]), k_addr = smem_u32(s.k[0]), v_addr = smem_u32(s.v[0]);
-  constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
-  constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);
-  uint32_t ph_q = 0, ph_k = 0, ph_v = 0, ph_s = 0, ph_o = 0;
-  bool ok = true;
+  const uint32_t tmem = s.tmem_base;
+  volatile int32_t* abort_flag = &s.abort;
+  uint32_t gp = 0;  // pops so far
 
-  for (;;) {
-    if (tid == 0) s.item_idx = atomicAdd(a.counter, 1);
+  // ---- work decoding shared by all roles (every role runs its own copy of the loops, see the backward kernel)
+  FwdRound rd;
+  int n_rounds = 0, it0 = 0;
+  auto next_pop = [&]() -> bool {
+    if (tid == 0) s.item_idx[gp & 1] = atomicAdd(a.counter, 2);
     tc_fence_before_sync();
-    ok = __syncthreads_and(ok);
+    __syncthreads();
     tc_fence_after_sync();
-    const int it = s.item_idx;
-    if (!ok || it >= a.n_items) break;
+    it0 = s.item_idx[gp & 1];
+    ++gp;
+    if (it0 >= a.n_items || *abort_flag) return false;
+    rd.a = a.items[it0];
+    const bool have_b = it0 + 1 < a.n_items;
+    rd.b = have_b ? a.items[it0 + 1] : rd.a;
+    const SegInfo sg = a.seg[rd.a.seg];
+    const int G = sg.hq / sg.hkv;
+    rd.joint = have_b && rd.b.seg == rd.a.seg && rd.b.tile == rd.a.tile && (rd.a.head / G == rd.b.head / G);
+    n_rounds = rd.joint ? 1 : (have_b ? 2 : 1);
+    return true;
+  };
+  // end of a round: every warp has finished with the Q tiles, the K/V rings and the TMEM accumulators
+  auto round_end = [&]() {
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+  };
 
-    const nsp_tile_t item = a.items[it];
-    const SegInfo sg = a.seg[item.seg];
-    const int h = item.head, g = h / (sg.hq / sg.hkv);
-    const int n_kv = item.cost;
-    const int q_row0 = item.tile * kBM;
-    const int tok0 = sg.tok_in_run;
-    const CUtensorMap* mq = &maps.q[sg.run];
-    const CUtensorMap* mk = &maps.k[sg.run];
-    const CUtensorMap* mv = &maps.v[sg.run];
-
-    if (tid == 0) {
-      mbar_expect_tx(&s.bar_q, kTileBytes);
-      tma_load_3d(s.q[0], mq, &s.bar_q, 0, h, tok0 + q_row0);
-      tma_load_3d(s.q[1], mq, &s.bar_q, 64, h, tok0 + q_row0);
-      mbar_expect_tx(&s.bar_k, kTileBytes);
-      tma_load_3d(s.k[0], mk, &s.bar_k, 0, g, tok0);
-      tma_load_3d(s.k[1], mk, &s.bar_k, 64, g, tok0);
-      mbar_expect_tx(&s.bar_v, kTileBytes);
-      tma_load_3d(s.v[0], mv, &s.bar_v, 0, g, tok0);
-      tma_load_3d(s.v[1], mv, &s.bar_v, 64, g, tok0);
-    }
-
-    float m_ref = -INFINITY;  // reference maximum (log2 domain) the stored P and l are relative to
-    float l = 0.f;            // running row sum of exp2(s - m_ref)
-
-    for (int j = 0; j < n_kv; ++j) {
-      // ---- S = Q K_j^T
-      if (tid == 0) {
-        bool okt = true;
-        if (j == 0) {
-          okt = mbar_wait(&s.bar_q, ph_q);
-          ph_q ^= 1;
-        }
-        okt = okt && mbar_wait(&s.bar_k, ph_k);
-        ph_k ^= 1;
-        if (okt) {
-          tc_fence_after_sync();
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk >> 2) * kHalfTileBytes + (kk & 3) * 32;
-            umma_ss(tS, make_smem_desc_sw128(q_addr + off, 16, 1024), make_smem_desc_sw128(k_addr + off, 16, 1024),
-                    idesc_qk, kk > 0);
+  if (wg == 2) {
+    fwd_setmaxnreg_dec<kFwdRegsAux>();
+    if (warp == 8) {
+      // ================================================================ TMA producer
+      uint32_t kn = 0, vn = 0;
+      while (next_pop()) {
+        for (int r = 0; r < n_rounds; ++r) {
+          if (lane == 0 && !*abort_flag) {
+            const nsp_tile_t ia = r == 0 ? rd.a : rd.b;
+            const SegInfo sg = a.seg[ia.seg];
+            const int g = ia.head / (sg.hq / sg.hkv);
+            const int tok0 = sg.tok_in_run, q_row0 = ia.tile * kBM, n_kv = ia.cost;
+            const CUtensorMap* mq = &maps.q[sg.run];
+            const CUtensorMap* mk = &maps.k[sg.run];
+            const CUtensorMap* mv = &maps.v[sg.run];
+            mbar_expect_tx(&s.bar_q, rd.joint ? 2 * kTileBytes : kTileBytes);
+            tma_load_3d(s.q[0][0], mq, &s.bar_q, 0, ia.head, tok0 + q_row0);
+            tma_load_3d(s.q[0][1], mq, &s.bar_q, 64, ia.head, tok0 + q_row0);
+            if (rd.joint) {
+              tma_load_3d(s.q[1][0], mq, &s.bar_q, 0, rd.b.head, tok0 + q_row0);
+              tma_load_3d(s.q[1][1], mq, &s.bar_q, 64, rd.b.head, tok0 + q_row0);
+            }
+            for (int j = 0; j < n_kv; ++j) {
+              if (*abort_flag) break;
+              uint32_t st = kn & 1;
+              if (!mbar_wait(&s.bar_k_empty[st], ((kn >> 1) & 1) ^ 1)) {
+                report_timeout(a.status, it0, kWhereFwdLoad, j);
+                *abort_flag = 1;
+                break;
+              }
+              mbar_expect_tx(&s.bar_k_full[st], kTileBytes);
+              tma_load_3d(s.k[st][0], mk, &s.bar_k_full[st], 0, g, tok0 + j * kBN);
+              tma_load_3d(s.k[st][1], mk, &s.bar_k_full[st], 64, g, tok0 + j * kBN);
+              ++kn;
+              st = vn & 1;
+              if (!mbar_wait(&s.bar_v_empty[st], ((vn >> 1) & 1) ^ 1)) {
+                report_timeout(a.status, it0, kWhereFwdLoad, 100000 + j);
+                *abort_flag = 1;
+                break;
+              }
+              mbar_expect_tx(&s.bar_v_full[st], kTileBytes);
+              tma_load_3d(s.v[st][0], mv, &s.bar_v_full[st], 0, g, tok0 + j * kBN);
+              tma_load_3d(s.v[st][1], mv, &s.bar_v_full[st], 64, g, tok0 + j * kBN);
+              ++vn;
+            }
           }
-          umma_commit(&s.bar_s);
-        } else {
-          report_timeout(a.status, it, kWhereFwdLoad, j);
+          round_end();
         }
       }
-      bool okw = mbar_wait(&s.bar_s, ph_s);
-      ph_s ^= 1;
-      okw = __all_sync(0xffffffffu, okw);
-      if (okw) {
-        tc_fence_after_sync();
-        if (tid == 0 && j + 1 < n_kv) {  // K buffer is free: prefetch the next key tile
-          mbar_expect_tx(&s.bar_k, kTileBytes);
-          tma_load_3d(s.k[0], mk, &s.bar_k, 0, g, tok0 + (j + 1) * kBN);
-          tma_load_3d(s.k[1], mk, &s.bar_k, 64, g, tok0 + (j + 1) * kBN);
-        }
-        // ---- online softmax of row `tid`
-        uint32_t sr[4][32];
+    } else if (warp == 9) {
+      // ================================================================ MMA issuer
+      constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
+      constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);  // A from TMEM, B MN-major
+      uint32_t qn = 0, kn = 0, vn = 0, pn[2] = {0, 0};
+      while (next_pop()) {
+        for (int r = 0; r < n_rounds; ++r) {
+          if (lane == 0 && !*abort_flag) {
+            const nsp_tile_t ia = r == 0 ? rd.a : rd.b;
+            const int n_kv = ia.cost;
+            const int joint = rd.joint;
+            int where = 0;
+            // S_x of key tile in stage kst -> TMEM columns [128*x, 128*x + 128)
+            auto issue_s = [&](int x, uint32_t kst) {
+              const uint32_t q_addr = smem_u32(s.q[x][0]), k_addr = smem_u32(s.k[kst][0]);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, sr[c]);
-        tmem_wait_ld();
-        const bool diag = (j == n_kv - 1);
-        float mx = -INFINITY;
+              for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t off = (kk >> 2) * kHalfTileBytes + (kk & 3) * 32;
+                umma_ss(tmem + 128 * x, make_smem_desc_sw128(q_addr + off, 16, 1024),
+                        make_smem_desc_sw128(k_addr + off, 16, 1024), idesc_qk, kk > 0);
+              }
+              umma_commit(&s.bar_s_full[x]);
+            };
+            // O_x += P_x V (P_x: bf16 pairs in the first 64 columns of S_x)
+            auto issue_pv = [&](int x, uint32_t vst, int j) {
+              const uint32_t v_addr = smem_u32(s.v[vst][0]);
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int x = 0; x < 32; ++x) {
-            float val = __uint_as_float(sr[c][x]);
-            if (diag && (c * 32 + x) > tid) val = -INFINITY;
-            sr[c][x] = __float_as_uint(val);
-            mx = fmaxf(mx, val);
+              for (int kk = 0; kk < 8; ++kk)
+                umma_ts(tmem + 256 + 128 * x, tmem + 128 * x + kk * 8,
+                        make_smem_desc_sw128(v_addr + kk * 2048, kHalfTileBytes, 1024), idesc_pv, (j > 0 || kk > 0));
+              umma_commit(&s.bar_pv_done[x]);
+            };
+            bool ok = mbar_wait(&s.bar_q, qn & 1);
+            ++qn;
+            if (!ok) where = kWhereFwdLoad;
+            uint32_t kst = 0;
+            for (int j = 0; ok && j < n_kv; ++j) {
+              if (*abort_flag) break;
+              if (j == 0) {
+                kst = kn & 1;
+                if (!mbar_wait(&s.bar_k_full[kst], (kn >> 1) & 1)) { ok = false; where = kWhereFwdLoad; break; }
+                tc_fence_after_sync();
+                issue_s(0, kst);
+                if (joint) issue_s(1, kst);
+                umma_commit(&s.bar_k_empty[kst]);
+                ++kn;
+              }
+              const uint32_t vst = vn & 1;
+              const bool more = j + 1 < n_kv;
+              if (!mbar_wait(&s.bar_p_ready[0], pn[0] & 1)) { ok = false; where = kWhereFwdS; break; }
+              ++pn[0];
+              if (!mbar_wait(&s.bar_v_full[vst], (vn >> 1) & 1)) { ok = false; where = kWhereFwdLoad; break; }
+              tc_fence_after_sync();
+              issue_pv(0, vst, j);
+              if (more) {  // S_A of the next key tile runs while softmax B is still working
+                kst = kn & 1;
+                if (!mbar_wait(&s.bar_k_full[kst], (kn >> 1) & 1)) { ok = false; where = kWhereFwdLoad; break; }
+                tc_fence_after_sync();
+                issue_s(0, kst);
+              }
+              if (joint) {
+                if (!mbar_wait(&s.bar_p_ready[1], pn[1] & 1)) { ok = false; where = kWhereFwdS; break; }
+                ++pn[1];
+                tc_fence_after_sync();
+                issue_pv(1, vst, j);
+              }
+              umma_commit(&s.bar_v_empty[vst]);
+              ++vn;
+              if (more) {
+                if (joint) issue_s(1, kst);
+                umma_commit(&s.bar_k_empty[kst]);
+                ++kn;
+              }
+            }
+            if (!ok) {
+              report_timeout(a.status, it0, where, 0);
+              *abort_flag = 1;
+            }
           }
-        mx *= a.scale_log2;
-        const bool need = mx > m_ref + 8.f;
-        float alpha = 1.f;
-        if (need) {
-          alpha = ex2f(m_ref - mx);
-          m_ref = mx;
+          round_end();
         }
-        l *= alpha;
-        float sum = 0.f;
-        uint32_t pk[2][32];
+      }
+    } else {
+      while (next_pop())
+        for (int r = 0; r < n_rounds; ++r) round_end();  // spare warps: only keep the CTA-wide barrier count
+    }
+  } else {
+    // ================================================================ softmax of item x (A: warps 0-3, B: warps 4-7)
+    fwd_setmaxnreg_inc<kFwdRegsSoftmax>();
+    const int x = wg;
+    const int rl = tid & 127;  // query row inside the tile = TMEM lane
+    const uint32_t tS = tmem + 128 * x, tO = tmem + 256 + 128 * x;
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    uint32_t sn = 0;   // S tiles consumed so far
+    uint32_t pvn = 0;  // PV products of this half issued before the current round
+    while (next_pop()) {
+      for (int r = 0; r < n_rounds; ++r) {
+        const bool active = (x == 0 || rd.joint) && !*abort_flag;
+        if (active) {
+          const nsp_tile_t ia = x == 0 ? (r == 0 ? rd.a : rd.b) : rd.b;
+          const SegInfo sg = a.seg[ia.seg];
+          const int h = ia.head, n_kv = ia.cost, q_row0 = ia.tile * kBM;
+          float m_ref = -INFINITY;  // reference maximum (log2 domain) the stored P and l are relative to
+          float l = 0.f;            // running row sum of exp2(s - m_ref)
+          bool ok = true;
+          int where = 0;
+          for (int j = 0; j < n_kv; ++j) {
+            if (*abort_flag) { ok = false; break; }
+            ok = mbar_wait(&s.bar_s_full[x], sn & 1);
+            ++sn;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) { where = kWhereFwdS; break; }
+            tc_fence_after_sync();
+            uint32_t sr[4][32];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int x = 0; x < 32; x += 2) {
-            const float p0 = ex2f(fmaf(__uint_as_float(sr[c][x]), a.scale_log2, -m_ref));
-            const float p1 = ex2f(fmaf(__uint_as_float(sr[c][x + 1]), a.scale_log2, -m_ref));
-            sum += p0 + p1;
-            pk[c >> 1][(c & 1) * 16 + (x >> 1)] = pack_bf16x2(p0, p1);
-          }
-        l += sum;
-        tmem_st32(tS + lane_off, pk[0]);
-        tmem_st32(tS + lane_off + 32, pk[1]);
-        // ---- rescale O in place when some row of this warp moved its reference maximum
-        if (j > 0 && __any_sync(0xffffffffu, need)) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t orow[32];
-            tmem_ld32(tO + lane_off + c * 32, orow);
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, sr[c]);
             tmem_wait_ld();
+            const bool diag = (j == n_kv - 1);
+            float mx = -INFINITY;
 #pragma unroll
-            for (int x = 0; x < 32; ++x) orow[x] = __float_as_uint(__uint_as_float(orow[x]) * alpha);
-            tmem_st32(tO + lane_off + c * 32, orow);
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                float val = __uint_as_float(sr[c][e]);
+                if (diag && (c * 32 + e) > rl) val = -INFINITY;
+                sr[c][e] = __float_as_uint(val);
+                mx = fmaxf(mx, val);
+              }
+            mx *= a.scale_log2;
+            const bool need = mx > m_ref + 8.f;
+            float alpha = 1.f;
+            if (need) {
+              alpha = ex2f(m_ref - mx);
+              m_ref = mx;
+            }
+            l *= alpha;
+            float sum = 0.f;
+            uint32_t pk[2][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+              for (int e = 0; e < 32; e += 2) {
+                const float p0 = ex2f(fmaf(__uint_as_float(sr[c][e]), a.scale_log2, -m_ref));
+                const float p1 = ex2f(fmaf(__uint_as_float(sr[c][e + 1]), a.scale_log2, -m_ref));
+                sum += p0 + p1;
+                pk[c >> 1][(c & 1) * 16 + (e >> 1)] = pack_bf16x2(p0, p1);
+              }
+            l += sum;
+            tmem_st32(tS + lane_off, pk[0]);
+            tmem_st32(tS + lane_off + 32, pk[1]);
+            // rescale O in place when some row of this warp moved its reference maximum; the previous PV
+            // product of this half must have completed first (the next one is not issued before p_ready)
+            if (j > 0 && __any_sync(0xffffffffu, need)) {
+              ok = mbar_wait(&s.bar_pv_done[x], (pvn + j - 1) & 1);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) { where = kWhereFwdO; break; }
+              tc_fence_after_sync();
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                uint32_t orow[32];
+                tmem_ld32(tO + lane_off + c * 32, orow);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) orow[e] = __float_as_uint(__uint_as_float(orow[e]) * alpha);
+                tmem_st32(tO + lane_off + c * 32, orow);
+              }
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&s.bar_p_ready[x]);
+          }
+          if (ok) {
+            ok = mbar_wait(&s.bar_pv_done[x], (pvn + n_kv - 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) where = kWhereFwdO;
+          }
+          pvn += n_kv;
+          if (ok) {
+            // ---- epilogue: O / l -> bf16, LSE
+            tc_fence_after_sync();
+            const int row = q_row0 + rl;
+            const bool valid = row < sg.len;
+            const float inv_l = 1.f / l;
+            __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              uint32_t orow[32];
+              tmem_ld32(tO + lane_off + c * 32, orow);
+              tmem_wait_ld();
+              if (valid) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  uint4 w;
+                  w.x = pack_bf16x2(__uint_as_float(orow[8 * e + 0]) * inv_l, __uint_as_float(orow[8 * e + 1]) * inv_l);
+                  w.y = pack_bf16x2(__uint_as_float(orow[8 * e + 2]) * inv_l, __uint_as_float(orow[8 * e + 3]) * inv_l);
+                  w.z = pack_bf16x2(__uint_as_float(orow[8 * e + 4]) * inv_l, __uint_as_float(orow[8 * e + 5]) * inv_l);
+                  w.w = pack_bf16x2(__uint_as_float(orow[8 * e + 6]) * inv_l, __uint_as_float(orow[8 * e + 7]) * inv_l);
+                  *reinterpret_cast<uint4*>(optr + c * 32 + e * 8) = w;
+                }
+              }
+            }
+            if (valid)
+              a.lse[sg.lse_off + static_cast<int64_t>(h) * sg.len + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
+          } else if (where != 0 && lane == 0) {
+            report_timeout(a.status, it0, where, 0);
+            *abort_flag = 1;
           }
         }
-        tmem_wait_st();
-      } else if (lane == 0) {
-        report_timeout(a.status, it, kWhereFwdS, j);
-      }
-      ok = ok && okw;
-      tc_fence_before_sync();
-      ok = __syncthreads_and(ok);
-      if (!ok) break;
-      // ---- O += P V_j
-      if (tid == 0) {
-        const bool okt = mbar_wait(&s.bar_v, ph_v);
-        ph_v ^= 1;
-        if (okt) {
-          tc_fence_after_sync();
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            umma_ts(tO, tS + kk * 8, make_smem_desc_sw128(v_addr + kk * 2048, kHalfTileBytes, 1024), idesc_pv,
-                    (j > 0 || kk > 0));
-          umma_commit(&s.bar_o);
-        } else {
-          report_timeout(a.status, it, kWhereFwdLoad, 1000 + j);
-        }
-      }
-      okw = mbar_wait(&s.bar_o, ph_o);
-      ph_o ^= 1;
-      okw = __all_sync(0xffffffffu, okw);
-      if (okw) {
-        tc_fence_after_sync();
-        if (tid == 0 && j + 1 < n_kv) {  // V buffer is free
-          mbar_expect_tx(&s.bar_v, kTileBytes);
-          tma_load_3d(s.v[0], mv, &s.bar_v, 0, g, tok0 + (j + 1) * kBN);
-          tma_load_3d(s.v[1], mv, &s.bar_v, 64, g, tok0 + (j + 1) * kBN);
-        }
-      } else if (lane == 0) {
-        report_timeout(a.status, it, kWhereFwdO, j);
-      }
-      ok = ok && okw;
-    }
-    if (!ok) continue;  // the uniform vote at the loop head ends the CTA
-
-    // ---- epilogue: O / l -> bf16, LSE
-    const int row = q_row0 + tid;
-    const bool valid = row < sg.len;
-    const float inv_l = 1.f / l;
-    __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint32_t orow[32];
-      tmem_ld32(tO + lane_off + c * 32, orow);
-      tmem_wait_ld();
-      if (valid) {
-#pragma unroll
-        for (int x = 0; x < 4; ++x) {
-          uint4 w;
-          w.x = pack_bf16x2(__uint_as_float(orow[8 * x + 0]) * inv_l, __uint_as_float(orow[8 * x + 1]) * inv_l);
-          w.y = pack_bf16x2(__uint_as_float(orow[8 * x + 2]) * inv_l, __uint_as_float(orow[8 * x + 3]) * inv_l);
-          w.z = pack_bf16x2(__uint_as_float(orow[8 * x + 4]) * inv_l, __uint_as_float(orow[8 * x + 5]) * inv_l);
-          w.w = pack_bf16x2(__uint_as_float(orow[8 * x + 6]) * inv_l, __uint_as_float(orow[8 * x + 7]) * inv_l);
-          *reinterpret_cast<uint4*>(optr + c * 32 + x * 8) = w;
-        }
+        round_end();
       }
     }
-    if (valid)
-      a.lse[sg.lse_off + static_cast<int64_t>(h) * sg.len + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
   }
 
   tc_fence_before_sync();
@@ -255,14 +391,11 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_kernel(const __grid_consta
 
 cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st) {
   if (args.n_items == 0) return cudaSuccess;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kFwdSmemBytes));
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  const int grid = args.n_items < 2 * num_sms ? args.n_items : 2 * num_sms;
+  cudaError_t e = cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(kFwdSmemBytes));
+  if (e != cudaSuccess) return e;
+  const int pops = (args.n_items + 1) / 2;
+  const int grid = pops < num_sms ? pops : num_sms;
   fwd_kernel<<<grid, kFwdThreads, kFwdSmemBytes, st>>>(maps, args);
   count_launches(1);
   return cudaGetLastError();

@@ -45,6 +45,7 @@ enum DeviceWhere : int32_t {
   kWhereFwdLoad = 1,
   kWhereFwdS = 2,
   kWhereFwdO = 3,
+  kWhereFwdSmemAlign = 4,
   kWhereBwdLoadKV = 11,
   kWhereBwdLoadQ = 12,
   kWhereBwdS = 13,
