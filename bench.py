@@ -34,8 +34,8 @@ from paper_2609_22755_b200 import workloads as W  # noqa: E402
 METRIC = "causal attention TFLOP/s fwd+bwd on 1 B200 and % of dense BF16 roofline"
 UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one backward-main launch on the bench workload, from the ncu
-# capture summarised under profiles/ (scaled from a smaller case where stated there); None until captured.
-BWD_MAIN_DRAM_TRAFFIC_BYTES = None
+# capture summarised in profiles/bwd_kernel_nested_profile_case_64k.md (captured on a smaller case, scaled there).
+BWD_MAIN_DRAM_TRAFFIC_BYTES = int(4.128e9 * 5.0)  # 4.13 GB on the 64K profile case x 5.0 (ratio of Q elements)
 
 
 def measured_peaks():

@@ -28,6 +28,17 @@ constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;
 constexpr uint32_t kFwdTmemCols = 512;  // S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512)
 constexpr int kFwdRegsSoftmax = 216, kFwdRegsAux = 72;  // 2*216 + 72 = 504 = 3 * 168, the launch-time allocation
 
+// Optional timeline (compiled in only with -DNSP_TRACE, for tuning): clock64 stamps of the first CTA's roles.
+#ifdef NSP_TRACE
+__device__ long long g_ftrace[64 * 24];
+#define NSP_FTRACE(slot)                                                                                          \
+  do {                                                                                                            \
+    if (blockIdx.x == 0 && gp == 1 && j >= 100 && j < 164) g_ftrace[(j - 100) * 24 + (slot)] = clock64();         \
+  } while (0)
+#else
+#define NSP_FTRACE(slot)
+#endif
+
 struct FwdSmem {
   uint8_t q[2][2][kHalfTileBytes];  // [A/B][64-column half]
   uint8_t k[2][2][kHalfTileBytes];  // [stage][half]
@@ -220,6 +231,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               const bool more = j + 1 < n_kv;
               if (!mbar_wait(&s.bar_p_ready[0], pn[0] & 1)) { ok = false; where = kWhereFwdS; break; }
               ++pn[0];
+              NSP_FTRACE(0);
               if (!mbar_wait(&s.bar_v_full[vst], (vn >> 1) & 1)) { ok = false; where = kWhereFwdLoad; break; }
               tc_fence_after_sync();
               issue_pv(0, vst, j);
@@ -229,9 +241,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 tc_fence_after_sync();
                 issue_s(0, kst);
               }
+              NSP_FTRACE(1);
               if (joint) {
                 if (!mbar_wait(&s.bar_p_ready[1], pn[1] & 1)) { ok = false; where = kWhereFwdS; break; }
                 ++pn[1];
+                NSP_FTRACE(2);
                 tc_fence_after_sync();
                 issue_pv(1, vst, j);
               }
@@ -242,6 +256,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 umma_commit(&s.bar_k_empty[kst]);
                 ++kn;
               }
+              NSP_FTRACE(3);
             }
             if (!ok) {
               report_timeout(a.status, it0, where, 0);
@@ -281,11 +296,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             ++sn;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { where = kWhereFwdS; break; }
+            if (rl == 0) NSP_FTRACE(4 + 8 * x);
             tc_fence_after_sync();
             uint32_t sr[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, sr[c]);
             tmem_wait_ld();
+            if (rl == 0) NSP_FTRACE(5 + 8 * x);
             const bool diag = (j == n_kv - 1);
             float mx = -INFINITY;
 #pragma unroll
@@ -305,6 +322,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               m_ref = mx;
             }
             l *= alpha;
+            if (rl == 0) NSP_FTRACE(6 + 8 * x);
+            if (rl == 0) NSP_FTRACE(7 + 8 * x);
             float sum = 0.f;
             uint32_t pk[2][32];
 #pragma unroll
@@ -319,6 +338,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             l += sum;
             tmem_st32(tS + lane_off, pk[0]);
             tmem_st32(tS + lane_off + 32, pk[1]);
+            if (rl == 0) NSP_FTRACE(8 + 8 * x);
             // rescale O in place when some row of this warp moved its reference maximum; the previous PV
             // product of this half must have completed first (the next one is not issued before p_ready)
             if (j > 0 && __any_sync(0xffffffffu, need)) {
@@ -339,6 +359,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&s.bar_p_ready[x]);
+            if (rl == 0) NSP_FTRACE(9 + 8 * x);
           }
           if (ok) {
             ok = mbar_wait(&s.bar_pv_done[x], (pvn + n_kv - 1) & 1);
@@ -388,6 +409,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
 }
 
 }  // namespace
+
+#ifdef NSP_TRACE
+extern "C" int nsp_debug_ftrace_read(long long* host, int n) {
+  return cudaMemcpyFromSymbol(host, g_ftrace, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st) {
   if (args.n_items == 0) return cudaSuccess;

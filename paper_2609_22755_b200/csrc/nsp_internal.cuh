@@ -46,6 +46,7 @@ enum DeviceWhere : int32_t {
   kWhereFwdS = 2,
   kWhereFwdO = 3,
   kWhereFwdSmemAlign = 4,
+  kWhereFwdTurn = 5,
   kWhereBwdLoadKV = 11,
   kWhereBwdLoadQ = 12,
   kWhereBwdS = 13,
