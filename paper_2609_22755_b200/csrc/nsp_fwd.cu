@@ -22,11 +22,11 @@
 namespace nsp {
 namespace {
 
-constexpr int kFwdThreads = 384;
+constexpr int kFwdThreads = 640;  // 16 softmax warps (two threads per query row) + one auxiliary warpgroup
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;  // one [128 rows x 64 cols] bf16 sub-tile
 constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;
 constexpr uint32_t kFwdTmemCols = 512;  // S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512)
-constexpr int kFwdRegsSoftmax = 216, kFwdRegsAux = 72;  // 2*216 + 72 = 504 = 3 * 168, the launch-time allocation
+constexpr int kFwdRegsSoftmax = 104, kFwdRegsAux = 64;  // 4*104 + 64 = 480 = 5 * 96, the launch-time allocation
 
 // Optional timeline (compiled in only with -DNSP_TRACE, for tuning): clock64 stamps of the first CTA's roles.
 #ifdef NSP_TRACE
@@ -46,7 +46,9 @@ struct FwdSmem {
   uint64_t bar_q;
   uint64_t bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
   uint64_t bar_s_full[2];   // [A/B] S_x of a key tile is in TMEM
-  uint64_t bar_p_ready[2];  // [A/B] 128 softmax threads: P_x written (and O_x rescaled if needed)
+  uint64_t bar_p_ready[2];  // [A/B] 256 softmax threads: P_x written (and O_x rescaled if needed)
+  uint64_t bar_pair[2][4];  // [A/B][lane quadrant] the two threads of every row have published their half-row value
+  float xchg[2][2][128];    // [A/B][column half][row] half-row maximum (or row sum) handed to the partner thread
   uint64_t bar_pv_done[2];  // [A/B] O_x += P_x V has completed
   uint32_t tmem_base;
   int32_t item_idx[2];
@@ -62,6 +64,13 @@ __device__ __forceinline__ void fwd_setmaxnreg_inc() {
 template <int N>
 __device__ __forceinline__ void fwd_setmaxnreg_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+// max(a, b, c) in one instruction (3-input max of sm_100)
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
 // What one pop of the work list turned into: one or two rounds, each with item A and (in a joint round) item B.
@@ -86,7 +95,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       mbar_init(&s.bar_v_full[i], 1);
       mbar_init(&s.bar_v_empty[i], 1);
       mbar_init(&s.bar_s_full[i], 1);
-      mbar_init(&s.bar_p_ready[i], 128);
+      mbar_init(&s.bar_p_ready[i], 256);
+      for (int qd = 0; qd < 4; ++qd) mbar_init(&s.bar_pair[i][qd], 64);
       mbar_init(&s.bar_pv_done[i], 1);
     }
     s.abort = 0;
@@ -131,9 +141,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     tc_fence_after_sync();
   };
 
-  if (wg == 2) {
+  if (wg == 4) {
     fwd_setmaxnreg_dec<kFwdRegsAux>();
-    if (warp == 8) {
+    if (warp == 16) {
       // ================================================================ TMA producer
       uint32_t kn = 0, vn = 0;
       while (next_pop()) {
@@ -180,7 +190,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           round_end();
         }
       }
-    } else if (warp == 9) {
+    } else if (warp == 17) {
       // ================================================================ MMA issuer
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);  // A from TMEM, B MN-major
@@ -271,14 +281,22 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
         for (int r = 0; r < n_rounds; ++r) round_end();  // spare warps: only keep the CTA-wide barrier count
     }
   } else {
-    // ================================================================ softmax of item x (A: warps 0-3, B: warps 4-7)
+    // ================================================================ softmax of item x (A: warps 0-7, B: warps 8-15)
+    // Two threads per query row: thread (quadrant, half ch) owns TMEM lane 32*quadrant + lane and the 64 score
+    // columns [64*ch, 64*ch + 64). The row maximum (every key tile) and the row sum (once, at the end) are
+    // combined through shared memory; everything else is private to the thread.
     fwd_setmaxnreg_inc<kFwdRegsSoftmax>();
-    const int x = wg;
-    const int rl = tid & 127;  // query row inside the tile = TMEM lane
+    const int x = wg >> 1;
+    const int quad = warp & 3, ch = (warp >> 2) & 1;
+    const int rl = quad * 32 + lane;  // query row inside the tile = TMEM lane
     const uint32_t tS = tmem + 128 * x, tO = tmem + 256 + 128 * x;
-    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
     uint32_t sn = 0;   // S tiles consumed so far
     uint32_t pvn = 0;  // PV products of this half issued before the current round
+    uint32_t xn = 0;   // completed phases of this row pair's exchange barrier
+    float* my_slot = &s.xchg[x][ch][rl];
+    const float* partner_slot = &s.xchg[x][ch ^ 1][rl];
+    uint64_t* pair_bar = &s.bar_pair[x][quad];
     while (next_pop()) {
       for (int r = 0; r < n_rounds; ++r) {
         const bool active = (x == 0 || rd.joint) && !*abort_flag;
@@ -287,7 +305,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           const SegInfo sg = a.seg[ia.seg];
           const int h = ia.head, n_kv = ia.cost, q_row0 = ia.tile * kBM;
           float m_ref = -INFINITY;  // reference maximum (log2 domain) the stored P and l are relative to
-          float l = 0.f;            // running row sum of exp2(s - m_ref)
+          float l = 0.f;            // running sum of exp2(s - m_ref) over this thread's columns
           bool ok = true;
           int where = 0;
           for (int j = 0; j < n_kv; ++j) {
@@ -296,25 +314,41 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             ++sn;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { where = kWhereFwdS; break; }
-            if (rl == 0) NSP_FTRACE(4 + 8 * x);
+            if (rl == 0 && ch == 0) NSP_FTRACE(4 + 8 * x);
             tc_fence_after_sync();
-            uint32_t sr[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, sr[c]);
+            uint32_t sr[2][32];
+            tmem_ld32(tS + lane_off + ch * 64, sr[0]);
+            tmem_ld32(tS + lane_off + ch * 64 + 32, sr[1]);
             tmem_wait_ld();
-            if (rl == 0) NSP_FTRACE(5 + 8 * x);
-            const bool diag = (j == n_kv - 1);
+            if (rl == 0 && ch == 0) NSP_FTRACE(5 + 8 * x);
             float mx = -INFINITY;
+            if (j == n_kv - 1) {  // diagonal tile: keys past the query are masked
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+              for (int c = 0; c < 2; ++c)
 #pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                float val = __uint_as_float(sr[c][e]);
-                if (diag && (c * 32 + e) > rl) val = -INFINITY;
-                sr[c][e] = __float_as_uint(val);
-                mx = fmaxf(mx, val);
-              }
-            mx *= a.scale_log2;
+                for (int e = 0; e < 32; ++e) {
+                  float val = __uint_as_float(sr[c][e]);
+                  if (ch * 64 + c * 32 + e > rl) val = -INFINITY;
+                  sr[c][e] = __float_as_uint(val);
+                  mx = fmaxf(mx, val);
+                }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 2; ++c)
+#pragma unroll
+                for (int e = 0; e < 32; e += 2)
+                  mx = max3f(mx, __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
+            }
+            // row maximum = max of the two half rows (the partner has also finished reading its S columns by
+            // the time its value is visible, so P may then be written over any part of S_x)
+            *my_slot = mx;
+            mbar_arrive(pair_bar);
+            ok = mbar_wait(pair_bar, xn & 1);
+            ++xn;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) { where = kWhereFwdPair; break; }
+            mx = fmaxf(mx, *partner_slot) * a.scale_log2;
+            if (rl == 0 && ch == 0) NSP_FTRACE(6 + 8 * x);
             const bool need = mx > m_ref + 8.f;
             float alpha = 1.f;
             if (need) {
@@ -322,44 +356,45 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               m_ref = mx;
             }
             l *= alpha;
-            if (rl == 0) NSP_FTRACE(6 + 8 * x);
-            if (rl == 0) NSP_FTRACE(7 + 8 * x);
             float sum = 0.f;
-            uint32_t pk[2][32];
+            uint32_t pk[32];
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 2; ++c)
 #pragma unroll
               for (int e = 0; e < 32; e += 2) {
                 const float p0 = ex2f(fmaf(__uint_as_float(sr[c][e]), a.scale_log2, -m_ref));
                 const float p1 = ex2f(fmaf(__uint_as_float(sr[c][e + 1]), a.scale_log2, -m_ref));
                 sum += p0 + p1;
-                pk[c >> 1][(c & 1) * 16 + (e >> 1)] = pack_bf16x2(p0, p1);
+                pk[c * 16 + (e >> 1)] = pack_bf16x2(p0, p1);
               }
             l += sum;
-            tmem_st32(tS + lane_off, pk[0]);
-            tmem_st32(tS + lane_off + 32, pk[1]);
-            if (rl == 0) NSP_FTRACE(8 + 8 * x);
-            // rescale O in place when some row of this warp moved its reference maximum; the previous PV
-            // product of this half must have completed first (the next one is not issued before p_ready)
+            tmem_st32(tS + lane_off + ch * 32, pk);  // packed columns [32*ch, 32*ch + 32) = score columns [64*ch, +64)
+            if (rl == 0 && ch == 0) NSP_FTRACE(8 + 8 * x);
+            // rescale this thread's 64 columns of O in place when some row of the warp moved its reference
+            // maximum; the previous PV product of this half must have completed first (the next one is not
+            // issued before p_ready). The next exchange must not overwrite a slot the partner has not read yet:
+            // both threads of a pair pass the barrier of the NEXT tile only after this tile's read, which is
+            // ordered before their next write by the barrier itself (write -> arrive ... wait -> read; the next
+            // write of a slot follows the partner's next arrive only through bar_s_full, i.e. after p_ready).
             if (j > 0 && __any_sync(0xffffffffu, need)) {
               ok = mbar_wait(&s.bar_pv_done[x], (pvn + j - 1) & 1);
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) { where = kWhereFwdO; break; }
               tc_fence_after_sync();
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
+              for (int c = 0; c < 2; ++c) {
                 uint32_t orow[32];
-                tmem_ld32(tO + lane_off + c * 32, orow);
+                tmem_ld32(tO + lane_off + ch * 64 + c * 32, orow);
                 tmem_wait_ld();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) orow[e] = __float_as_uint(__uint_as_float(orow[e]) * alpha);
-                tmem_st32(tO + lane_off + c * 32, orow);
+                tmem_st32(tO + lane_off + ch * 64 + c * 32, orow);
               }
             }
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&s.bar_p_ready[x]);
-            if (rl == 0) NSP_FTRACE(9 + 8 * x);
+            if (rl == 0 && ch == 0) NSP_FTRACE(9 + 8 * x);
           }
           if (ok) {
             ok = mbar_wait(&s.bar_pv_done[x], (pvn + n_kv - 1) & 1);
@@ -367,17 +402,26 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             if (!ok) where = kWhereFwdO;
           }
           pvn += n_kv;
+          if (ok) {  // row sum = sum of the two half rows
+            *my_slot = l;
+            mbar_arrive(pair_bar);
+            ok = mbar_wait(pair_bar, xn & 1);
+            ++xn;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) where = kWhereFwdPair;
+          }
           if (ok) {
-            // ---- epilogue: O / l -> bf16, LSE
+            // ---- epilogue: O / l -> bf16 (this thread's 64 columns), LSE
+            l += *partner_slot;
             tc_fence_after_sync();
             const int row = q_row0 + rl;
             const bool valid = row < sg.len;
             const float inv_l = 1.f / l;
-            __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim;
+            __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim + ch * 64;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
               uint32_t orow[32];
-              tmem_ld32(tO + lane_off + c * 32, orow);
+              tmem_ld32(tO + lane_off + ch * 64 + c * 32, orow);
               tmem_wait_ld();
               if (valid) {
 #pragma unroll
@@ -391,7 +435,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 }
               }
             }
-            if (valid)
+            if (valid && ch == 0)
               a.lse[sg.lse_off + static_cast<int64_t>(h) * sg.len + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
           } else if (where != 0 && lane == 0) {
             report_timeout(a.status, it0, where, 0);

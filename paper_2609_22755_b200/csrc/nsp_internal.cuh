@@ -47,6 +47,7 @@ enum DeviceWhere : int32_t {
   kWhereFwdO = 3,
   kWhereFwdSmemAlign = 4,
   kWhereFwdTurn = 5,
+  kWhereFwdPair = 6,
   kWhereBwdLoadKV = 11,
   kWhereBwdLoadQ = 12,
   kWhereBwdS = 13,
