@@ -75,24 +75,6 @@ bool encode_run_map(CUtensorMap* out, const void* base, int64_t elem_off, int64_
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// fp32 [tokens, heads, 128] accumulator of one run; tiles are {32 dims, 1 head, 128 tokens}, 128-byte swizzle.
-bool encode_run_map_f32(CUtensorMap* out, const void* base, int64_t elem_off, int64_t tokens, int heads) {
-  EncodeTiledFn enc = get_encode_fn();
-  if (!enc) return false;
-  if (tokens <= 0) {
-    std::memset(out, 0, sizeof(*out));
-    return true;
-  }
-  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(kHeadDim), static_cast<cuuint64_t>(heads),
-                              static_cast<cuuint64_t>(tokens)};
-  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(kHeadDim) * 4, static_cast<cuuint64_t>(heads) * kHeadDim * 4};
-  const cuuint32_t box[3] = {32, 1, 128};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  void* ptr = const_cast<char*>(static_cast<const char*>(base)) + elem_off * 4;
-  return enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -376,7 +358,6 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
     const RunInfo& run = plan->runs[r];
     if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq) ||
         !encode_run_map(&maps.d_o[r], d_o, run.q_off, run.tokens, run.hq) ||
-        !encode_run_map_f32(&maps.dq[r], dq_acc, run.q_off, run.tokens, run.hq) ||
         !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv) ||
         !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv))
       return NSP_ERR_CUDA;

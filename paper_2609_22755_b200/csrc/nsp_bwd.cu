@@ -5,7 +5,7 @@
 //   main         key-stationary persistent kernel, see below
 //   postprocess  dQ = scale * fp32 accumulator -> bf16 / fp32                   (HBM-bound)
 //
-// Main kernel. One CTA per SM (512 threads, four warpgroups with their own register budgets) pops items
+// Main kernel. One CTA per SM (640 threads, five warpgroups with their own register budgets) pops items
 // (segment, kv head, key tile n) from the longest-first list. K_n and V_n stay in shared memory; the CTA walks
 // every q head of the KV group and every q tile m >= n. All score-shaped quantities are computed TRANSPOSED
 // (key index on the TMEM lanes) so that P^T and dS^T are directly the A operands of the dV and dK products:
@@ -13,19 +13,30 @@
 //     P^T  = exp2(S^T * scale*log2e - LSE*log2e),  dS^T = P^T o (dP^T - delta)
 //     dV  += P^T dO                               A = P^T (bf16, written over S^T in R0), B = dO  MN-major
 //     dK  += dS^T Q                               A = dS^T (shared memory, K-major), B = Q MN-major
-//     dQ_m = dS K  -> R1 (over dP^T)              A = dS^T read MN-major, B = K MN-major
+//     dQ_m^T = K^T dS^T -> R1 (over dP^T)         A = K read MN-major, B = dS^T read MN-major
 // TMEM: R0 [0,128), R1 [128,256), dK [256,384), dV [384,512).
 // Roles:  warps 0-7  softmax / dS (key row = TMEM lane, two column halves)
-//         warps 8-11 dQ: TMEM -> fp32 accumulator in global memory (vector reductions)
-//         warp 12    TMA producer (K, V once per item; Q, dO two-stage ring)
-//         warp 13    MMA issuer (single thread)
-//         warp 14    LSE / delta loader (two-stage ring in shared memory)
-// The MMA thread issues S^T of the next step right behind dQ of the current one, so the next S^T runs while
-// the dQ warps drain R1; dP^T waits for R1. dK and dV accumulate in TMEM over the whole item in a fixed order
-// (heads ascending, tiles ascending), so the reduction over the query heads of a group is deterministic.
+//         warps 8-15 dQ: TMEM -> fp32 accumulator in global memory (lane quadrant x 64-column half)
+//         warp 16    TMA producer (K, V once per item; Q, dO two-stage ring)
+//         warp 17    MMA issuer A (single thread): dV(t), S^T(t+1)
+//         warp 18    LSE / delta loader (two-stage ring in shared memory)
+//         warp 19    MMA issuer B (single thread): dK(t), dQ^T(t), dP^T(t+1)
+// The softmax warps hand over P^T first (p_ready) and dS^T second (ds_ready), so dV(t) and S^T(t+1) run under
+// the dS phase of step t, and dK(t), dQ^T(t), dP^T(t+1) under the exp2 phase of step t+1.
+// dQ is produced TRANSPOSED (head dimension on the TMEM lanes): a warp of the dQ warpgroups then holds 32
+// consecutive head-dimension values of one query row per register, and a plain red.global.add.f32 per register
+// is one fully coalesced 128-byte reduction into the fp32 accumulator. No shared-memory staging: shared-memory
+// bandwidth (MMA operand reads, TMA fills, dS^T) is a scarce resource of this kernel.
+// dK and dV accumulate in TMEM over the whole item in a fixed order (heads ascending, tiles ascending), so the
+// reduction over the query heads of a group is deterministic.
 // For the first q tile of a segment (rows 0..127, where P is O(1)) the step runs twice, once with the bf16
 // value of P and dS and once with the bf16 residual (hi + lo), and delta is recomputed in fp32 as
 // sum_j P_ij dP_ij instead of taking it from the bf16-rounded O; this keeps dK/dV/dQ inside the 2e-2 tolerance.
+//
+// Code size matters here: twenty warps of five roles share one instruction cache, and a step loop whose roles
+// together do not fit in it runs at the speed of instruction fetch. So the common step (an interior tile) has
+// its own lean, fully unrolled path; everything rare (diagonal tile, first-tile passes, ragged tail, item
+// epilogue) goes through compact rolled loops; an item is decoded once, by one thread, into shared memory.
 #include <cuda_bf16.h>
 #include "nsp_internal.cuh"
 #include "sm100_ptx.cuh"
@@ -33,12 +44,36 @@
 namespace nsp {
 namespace {
 
-constexpr int kBwdThreads = 512;
+constexpr int kBwdThreads = 640;  // 8 softmax warps, 8 dQ warps, one auxiliary warpgroup
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;
 constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kRegsSoftmax = 168, kRegsReduce = 120, kRegsAux = 56;  // 2*168 + 120 + 56 = 512 = 65536 / 128
+// setmaxnreg redistributes the launch-time allocation (96 per thread): 256*136 + 256*80 + 128*48 = 640*96
+constexpr int kRegsSoftmax = 136, kRegsReduce = 80, kRegsAux = 48;
+
+// Optional step timeline (compiled in only with -DNSP_TRACE, for tuning): clock64 stamps of the first CTA's roles.
+#ifdef NSP_TRACE
+__device__ long long g_trace[64 * 24];
+#define NSP_TRACE_STAMP(slot)                                                                               \
+  do {                                                                                                      \
+    if (blockIdx.x == 0 && gi == 0 && vt >= 200 && vt < 264) g_trace[(vt - 200) * 24 + (slot)] = clock64(); \
+  } while (0)
+#else
+#define NSP_TRACE_STAMP(slot)
+#endif
+
+// A decoded work item: written by thread 0, read by every role after the CTA-wide barrier of next_item().
+struct ItemCtx {
+  int64_t q_off, kv_off, lse_off;  // element offsets of the segment
+  int32_t it;                      // position in the work list (>= n_items: no more work)
+  int32_t len, hq, hkv, run, tok0;
+  int32_t g, n;                    // kv head, key tile
+  int32_t G;                       // q heads per kv head
+  int32_t first, two_pass, mode_first;
+  int32_t per_head;                // steps per q head
+  int32_t steps;                   // G * per_head
+};
 
 struct BwdSmem {
   uint8_t k[2][kHalfTileBytes];
@@ -48,21 +83,24 @@ struct BwdSmem {
   uint8_t ds[2][kHalfTileBytes];      // dS^T, [key row][query col], two 64-column halves
   float lse[2][128];                  // [stage] LSE * log2(e) of the q tile (+inf for rows past the segment)
   float delta[2][128];                // [stage]
+  ItemCtx ctx[2];
   uint64_t bar_kv;
-  uint64_t bar_q_full[2], bar_q_empty[2];
+  uint64_t bar_q_full[2];
+  uint64_t bar_q_empty[2][2];  // [stage][issuer A / B]: that issuer's MMAs reading the stage have completed
+  uint64_t bar_a_done;         // dV of the step (issuer A) has completed
   uint64_t bar_ld_full[2], bar_ld_empty[2];
-  uint64_t bar_s_full, bar_dp_full, bar_p_ready, bar_dq_full, bar_dq_empty;
-  uint64_t bar_staged;    // 128 dQ threads: the fp32 dQ tile is in the staging buffer
+  uint64_t bar_s_full, bar_dp_full, bar_dq_full, bar_dq_empty;
+  uint64_t bar_p_ready;   // 256 softmax threads: P^T of the step is in R0
+  uint64_t bar_ds_ready;  // 256 softmax threads: dS^T of the step is in shared memory
   uint64_t bar_delta[2];  // 128 softmax threads of one column half: partial / final sums of the exact delta
   uint32_t tmem_base;
-  int32_t item_idx[2];
   int32_t abort;
 };
 static_assert(sizeof(BwdSmem) <= 232448, "shared memory budget (227 KB)");
 constexpr size_t kBwdSmemBytes = sizeof(BwdSmem);
 
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+__device__ __forceinline__ void red_add_f32(float* addr, float v) {
+  asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
 }
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
@@ -72,34 +110,30 @@ template <int N>
 __device__ __forceinline__ void setmaxnreg_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
-__device__ __forceinline__ void named_barrier(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
 
-// Decoded work item and the mapping from a step index to (q head, q tile, mode).
+// Walks the steps of an item: q heads of the group in ascending order, per head the q tiles in ascending order.
 // mode bit 0: recompute delta exactly; bit 1: residual (lo) pass of the hi/lo split.
-struct ItemCtx {
-  int g, n, G, n_m, per_head, steps, first, two_pass, mode_first;
-};
-__device__ __forceinline__ void decode_step(const ItemCtx& c, int vt, int& h, int& m, int& mode) {
-  const int hh = vt / c.per_head, rr = vt - hh * c.per_head;
-  h = c.g * c.G + hh;
-  if (c.first) {
-    if (rr == 0) {
-      m = 0;
-      mode = c.mode_first;
-    } else if (c.two_pass && rr == 1) {
-      m = 0;
-      mode = c.mode_first | 2;
-    } else {
-      m = rr - c.two_pass;
-      mode = 0;
-    }
-  } else {
+struct StepWalk {
+  int hh, rr;
+  __device__ __forceinline__ void reset() { hh = 0, rr = 0; }
+  __device__ __forceinline__ void get(const ItemCtx& c, int& h, int& m, int& mode) const {
+    h = c.g * c.G + hh;
     m = c.n + rr;
     mode = 0;
+    if (c.first) {
+      if (rr == 0) {
+        m = 0, mode = c.mode_first;
+      } else if (c.two_pass && rr == 1) {
+        m = 0, mode = c.mode_first | 2;
+      } else {
+        m = rr - c.two_pass;
+      }
+    }
   }
-}
+  __device__ __forceinline__ void next(const ItemCtx& c) {
+    if (++rr == c.per_head) rr = 0, ++hh;
+  }
+};
 
 __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -114,16 +148,18 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     mbar_init(&s.bar_kv, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s.bar_q_full[i], 1);
-      mbar_init(&s.bar_q_empty[i], 1);
+      mbar_init(&s.bar_q_empty[i][0], 1);
+      mbar_init(&s.bar_q_empty[i][1], 1);
       mbar_init(&s.bar_ld_full[i], 32);
       mbar_init(&s.bar_ld_empty[i], 256);
     }
     mbar_init(&s.bar_s_full, 1);
     mbar_init(&s.bar_dp_full, 1);
     mbar_init(&s.bar_p_ready, 256);
+    mbar_init(&s.bar_ds_ready, 256);
     mbar_init(&s.bar_dq_full, 1);
-    mbar_init(&s.bar_dq_empty, 128);
-    mbar_init(&s.bar_staged, 128);
+    mbar_init(&s.bar_a_done, 1);
+    mbar_init(&s.bar_dq_empty, 256);
     mbar_init(&s.bar_delta[0], 128);
     mbar_init(&s.bar_delta[1], 128);
     s.abort = 0;
@@ -137,175 +173,255 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   __syncthreads();
   tc_fence_after_sync();
 
-  const uint32_t tR0 = s.tmem_base, tR1 = tR0 + 128, tDK = tR0 + 256, tDV = tR0 + 384;
+  // The CTA owns all 512 TMEM columns, so the allocation starts at column 0 and every TMEM address is a
+  // compile-time constant.
+  constexpr uint32_t tR0 = 0, tR1 = 128, tDK = 256, tDV = 384;
+  if (s.tmem_base != 0) {
+    if (tid == 0) report_timeout(a.status, -1, kWhereBwdTmemBase, static_cast<int32_t>(s.tmem_base));
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(s.tmem_base, kBwdTmemCols);
+    return;
+  }
   volatile int32_t* abort_flag = &s.abort;
   uint32_t gs = 0;  // steps completed so far by this CTA (every role advances it identically)
   uint32_t gi = 0;  // items completed so far
 
   // Every role runs its own copy of the item loop (so that its register budget, set by setmaxnreg at the top of
   // the role, governs the whole loop); the loops meet at the CTA-wide barrier inside next_item().
-  nsp_tile_t item;
-  SegInfo sg;
-  ItemCtx c;
-  int it = 0, tok0 = 0;
+  const ItemCtx* cx = nullptr;
   auto next_item = [&]() -> bool {
-    if (tid == 0) s.item_idx[gi & 1] = atomicAdd(a.counter, 1);
+    ItemCtx& x = s.ctx[gi & 1];
+    if (tid == 0) {
+      const int idx = atomicAdd(a.counter, 1);
+      x.it = idx;
+      if (idx < a.n_items) {
+        const nsp_tile_t item = a.items[idx];
+        const SegInfo sg = a.seg[item.seg];
+        x.q_off = sg.q_off, x.kv_off = sg.kv_off, x.lse_off = sg.lse_off;
+        x.len = sg.len, x.hq = sg.hq, x.hkv = sg.hkv, x.run = sg.run, x.tok0 = sg.tok_in_run;
+        x.g = item.head, x.n = item.tile;
+        x.G = sg.hq / sg.hkv;
+        x.first = (item.tile == 0);
+        x.two_pass = (x.first && (a.debug_flags & 1) == 0) ? 1 : 0;
+        x.mode_first = (a.debug_flags & 2) == 0 ? 1 : 0;
+        x.per_head = (sg.len + kBM - 1) / kBM - item.tile + x.two_pass;  // q tiles n .. Mt-1 (bm == bn)
+        x.steps = x.G * x.per_head;
+      }
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    it = s.item_idx[gi & 1];
-    if (it >= a.n_items || *abort_flag) return false;
-    item = a.items[it];
-    sg = a.seg[item.seg];
-    c.g = item.head;
-    c.n = item.tile;
-    c.G = sg.hq / sg.hkv;
-    c.n_m = (sg.len + kBM - 1) / kBM - c.n;  // q tiles n .. Mt-1 (bm == bn)
-    c.first = (c.n == 0);
-    c.two_pass = (c.first && (a.debug_flags & 1) == 0) ? 1 : 0;
-    c.mode_first = (a.debug_flags & 2) == 0 ? 1 : 0;
-    c.per_head = c.n_m + c.two_pass;
-    c.steps = c.G * c.per_head;
-    tok0 = sg.tok_in_run;
-    return true;
+    cx = &x;
+    return x.it < a.n_items && !*abort_flag;
   };
   auto item_done = [&]() {
-    gs += static_cast<uint32_t>(c.steps);
+    gs += static_cast<uint32_t>(cx->steps);
     gi += 1;
   };
 
-  if (wg == 3) {
+  if (wg == 4) {
     setmaxnreg_dec<kRegsAux>();
-    if (warp == 12) {
+    if (warp == 16) {
       // ================================================================ TMA producer
       while (next_item()) {
-      if (lane == 0) {
-        const CUtensorMap* mq = &maps.q[sg.run];
-        const CUtensorMap* mdo = &maps.d_o[sg.run];
-        mbar_expect_tx(&s.bar_kv, 2 * kTileBytes);
-        tma_load_3d(s.k[0], &maps.k[sg.run], &s.bar_kv, 0, c.g, tok0 + c.n * kBN);
-        tma_load_3d(s.k[1], &maps.k[sg.run], &s.bar_kv, 64, c.g, tok0 + c.n * kBN);
-        tma_load_3d(s.v[0], &maps.v[sg.run], &s.bar_kv, 0, c.g, tok0 + c.n * kBN);
-        tma_load_3d(s.v[1], &maps.v[sg.run], &s.bar_kv, 64, c.g, tok0 + c.n * kBN);
+        if (lane == 0) {
+          const ItemCtx c = *cx;
+          const CUtensorMap* mq = &maps.q[c.run];
+          const CUtensorMap* mdo = &maps.d_o[c.run];
+          mbar_expect_tx(&s.bar_kv, 2 * kTileBytes);
+          tma_load_3d(s.k[0], &maps.k[c.run], &s.bar_kv, 0, c.g, c.tok0 + c.n * kBN);
+          tma_load_3d(s.k[1], &maps.k[c.run], &s.bar_kv, 64, c.g, c.tok0 + c.n * kBN);
+          tma_load_3d(s.v[0], &maps.v[c.run], &s.bar_kv, 0, c.g, c.tok0 + c.n * kBN);
+          tma_load_3d(s.v[1], &maps.v[c.run], &s.bar_kv, 64, c.g, c.tok0 + c.n * kBN);
+          StepWalk w;
+          w.reset();
+#pragma unroll 1
+          for (int vt = 0; vt < c.steps; ++vt) {
+            const uint32_t cs = gs + vt, st = cs & 1;
+            if (*abort_flag) break;
+            if (!mbar_wait(&s.bar_q_empty[st][0], ((cs >> 1) & 1) ^ 1) ||
+                !mbar_wait(&s.bar_q_empty[st][1], ((cs >> 1) & 1) ^ 1)) {
+              report_timeout(a.status, c.it, kWhereBwdQEmpty, vt);
+              *abort_flag = 1;
+              break;
+            }
+            NSP_TRACE_STAMP(14);
+            int h, m, mode;
+            w.get(c, h, m, mode);
+            w.next(c);
+            mbar_expect_tx(&s.bar_q_full[st], 2 * kTileBytes);
+            tma_load_3d(s.q[st][0], mq, &s.bar_q_full[st], 0, h, c.tok0 + m * kBM);
+            tma_load_3d(s.q[st][1], mq, &s.bar_q_full[st], 64, h, c.tok0 + m * kBM);
+            tma_load_3d(s.d_o[st][0], mdo, &s.bar_q_full[st], 0, h, c.tok0 + m * kBM);
+            tma_load_3d(s.d_o[st][1], mdo, &s.bar_q_full[st], 64, h, c.tok0 + m * kBM);
+          }
+        }
+        item_done();
+      }
+    } else if (warp == 17 || warp == 19) {
+      // ================================================================ MMA issuers
+      // Two issuing threads share the step: thread A (warp 17) owns R0 and dV: dV(t), S^T(t+1); thread B
+      // (warp 19) owns R1 and dK: dK(t), dQ^T(t), dP^T(t+1). Each has its own chain of waits, so the bookkeeping
+      // of one (a single thread on a busy sub-partition runs at a dozen clocks per instruction) hides behind
+      // the MMAs of the other. Each thread signals completion on barriers of its own (a tcgen05.commit covers
+      // only the issuing thread's MMAs); whoever depends on both waits for both.
+      const bool is_a = warp == 17;
+      while (next_item()) {
+        if (lane == 0) {
+          constexpr uint32_t idesc_kk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
+          constexpr uint32_t idesc_kn = make_idesc_bf16(128, 128, 0, 1);  // A K-major (or TMEM), B MN-major
+          constexpr uint32_t idesc_nn = make_idesc_bf16(128, 128, 1, 1);  // A MN-major, B MN-major
+          // Descriptors are {low word, high word}; an operand advances inside its tile by adding the byte offset
+          // (in 16-byte units) to the low word (the 14-bit address field cannot overflow: every tile sits below
+          // 256 KB). K-major operands step 32 bytes per 16 contraction elements inside a 64-column half;
+          // MN-major operands step 16 rows = 2048 bytes. The high word is the same for both kinds.
+          const uint32_t hi = static_cast<uint32_t>(make_smem_desc_sw128(0, 16, 1024) >> 32);
+          constexpr uint32_t lbo_km = (16u >> 4) << 16, lbo_mn = (kHalfTileBytes >> 4) << 16;
+          constexpr uint32_t kStageStep = kTileBytes >> 4;  // descriptor distance between the two stages
+          const int steps = cx->steps, item_it = cx->it;
+          int where = 0;
+          bool okm = mbar_wait(&s.bar_kv, gi & 1);
+          if (!okm) where = kWhereBwdLoadKV;
+          if (is_a) {
+            const uint32_t k_km = (smem_u32(s.k[0]) >> 4) | lbo_km;
+            const uint32_t q0_lo = smem_u32(s.q[0][0]) >> 4, do0_lo = smem_u32(s.d_o[0][0]) >> 4;
+            // S^T of step vt -> R0 (A = K, B = Q of the step's stage, both K-major)
+            auto issue_s = [&](int vt) -> bool {
+              const uint32_t cs = gs + vt, st = cs & 1;
+              if (!mbar_wait(&s.bar_q_full[st], (cs >> 1) & 1)) { where = kWhereBwdLoadQ; return false; }
+              tc_fence_after_sync();
+              const uint32_t b_lo = (q0_lo + st * kStageStep) | lbo_km;
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
+                umma_ss_lh(tR0, k_km + off, hi, b_lo + off, hi, idesc_kk, kk > 0);
+              }
+              umma_commit(&s.bar_s_full);
+              return true;
+            };
+            okm = okm && issue_s(0);
+#pragma unroll 1
+            for (int vt = 0; okm && vt < steps; ++vt) {
+              const uint32_t cs = gs + vt, st = cs & 1;
+              if (*abort_flag) break;
+              if (!mbar_wait(&s.bar_p_ready, cs & 1)) { okm = false; where = kWhereBwdPReady; break; }
+              NSP_TRACE_STAMP(0);
+              tc_fence_after_sync();
+              const uint32_t acc = vt > 0;
+              const uint32_t do_mn = (do0_lo + st * kStageStep) | lbo_mn;
+              // dV += P^T dO; packed P^T columns of K-step kk (16 query columns) sit at R0 + (kk/2)*32 + (kk%2)*8
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk)
+                umma_ts_lh(tDV, tR0 + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + kk * 128, hi, idesc_kn, acc | (kk > 0));
+              umma_commit(&s.bar_a_done);          // S^T and dV of the step
+              umma_commit(&s.bar_q_empty[st][0]);
+              NSP_TRACE_STAMP(15);
+#ifdef NSP_TRACE
+              if (vt + 1 < steps) mbar_wait(&s.bar_q_full[(cs + 1) & 1], ((cs + 1) >> 1) & 1);
+              NSP_TRACE_STAMP(13);
+#endif
+              if (vt + 1 < steps && !issue_s(vt + 1)) { okm = false; break; }
+              NSP_TRACE_STAMP(1);
+            }
+          } else {
+            const uint32_t v_km = (smem_u32(s.v[0]) >> 4) | lbo_km, k_mn = (smem_u32(s.k[0]) >> 4) | lbo_mn;
+            const uint32_t ds_km = (smem_u32(s.ds[0]) >> 4) | lbo_km, ds_mn = (smem_u32(s.ds[0]) >> 4) | lbo_mn;
+            const uint32_t q0_lo = smem_u32(s.q[0][0]) >> 4, do0_lo = smem_u32(s.d_o[0][0]) >> 4;
+            // dP^T of step vt -> R1, once the dQ warps have drained dQ^T of the previous step from it
+            auto issue_dp = [&](int vt) -> bool {
+              const uint32_t cs = gs + vt, st = cs & 1;
+              if (!mbar_wait(&s.bar_q_full[st], (cs >> 1) & 1)) { where = kWhereBwdLoadQ; return false; }
+              if (!mbar_wait(&s.bar_dq_empty, (cs & 1) ^ 1)) { where = kWhereBwdDqEmpty; return false; }
+              tc_fence_after_sync();
+              const uint32_t b_lo = (do0_lo + st * kStageStep) | lbo_km;
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
+                umma_ss_lh(tR1, v_km + off, hi, b_lo + off, hi, idesc_kk, kk > 0);
+              }
+              umma_commit(&s.bar_dp_full);
+              return true;
+            };
+            okm = okm && issue_dp(0);
+#pragma unroll 1
+            for (int vt = 0; okm && vt < steps; ++vt) {
+              const uint32_t cs = gs + vt, st = cs & 1;
+              if (*abort_flag) break;
+              if (!mbar_wait(&s.bar_ds_ready, cs & 1)) { okm = false; where = kWhereBwdDsReady; break; }
+              NSP_TRACE_STAMP(2);
+              tc_fence_after_sync();
+              const uint32_t acc = vt > 0;
+              const uint32_t q_mn = (q0_lo + st * kStageStep) | lbo_mn;
+              // dK += dS^T Q
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
+                umma_ss_lh(tDK, ds_km + off, hi, q_mn + kk * 128, hi, idesc_kn, acc | (kk > 0));
+              }
+              // dQ^T = K^T dS^T -> R1 (dP^T of this step has been consumed: ds_ready)
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk) umma_ss_lh(tR1, k_mn + kk * 128, hi, ds_mn + kk * 128, hi, idesc_nn, kk > 0);
+              umma_commit(&s.bar_dq_full);         // dP^T, dK and dQ^T of the step
+              umma_commit(&s.bar_q_empty[st][1]);
+              NSP_TRACE_STAMP(3);
+              if (vt + 1 < steps && !issue_dp(vt + 1)) { okm = false; break; }
+              NSP_TRACE_STAMP(4);
+            }
+          }
+          if (!okm) {
+            report_timeout(a.status, item_it, where, is_a ? 0 : 1);
+            *abort_flag = 1;
+          }
+        }
+        item_done();
+      }
+    } else if (warp == 18) {
+      // ================================================================ LSE / delta loader
+      while (next_item()) {
+        const ItemCtx c = *cx;
+        StepWalk w;
+        w.reset();
+#pragma unroll 1
         for (int vt = 0; vt < c.steps; ++vt) {
           const uint32_t cs = gs + vt, st = cs & 1;
           if (*abort_flag) break;
-          if (!mbar_wait(&s.bar_q_empty[st], ((cs >> 1) & 1) ^ 1)) {
-            report_timeout(a.status, it, kWhereBwdQEmpty, vt);
-            *abort_flag = 1;
+          bool okl = mbar_wait(&s.bar_ld_empty[st], ((cs >> 1) & 1) ^ 1);
+          okl = __all_sync(0xffffffffu, okl);
+          if (!okl) {
+            if (lane == 0) {
+              report_timeout(a.status, c.it, kWhereBwdLdEmpty, vt);
+              *abort_flag = 1;
+            }
             break;
           }
           int h, m, mode;
-          decode_step(c, vt, h, m, mode);
-          mbar_expect_tx(&s.bar_q_full[st], 2 * kTileBytes);
-          tma_load_3d(s.q[st][0], mq, &s.bar_q_full[st], 0, h, tok0 + m * kBM);
-          tma_load_3d(s.q[st][1], mq, &s.bar_q_full[st], 64, h, tok0 + m * kBM);
-          tma_load_3d(s.d_o[st][0], mdo, &s.bar_q_full[st], 0, h, tok0 + m * kBM);
-          tma_load_3d(s.d_o[st][1], mdo, &s.bar_q_full[st], 64, h, tok0 + m * kBM);
-        }
-      }
-      item_done();
-      }
-    } else if (warp == 13) {
-      // ================================================================ MMA issuer
-      while (next_item()) {
-      if (lane == 0) {
-        constexpr uint32_t idesc_kk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
-        constexpr uint32_t idesc_kn = make_idesc_bf16(128, 128, 0, 1);  // A K-major (or TMEM), B MN-major
-        constexpr uint32_t idesc_nn = make_idesc_bf16(128, 128, 1, 1);  // A MN-major, B MN-major
-        const uint32_t k_addr = smem_u32(s.k[0]), v_addr = smem_u32(s.v[0]), ds_addr = smem_u32(s.ds[0]);
-        int where = 0;
-        bool okm = mbar_wait(&s.bar_kv, gi & 1);
-        if (!okm) where = kWhereBwdLoadKV;
-        for (int vt = 0; okm && vt < c.steps; ++vt) {
-          const uint32_t cs = gs + vt, st = cs & 1;
-          if (*abort_flag) break;
-          const uint32_t q_addr = smem_u32(s.q[st][0]), do_addr = smem_u32(s.d_o[st][0]);
-          if (!mbar_wait(&s.bar_q_full[st], (cs >> 1) & 1)) { okm = false; where = kWhereBwdLoadQ; break; }
-          tc_fence_after_sync();
+          w.get(c, h, m, mode);
+          w.next(c);
+          const int64_t base = c.lse_off + static_cast<int64_t>(h) * c.len;
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk >> 2) * kHalfTileBytes + (kk & 3) * 32;
-            umma_ss(tR0, make_smem_desc_sw128(k_addr + off, 16, 1024), make_smem_desc_sw128(q_addr + off, 16, 1024),
-                    idesc_kk, kk > 0);
+          for (int x = 0; x < 4; ++x) {
+            const int col = lane + 32 * x, qi = m * kBM + col;
+            const bool valid = qi < c.len;
+            s.lse[st][col] = valid ? a.lse[base + qi] * kLog2e : INFINITY;
+            s.delta[st][col] = valid ? a.delta[base + qi] : 0.f;
           }
-          umma_commit(&s.bar_s_full);
-          // R1 still holds dQ of the previous step until the dQ warps have drained it
-          if (!mbar_wait(&s.bar_dq_empty, (cs & 1) ^ 1)) { okm = false; where = kWhereBwdDqEmpty; break; }
-          tc_fence_after_sync();
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk >> 2) * kHalfTileBytes + (kk & 3) * 32;
-            umma_ss(tR1, make_smem_desc_sw128(v_addr + off, 16, 1024), make_smem_desc_sw128(do_addr + off, 16, 1024),
-                    idesc_kk, kk > 0);
-          }
-          umma_commit(&s.bar_dp_full);
-          if (!mbar_wait(&s.bar_p_ready, cs & 1)) { okm = false; where = kWhereBwdPReady; break; }
-          tc_fence_after_sync();
-          const uint32_t acc = vt > 0;
-          // packed P^T columns of K-step kk (16 query columns) sit at R0 + (kk/2)*32 + (kk%2)*8
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            umma_ts(tDV, tR0 + (kk >> 1) * 32 + (kk & 1) * 8,
-                    make_smem_desc_sw128(do_addr + kk * 2048, kHalfTileBytes, 1024), idesc_kn, acc | (kk > 0));
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk >> 2) * kHalfTileBytes + (kk & 3) * 32;
-            umma_ss(tDK, make_smem_desc_sw128(ds_addr + off, 16, 1024),
-                    make_smem_desc_sw128(q_addr + kk * 2048, kHalfTileBytes, 1024), idesc_kn, acc | (kk > 0));
-          }
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            umma_ss(tR1, make_smem_desc_sw128(ds_addr + kk * 2048, kHalfTileBytes, 1024),
-                    make_smem_desc_sw128(k_addr + kk * 2048, kHalfTileBytes, 1024), idesc_nn, kk > 0);
-          umma_commit(&s.bar_dq_full);  // the dQ warps release the Q/dO stage after using it as staging
+          mbar_arrive(&s.bar_ld_full[st]);
         }
-        if (!okm) {
-          report_timeout(a.status, it, where, 0);
-          *abort_flag = 1;
-        }
+        item_done();
       }
-      item_done();
-      }
-    } else if (warp == 14) {
-      // ================================================================ LSE / delta loader
-      while (next_item()) {
-      for (int vt = 0; vt < c.steps; ++vt) {
-        const uint32_t cs = gs + vt, st = cs & 1;
-        if (*abort_flag) break;
-        bool okl = mbar_wait(&s.bar_ld_empty[st], ((cs >> 1) & 1) ^ 1);
-        okl = __all_sync(0xffffffffu, okl);
-        if (!okl) {
-          if (lane == 0) {
-            report_timeout(a.status, it, kWhereBwdLdEmpty, vt);
-            *abort_flag = 1;
-          }
-          break;
-        }
-        int h, m, mode;
-        decode_step(c, vt, h, m, mode);
-        const int64_t base = sg.lse_off + static_cast<int64_t>(h) * sg.len;
-#pragma unroll
-        for (int x = 0; x < 4; ++x) {
-          const int col = lane * 4 + x, qi = m * kBM + col;
-          const bool valid = qi < sg.len;
-          s.lse[st][col] = valid ? a.lse[base + qi] * kLog2e : INFINITY;
-          s.delta[st][col] = valid ? a.delta[base + qi] : 0.f;
-        }
-        mbar_arrive(&s.bar_ld_full[st]);
-      }
-      item_done();
-      }
-    } else {
-      while (next_item()) item_done();  // spare warp: only keeps the CTA-wide barrier count
     }
-  } else if (wg == 2) {
-    {
-      // ================================================================ dQ: R1 -> global fp32 accumulator
-      setmaxnreg_dec<kRegsReduce>();
-      const int quad = warp & 3;
-      const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
-      while (next_item()) {
+  } else if (wg >= 2) {
+    // ================================================================ dQ^T: R1 -> global fp32 accumulator
+    setmaxnreg_dec<kRegsReduce>();
+    const int quad = warp & 3, colhalf = wg - 2;  // this warp drains query columns [64*colhalf, 64*colhalf + 64)
+    const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
+    const int d = quad * 32 + lane;  // head-dimension index = TMEM lane
+    while (next_item()) {
+      const ItemCtx c = *cx;
+      const int64_t q_stride = static_cast<int64_t>(c.hq) * kHeadDim;  // floats between consecutive query rows
+      StepWalk w;
+      w.reset();
+#pragma unroll 1
       for (int vt = 0; vt < c.steps; ++vt) {
         const uint32_t cs = gs + vt;
         if (*abort_flag) break;
@@ -313,246 +429,282 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         okr = __all_sync(0xffffffffu, okr);
         if (!okr) {
           if (lane == 0) {
-            report_timeout(a.status, it, kWhereBwdDqFull, vt);
+            report_timeout(a.status, c.it, kWhereBwdDqFull, vt);
             *abort_flag = 1;
           }
           break;
         }
         tc_fence_after_sync();
+        if (warp == 8 && lane == 0) NSP_TRACE_STAMP(10);
         int h, m, mode;
-        decode_step(c, vt, h, m, mode);
-        // The Q/dO stage of this step is dead once its MMAs are done (bar_dq_full): use it as a 64 KB staging
-        // buffer for the fp32 dQ tile, four [128 rows x 32 columns] boxes in the 128-byte-swizzled layout of
-        // the accumulator's tensor map, and let TMA add the boxes into global memory. Rows past the segment
-        // end hold exact zeros (their dS columns are zero), rows past the run are clipped by TMA.
-        const uint32_t st = cs & 1;
-        const int row = quad * 32 + lane;
-#pragma unroll
-        for (int pair = 0; pair < 2; ++pair) {
+        w.get(c, h, m, mode);
+        w.next(c);
+        // Register e of a column chunk is dQ^T[d][query]: the 32 lanes of a warp add 32 consecutive floats of
+        // one accumulator row (128 bytes, one request). Eight warps issue them: one SM sustains about 25 bytes
+        // per clock of reductions, and four warps reach only half of that. Rows past the segment end are
+        // skipped (their dS^T columns are zero, and they may lie outside the buffer).
+        const int n_valid = min(kBM, c.len - m * kBM) - colhalf * 64;
+        float* p0 = a.dq_acc + c.q_off + ((static_cast<int64_t>(m) * kBM + colhalf * 64) * c.hq + h) * kHeadDim + d;
+        const bool do_red = (a.debug_flags & 4) == 0;
+        if (n_valid >= 64) {  // interior tile: no row checks
           uint32_t v0[32], v1[32];
-          tmem_ld32(tR1 + lane_off + pair * 64, v0);
-          tmem_ld32(tR1 + lane_off + pair * 64 + 32, v1);
+          tmem_ld32(tR1 + lane_off + colhalf * 64, v0);
+          tmem_ld32(tR1 + lane_off + colhalf * 64 + 32, v1);
           tmem_wait_ld();
-          if (pair == 1) {  // R1 is drained: the next dP^T may overwrite it
-            tc_fence_before_sync();
-            mbar_arrive(&s.bar_dq_empty);
-          }
-          uint8_t* box0 = (pair == 0 ? s.q[st][0] : s.d_o[st][0]) + row * 128;
-          uint8_t* box1 = (pair == 0 ? s.q[st][1] : s.d_o[st][1]) + row * 128;
+          tc_fence_before_sync();
+          mbar_arrive(&s.bar_dq_empty);  // R1 is drained: the next dP^T may overwrite it
+          if (warp == 8 && lane == 0) NSP_TRACE_STAMP(11);
+          if (do_red) {
+            float* p1 = p0 + 32 * q_stride;
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch) {
-            const int chunk = (ch ^ (row & 7)) * 16;
-            *reinterpret_cast<uint4*>(box0 + chunk) = make_uint4(v0[4 * ch], v0[4 * ch + 1], v0[4 * ch + 2], v0[4 * ch + 3]);
-            *reinterpret_cast<uint4*>(box1 + chunk) = make_uint4(v1[4 * ch], v1[4 * ch + 1], v1[4 * ch + 2], v1[4 * ch + 3]);
+            for (int e = 0; e < 32; ++e) {
+              red_add_f32(p0, __uint_as_float(v0[e]));
+              red_add_f32(p1, __uint_as_float(v1[e]));
+              p0 += q_stride;
+              p1 += q_stride;
+#ifdef NSP_RED_PACE_NS
+              if ((e & NSP_RED_PACE_MASK) == NSP_RED_PACE_MASK) __nanosleep(NSP_RED_PACE_NS);
+#endif
+            }
+          }
+        } else {  // ragged tail: 16 columns at a time, each row checked
+#pragma unroll 1
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t v[16];
+            tmem_ld16(tR1 + lane_off + colhalf * 64 + ch * 16, v);
+            tmem_wait_ld();
+            if (ch == 3) {
+              tc_fence_before_sync();
+              mbar_arrive(&s.bar_dq_empty);
+            }
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              if (do_red && ch * 16 + e < n_valid) red_add_f32(p0, __uint_as_float(v[e]));
+              p0 += q_stride;
+            }
           }
         }
-        fence_proxy_async_smem();
-        mbar_arrive(&s.bar_staged);
-        if (warp == 8 && lane == 0) {
-          if (!mbar_wait(&s.bar_staged, cs & 1)) {
-            report_timeout(a.status, it, kWhereBwdStaged, vt);
-            *abort_flag = 1;
-          } else if ((a.debug_flags & 4) == 0) {
-            const CUtensorMap* mdq = &maps.dq[sg.run];
-            tma_reduce_add_3d(mdq, s.q[st][0], 0, h, tok0 + m * kBM);
-            tma_reduce_add_3d(mdq, s.q[st][1], 32, h, tok0 + m * kBM);
-            tma_reduce_add_3d(mdq, s.d_o[st][0], 64, h, tok0 + m * kBM);
-            tma_reduce_add_3d(mdq, s.d_o[st][1], 96, h, tok0 + m * kBM);
-            bulk_commit_group();
-            bulk_wait_read_all();
-          }
-          mbar_arrive(&s.bar_q_empty[st]);  // stage free: the producer may refill it
-        }
+        if (warp == 8 && lane == 0) NSP_TRACE_STAMP(12);
       }
-      if (warp == 8 && lane == 0) bulk_wait_all();  // all reductions of this item performed
       item_done();
-      }
     }
   } else {
-    {
-      // ================================================================ softmax / dS (key row r, 64 query columns)
-      setmaxnreg_inc<kRegsSoftmax>();
-      const int quad = warp & 3, half = wg;
-      const int r = quad * 32 + lane;
-      const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
-      uint32_t nd = 0;  // completed phases of bar_delta[half]
-      while (next_item()) {
+    // ================================================================ softmax / dS (key row r, 64 query columns)
+    setmaxnreg_inc<kRegsSoftmax>();
+    const int quad = warp & 3, half = wg;
+    const int r = quad * 32 + lane;
+    const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
+    const uint32_t tS = tR0 + lane_off + half * 64, tDP = tR1 + lane_off + half * 64;
+    uint8_t* const ds_row = s.ds[half] + r * 128;  // this thread's 128-byte row of the swizzled dS^T half tile
+    uint32_t nd = 0;                               // completed phases of bar_delta[half]
+    while (next_item()) {
+      const ItemCtx c = *cx;
       bool oks = true;
       int where = 0;
+      StepWalk w;
+      w.reset();
+#pragma unroll 1
       for (int vt = 0; vt < c.steps; ++vt) {
         const uint32_t cs = gs + vt, st = cs & 1;
         if (*abort_flag) { oks = false; where = 0; break; }
         int h, m, mode;
-        decode_step(c, vt, h, m, mode);
+        w.get(c, h, m, mode);
+        w.next(c);
         oks = mbar_wait(&s.bar_ld_full[st], (cs >> 1) & 1) && mbar_wait(&s.bar_s_full, cs & 1);
         oks = __all_sync(0xffffffffu, oks);
         if (!oks) { where = kWhereBwdS; break; }
         tc_fence_after_sync();
-        const bool diag = (m == c.n);
-        const float* lse_s = s.lse[st];
-        float* delta_s = s.delta[st];
-        bool have_dp = false;
-        if (mode & 1) {
-          // delta_i = sum_j P_ij dP_ij over the keys of this tile (all keys of rows 0..127), fp32
+        if (tid == 0) NSP_TRACE_STAMP(5);
+        const float* lse_s = s.lse[st] + half * 64;
+        float* delta_s = s.delta[st] + half * 64;
+        if (mode == 0 && m != c.n) {
+          // ---- common step (interior tile). Phase 1: P^T = exp2(S^T * c - LSE) for this thread's 64 query
+          // columns, bf16 pairs over the S^T columns already read. The dV product needs only P^T, so it is
+          // released to the MMA thread before dS^T is formed.
+          uint32_t pv[2][32];
+          tmem_ld32(tS, pv[0]);
+          tmem_ld32(tS + 32, pv[1]);
+          tmem_wait_ld();
+          if (tid == 0) NSP_TRACE_STAMP(6);
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            uint32_t pp[16];
+#pragma unroll
+            for (int x = 0; x < 32; x += 4) {
+              const float4 l4 = *reinterpret_cast<const float4*>(lse_s + cc * 32 + x);
+              const float p0 = ex2f(fmaf(__uint_as_float(pv[cc][x + 0]), a.scale_log2, -l4.x));
+              const float p1 = ex2f(fmaf(__uint_as_float(pv[cc][x + 1]), a.scale_log2, -l4.y));
+              const float p2 = ex2f(fmaf(__uint_as_float(pv[cc][x + 2]), a.scale_log2, -l4.z));
+              const float p3 = ex2f(fmaf(__uint_as_float(pv[cc][x + 3]), a.scale_log2, -l4.w));
+              pv[cc][x + 0] = __float_as_uint(p0);
+              pv[cc][x + 1] = __float_as_uint(p1);
+              pv[cc][x + 2] = __float_as_uint(p2);
+              pv[cc][x + 3] = __float_as_uint(p3);
+              pp[(x >> 1) + 0] = pack_bf16x2(p0, p1);
+              pp[(x >> 1) + 1] = pack_bf16x2(p2, p3);
+            }
+            tmem_st16(tS + cc * 32, pp);  // query columns [32cc, 32cc + 32) -> packed columns [32cc, 32cc + 16)
+          }
+          tmem_wait_st();
+          tc_fence_before_sync();
+          mbar_arrive(&s.bar_p_ready);
+          if (tid == 0) NSP_TRACE_STAMP(7);
+          if (lane == 0) NSP_TRACE_STAMP(16 + warp);
+          // Phase 2: dS^T = P^T o (dP^T - delta) -> swizzled shared memory. The dS buffer is free: dP^T of this
+          // step was issued behind dK / dQ^T of the previous step, so bar_dp_full implies they have completed.
           oks = mbar_wait(&s.bar_dp_full, cs & 1);
           oks = __all_sync(0xffffffffu, oks);
           if (!oks) { where = kWhereBwdDp; break; }
           tc_fence_after_sync();
-          have_dp = true;
-          float* part = reinterpret_cast<float*>(s.ds[half]);  // [4 quadrants][64 columns]; free until dS is written
+          if (tid == 0) NSP_TRACE_STAMP(8);
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
-            const int col0 = half * 64 + cc * 32;
-            uint32_t sv[32], dpv[32];
-            tmem_ld32(tR0 + lane_off + col0, sv);
-            tmem_ld32(tR1 + lane_off + col0, dpv);
+            uint32_t dpv[32], dsp[16];
+            tmem_ld32(tDP + cc * 32, dpv);
             tmem_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 32; ++x) {
-              float p = ex2f(fmaf(__uint_as_float(sv[x]), a.scale_log2, -lse_s[col0 + x]));
-              if (col0 + x < r) p = 0.f;
-              float v = p * __uint_as_float(dpv[x]);
+            for (int x = 0; x < 32; x += 4) {
+              const float4 d4 = *reinterpret_cast<const float4*>(delta_s + cc * 32 + x);
+              const float d0 = __uint_as_float(pv[cc][x + 0]) * (__uint_as_float(dpv[x + 0]) - d4.x);
+              const float d1 = __uint_as_float(pv[cc][x + 1]) * (__uint_as_float(dpv[x + 1]) - d4.y);
+              const float d2 = __uint_as_float(pv[cc][x + 2]) * (__uint_as_float(dpv[x + 2]) - d4.z);
+              const float d3 = __uint_as_float(pv[cc][x + 3]) * (__uint_as_float(dpv[x + 3]) - d4.w);
+              dsp[(x >> 1) + 0] = pack_bf16x2(d0, d1);
+              dsp[(x >> 1) + 1] = pack_bf16x2(d2, d3);
+            }
+            // dS^T row r, columns 32cc .. 32cc+31 of the half -> four 16-byte chunks of the swizzled row
 #pragma unroll
-              for (int sft = 16; sft > 0; sft >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sft);
-              if (lane == 0) part[quad * 64 + cc * 32 + x] = v;
+            for (int ch = 0; ch < 4; ++ch) {
+              const int chunk = (cc * 4 + ch) ^ (r & 7);
+              *reinterpret_cast<uint4*>(ds_row + chunk * 16) =
+                  make_uint4(dsp[ch * 4 + 0], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
             }
           }
-          mbar_arrive(&s.bar_delta[half]);
-          oks = mbar_wait(&s.bar_delta[half], nd & 1);
-          ++nd;
+        } else {
+          // ---- rare step (diagonal tile and/or one of the two first-tile passes): compact rolled loops, 16 query
+          // columns at a time; P^T and dS^T are handed over together at the end.
+          oks = mbar_wait(&s.bar_dp_full, cs & 1);
           oks = __all_sync(0xffffffffu, oks);
-          if (!oks) { where = kWhereBwdDelta; break; }
-          if (r < 64) delta_s[half * 64 + r] = (part[r] + part[64 + r]) + (part[128 + r] + part[192 + r]);
-          mbar_arrive(&s.bar_delta[half]);
-          oks = mbar_wait(&s.bar_delta[half], nd & 1);
-          ++nd;
-          oks = __all_sync(0xffffffffu, oks);
-          if (!oks) { where = kWhereBwdDelta; break; }
-        }
+          if (!oks) { where = kWhereBwdDp; break; }
+          tc_fence_after_sync();
+          const bool diag = (m == c.n);
+          if (mode & 1) {
+            // delta_i = sum_j P_ij dP_ij over the keys of this tile (all keys of rows 0..127), fp32
+            float* part = reinterpret_cast<float*>(s.ds[half]);  // [4 quadrants][64 columns]; free until dS is written
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
+              uint32_t sv[16], dpv[16];
+              tmem_ld16(tS + ch * 16, sv);
+              tmem_ld16(tDP + ch * 16, dpv);
+              tmem_wait_ld();
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {  // 32 query columns at a time
-          const int col0 = half * 64 + cc * 32;
-          uint32_t sv[32];
-          tmem_ld32(tR0 + lane_off + col0, sv);
-          tmem_wait_ld();
+              for (int x = 0; x < 16; ++x) {
+                float p = ex2f(fmaf(__uint_as_float(sv[x]), a.scale_log2, -lse_s[ch * 16 + x]));
+                if (half * 64 + ch * 16 + x < r) p = 0.f;
+                float v = p * __uint_as_float(dpv[x]);
 #pragma unroll
-          for (int x = 0; x < 32; x += 4) {
-            const float4 l4 = *reinterpret_cast<const float4*>(lse_s + col0 + x);
-            float p0 = ex2f(fmaf(__uint_as_float(sv[x + 0]), a.scale_log2, -l4.x));
-            float p1 = ex2f(fmaf(__uint_as_float(sv[x + 1]), a.scale_log2, -l4.y));
-            float p2 = ex2f(fmaf(__uint_as_float(sv[x + 2]), a.scale_log2, -l4.z));
-            float p3 = ex2f(fmaf(__uint_as_float(sv[x + 3]), a.scale_log2, -l4.w));
-            if (diag) {  // query index must be >= key index
-              if (col0 + x + 0 < r) p0 = 0.f;
-              if (col0 + x + 1 < r) p1 = 0.f;
-              if (col0 + x + 2 < r) p2 = 0.f;
-              if (col0 + x + 3 < r) p3 = 0.f;
+                for (int sft = 16; sft > 0; sft >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sft);
+                if (lane == 0) part[quad * 64 + ch * 16 + x] = v;
+              }
             }
-            sv[x + 0] = __float_as_uint(p0);
-            sv[x + 1] = __float_as_uint(p1);
-            sv[x + 2] = __float_as_uint(p2);
-            sv[x + 3] = __float_as_uint(p3);
-          }
-          if (!have_dp) {
-            oks = mbar_wait(&s.bar_dp_full, cs & 1);
+            mbar_arrive(&s.bar_delta[half]);
+            oks = mbar_wait(&s.bar_delta[half], nd & 1);
+            ++nd;
             oks = __all_sync(0xffffffffu, oks);
-            if (!oks) { where = kWhereBwdDp; break; }
-            tc_fence_after_sync();
-            have_dp = true;
+            if (!oks) { where = kWhereBwdDelta; break; }
+            if (r < 64) delta_s[r] = (part[r] + part[64 + r]) + (part[128 + r] + part[192 + r]);
+            mbar_arrive(&s.bar_delta[half]);
+            oks = mbar_wait(&s.bar_delta[half], nd & 1);
+            ++nd;
+            oks = __all_sync(0xffffffffu, oks);
+            if (!oks) { where = kWhereBwdDelta; break; }
           }
-          uint32_t dpv[32];
-          tmem_ld32(tR1 + lane_off + col0, dpv);
-          tmem_wait_ld();
-          uint32_t pp[16], dsp[16];
-#pragma unroll
-          for (int x = 0; x < 32; x += 4) {
-            const float4 d4 = *reinterpret_cast<const float4*>(delta_s + col0 + x);
-            float p0 = __uint_as_float(sv[x + 0]), p1 = __uint_as_float(sv[x + 1]);
-            float p2 = __uint_as_float(sv[x + 2]), p3 = __uint_as_float(sv[x + 3]);
-            float d0 = p0 * (__uint_as_float(dpv[x + 0]) - d4.x), d1 = p1 * (__uint_as_float(dpv[x + 1]) - d4.y);
-            float d2 = p2 * (__uint_as_float(dpv[x + 2]) - d4.z), d3 = p3 * (__uint_as_float(dpv[x + 3]) - d4.w);
-            uint32_t pa = pack_bf16x2(p0, p1), pb = pack_bf16x2(p2, p3);
-            uint32_t da = pack_bf16x2(d0, d1), db = pack_bf16x2(d2, d3);
-            if (mode & 2) {  // residual pass: what the bf16 value left behind
-              pa = pack_bf16x2(p0 - __uint_as_float(pa << 16), p1 - __uint_as_float(pa & 0xffff0000u));
-              pb = pack_bf16x2(p2 - __uint_as_float(pb << 16), p3 - __uint_as_float(pb & 0xffff0000u));
-              da = pack_bf16x2(d0 - __uint_as_float(da << 16), d1 - __uint_as_float(da & 0xffff0000u));
-              db = pack_bf16x2(d2 - __uint_as_float(db << 16), d3 - __uint_as_float(db & 0xffff0000u));
-            }
-            pp[(x >> 1) + 0] = pa;
-            pp[(x >> 1) + 1] = pb;
-            dsp[(x >> 1) + 0] = da;
-            dsp[(x >> 1) + 1] = db;
-          }
-          // P^T (bf16 pairs) goes over S^T columns this warp has already read: query columns
-          // [col0, col0+32) -> packed columns [col0, col0+16)
-          tmem_st16(tR0 + lane_off + col0, pp);
-          // dS^T row r, columns col0 .. col0+31 -> four 16-byte chunks of the swizzled half tile
-          uint8_t* base = s.ds[half] + r * 128;
-#pragma unroll
+#pragma unroll 1
           for (int ch = 0; ch < 4; ++ch) {
-            const int chunk = (cc * 4 + ch) ^ (r & 7);
-            *reinterpret_cast<uint4*>(base + chunk * 16) =
-                make_uint4(dsp[ch * 4 + 0], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
+            uint32_t sv[16], dpv[16], pp[8], dsp[8];
+            tmem_ld16(tS + ch * 16, sv);
+            tmem_ld16(tDP + ch * 16, dpv);
+            tmem_wait_ld();
+#pragma unroll
+            for (int x = 0; x < 16; x += 2) {
+              float p0 = ex2f(fmaf(__uint_as_float(sv[x + 0]), a.scale_log2, -lse_s[ch * 16 + x + 0]));
+              float p1 = ex2f(fmaf(__uint_as_float(sv[x + 1]), a.scale_log2, -lse_s[ch * 16 + x + 1]));
+              if (diag) {  // query index must be >= key index
+                if (half * 64 + ch * 16 + x + 0 < r) p0 = 0.f;
+                if (half * 64 + ch * 16 + x + 1 < r) p1 = 0.f;
+              }
+              const float d0 = p0 * (__uint_as_float(dpv[x + 0]) - delta_s[ch * 16 + x + 0]);
+              const float d1 = p1 * (__uint_as_float(dpv[x + 1]) - delta_s[ch * 16 + x + 1]);
+              uint32_t pa = pack_bf16x2(p0, p1), da = pack_bf16x2(d0, d1);
+              if (mode & 2) {  // residual pass: what the bf16 value left behind
+                pa = pack_bf16x2(p0 - __uint_as_float(pa << 16), p1 - __uint_as_float(pa & 0xffff0000u));
+                da = pack_bf16x2(d0 - __uint_as_float(da << 16), d1 - __uint_as_float(da & 0xffff0000u));
+              }
+              pp[x >> 1] = pa;
+              dsp[x >> 1] = da;
+            }
+            // query columns [16ch, 16ch + 16) -> packed columns 32*(ch/2) + 8*(ch%2) .. +8 (never ahead of a
+            // column this thread still has to read)
+            tmem_st8(tS + (ch >> 1) * 32 + (ch & 1) * 8, pp);
+            *reinterpret_cast<uint4*>(ds_row + ((2 * ch) ^ (r & 7)) * 16) = make_uint4(dsp[0], dsp[1], dsp[2], dsp[3]);
+            *reinterpret_cast<uint4*>(ds_row + ((2 * ch + 1) ^ (r & 7)) * 16) = make_uint4(dsp[4], dsp[5], dsp[6], dsp[7]);
           }
+          tmem_wait_st();
+          tc_fence_before_sync();
+          mbar_arrive(&s.bar_p_ready);
         }
-        if (!oks) break;
-        tmem_wait_st();
         fence_proxy_async_smem();
         tc_fence_before_sync();
-        mbar_arrive(&s.bar_p_ready);
+        mbar_arrive(&s.bar_ds_ready);
         mbar_arrive(&s.bar_ld_empty[st]);
+        if (tid == 0) NSP_TRACE_STAMP(9);
       }
       // ---- epilogue: wait for the last MMAs of the item, then write dK (scaled) and dV of this key tile
       if (oks) {
-        oks = mbar_wait(&s.bar_dq_full, (gs + c.steps - 1) & 1);
+        oks = mbar_wait(&s.bar_dq_full, (gs + c.steps - 1) & 1) && mbar_wait(&s.bar_a_done, (gs + c.steps - 1) & 1);
         oks = __all_sync(0xffffffffu, oks);
         if (!oks) where = kWhereBwdDqFull;
       }
       if (oks) {
         tc_fence_after_sync();
         const int kj = c.n * kBN + r;
-        const bool valid = kj < sg.len;
-        const int64_t off = sg.kv_off + (static_cast<int64_t>(kj) * sg.hkv + c.g) * kHeadDim + half * 64;
-#pragma unroll
-        for (int which = 0; which < 2; ++which) {
-          const uint32_t tsrc = which == 0 ? tDK : tDV;
+        const bool valid = kj < c.len;
+        const int64_t off = c.kv_off + (static_cast<int64_t>(kj) * c.hkv + c.g) * kHeadDim + half * 64;
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {  // (dK, dV) x two 32-column chunks
+          const int which = part >> 1, cc = part & 1;
           const float mul = which == 0 ? a.scale : 1.f;
           void* outp = which == 0 ? a.dk : a.dv;
+          uint32_t v[32];
+          tmem_ld32(tDK + which * 128 + lane_off + half * 64 + cc * 32, v);
+          tmem_wait_ld();
+          if (valid) {
+            if (a.dkv_f32) {
+              float* o = static_cast<float*>(outp) + off + cc * 32;
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            uint32_t v[32];
-            tmem_ld32(tsrc + lane_off + half * 64 + cc * 32, v);
-            tmem_wait_ld();
-            if (valid) {
-              if (a.dkv_f32) {
-                float* o = static_cast<float*>(outp) + off + cc * 32;
+              for (int x = 0; x < 32; x += 4)
+                *reinterpret_cast<float4*>(o + x) =
+                    make_float4(__uint_as_float(v[x]) * mul, __uint_as_float(v[x + 1]) * mul,
+                                __uint_as_float(v[x + 2]) * mul, __uint_as_float(v[x + 3]) * mul);
+            } else {
+              __nv_bfloat16* o = static_cast<__nv_bfloat16*>(outp) + off + cc * 32;
 #pragma unroll
-                for (int x = 0; x < 32; x += 4)
-                  *reinterpret_cast<float4*>(o + x) =
-                      make_float4(__uint_as_float(v[x]) * mul, __uint_as_float(v[x + 1]) * mul,
-                                  __uint_as_float(v[x + 2]) * mul, __uint_as_float(v[x + 3]) * mul);
-              } else {
-                __nv_bfloat16* o = static_cast<__nv_bfloat16*>(outp) + off + cc * 32;
-#pragma unroll
-                for (int x = 0; x < 32; x += 8) {
-                  uint4 w;
-                  w.x = pack_bf16x2(__uint_as_float(v[x]) * mul, __uint_as_float(v[x + 1]) * mul);
-                  w.y = pack_bf16x2(__uint_as_float(v[x + 2]) * mul, __uint_as_float(v[x + 3]) * mul);
-                  w.z = pack_bf16x2(__uint_as_float(v[x + 4]) * mul, __uint_as_float(v[x + 5]) * mul);
-                  w.w = pack_bf16x2(__uint_as_float(v[x + 6]) * mul, __uint_as_float(v[x + 7]) * mul);
-                  *reinterpret_cast<uint4*>(o + x) = w;
-                }
+              for (int x = 0; x < 32; x += 8) {
+                uint4 wv;
+                wv.x = pack_bf16x2(__uint_as_float(v[x]) * mul, __uint_as_float(v[x + 1]) * mul);
+                wv.y = pack_bf16x2(__uint_as_float(v[x + 2]) * mul, __uint_as_float(v[x + 3]) * mul);
+                wv.z = pack_bf16x2(__uint_as_float(v[x + 4]) * mul, __uint_as_float(v[x + 5]) * mul);
+                wv.w = pack_bf16x2(__uint_as_float(v[x + 6]) * mul, __uint_as_float(v[x + 7]) * mul);
+                *reinterpret_cast<uint4*>(o + x) = wv;
               }
             }
           }
         }
       } else if (where != 0 && lane == 0) {
-        report_timeout(a.status, it, where, 0);
+        report_timeout(a.status, c.it, where, 0);
         *abort_flag = 1;
       }
       item_done();
-      }
     }
   }
 
@@ -611,6 +763,12 @@ __global__ void bwd_postprocess_kernel(const float* __restrict__ acc, void* __re
 }
 
 }  // namespace
+
+#ifdef NSP_TRACE
+extern "C" int nsp_debug_trace_read(long long* host, int n) {
+  return cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
                                   const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, cudaStream_t st) {

@@ -203,23 +203,28 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             const int joint = rd.joint;
             int where = 0;
             // S_x of key tile in stage kst -> TMEM columns [128*x, 128*x + 128)
+            // Descriptors are built once per round; inside the loops an operand advances by adding the byte
+            // offset (in 16-byte units) to the low word, which keeps the single issuing thread fast.
+            const uint64_t dq[2] = {make_smem_desc_sw128(smem_u32(s.q[0][0]), 16, 1024),
+                                    make_smem_desc_sw128(smem_u32(s.q[1][0]), 16, 1024)};
+            const uint64_t dk[2] = {make_smem_desc_sw128(smem_u32(s.k[0][0]), 16, 1024),
+                                    make_smem_desc_sw128(smem_u32(s.k[1][0]), 16, 1024)};
+            const uint64_t dv[2] = {make_smem_desc_sw128(smem_u32(s.v[0][0]), kHalfTileBytes, 1024),
+                                    make_smem_desc_sw128(smem_u32(s.v[1][0]), kHalfTileBytes, 1024)};
             auto issue_s = [&](int x, uint32_t kst) {
-              const uint32_t q_addr = smem_u32(s.q[x][0]), k_addr = smem_u32(s.k[kst][0]);
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t off = (kk >> 2) * kHalfTileBytes + (kk & 3) * 32;
-                umma_ss(tmem + 128 * x, make_smem_desc_sw128(q_addr + off, 16, 1024),
-                        make_smem_desc_sw128(k_addr + off, 16, 1024), idesc_qk, kk > 0);
+                const uint64_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
+                umma_ss(tmem + 128 * x, dq[x] + off, dk[kst] + off, idesc_qk, kk > 0);
               }
               umma_commit(&s.bar_s_full[x]);
             };
             // O_x += P_x V (P_x: bf16 pairs in the first 64 columns of S_x)
             auto issue_pv = [&](int x, uint32_t vst, int j) {
-              const uint32_t v_addr = smem_u32(s.v[vst][0]);
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk)
-                umma_ts(tmem + 256 + 128 * x, tmem + 128 * x + kk * 8,
-                        make_smem_desc_sw128(v_addr + kk * 2048, kHalfTileBytes, 1024), idesc_pv, (j > 0 || kk > 0));
+                umma_ts(tmem + 256 + 128 * x, tmem + 128 * x + kk * 8, dv[vst] + ((kk * 2048) >> 4), idesc_pv,
+                        (j > 0 || kk > 0));
               umma_commit(&s.bar_pv_done[x]);
             };
             bool ok = mbar_wait(&s.bar_q, qn & 1);

@@ -37,7 +37,6 @@ struct FwdMaps {
 };
 struct BwdMaps {
   CUtensorMap q[NSP_MAX_RUNS], d_o[NSP_MAX_RUNS], k[NSP_MAX_RUNS], v[NSP_MAX_RUNS];
-  CUtensorMap dq[NSP_MAX_RUNS];  // fp32 dQ accumulator, tiles {32 dims, 1 head, 128 tokens}
 };
 
 // Device status word: {code, item, where, aux}; first writer wins (atomicCAS on code).
@@ -63,6 +62,7 @@ enum DeviceWhere : int32_t {
   kWhereBwdDelta = 23,
   kWhereBwdDsReady = 24,
   kWhereBwdItemBarrier = 25,
+  kWhereBwdTmemBase = 26,
 };
 
 __device__ __forceinline__ void report_timeout(int32_t* status, int32_t item, int32_t where, int32_t aux) {
