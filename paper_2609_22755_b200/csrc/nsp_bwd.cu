@@ -78,16 +78,19 @@ struct ItemCtx {
 struct BwdSmem {
   uint8_t k[2][kHalfTileBytes];
   uint8_t v[2][kHalfTileBytes];
-  uint8_t q[2][2][kHalfTileBytes];    // [stage][64-column half]
-  uint8_t d_o[2][2][kHalfTileBytes];  // [stage][half]
+  uint8_t q[3][2][kHalfTileBytes];    // [stage][64-column half]: three-stage ring, loaded a whole step ahead
+  uint8_t d_o[2][kHalfTileBytes];     // [half]: single buffer (its consumers leave a long window for the refill)
   uint8_t ds[2][kHalfTileBytes];      // dS^T, [key row][query col], two 64-column halves
   float lse[2][128];                  // [stage] LSE * log2(e) of the q tile (+inf for rows past the segment)
   float delta[2][128];                // [stage]
   ItemCtx ctx[2];
   uint64_t bar_kv;
-  uint64_t bar_q_full[2];
-  uint64_t bar_q_empty[2][2];  // [stage][issuer A / B]: that issuer's MMAs reading the stage have completed
+  uint64_t bar_q_full[3];
+  uint64_t bar_q_empty[3][2];  // [stage][issuer A / B]: that issuer's MMAs reading the Q stage have completed
+  uint64_t bar_do_full;
+  uint64_t bar_do_empty[2];    // [issuer A / B]: that issuer's MMAs reading the dO buffer have completed
   uint64_t bar_a_done;         // dV of the step (issuer A) has completed
+  uint64_t bar_b_done;         // dK of the step (issuer B) has completed
   uint64_t bar_ld_full[2], bar_ld_empty[2];
   uint64_t bar_s_full, bar_dp_full, bar_dq_full, bar_dq_empty;
   uint64_t bar_p_ready;   // 256 softmax threads: P^T of the step is in R0
@@ -135,6 +138,15 @@ struct StepWalk {
   }
 };
 
+// Position in the three-stage Q ring; it runs on across items. ph is the parity of the number of earlier uses of
+// the current stage.
+struct QRing {
+  uint32_t st = 0, ph = 0;
+  __device__ __forceinline__ void next() {
+    if (++st == 3) st = 0, ph ^= 1;
+  }
+};
+
 __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   BwdSmem& s = *reinterpret_cast<BwdSmem*>(smem_raw);
@@ -146,10 +158,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
 
   if (tid == 0) {
     mbar_init(&s.bar_kv, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 3; ++i) {
       mbar_init(&s.bar_q_full[i], 1);
       mbar_init(&s.bar_q_empty[i][0], 1);
       mbar_init(&s.bar_q_empty[i][1], 1);
+    }
+    mbar_init(&s.bar_do_full, 1);
+    mbar_init(&s.bar_do_empty[0], 1);
+    mbar_init(&s.bar_do_empty[1], 1);
+    for (int i = 0; i < 2; ++i) {
       mbar_init(&s.bar_ld_full[i], 32);
       mbar_init(&s.bar_ld_empty[i], 256);
     }
@@ -159,6 +176,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     mbar_init(&s.bar_ds_ready, 256);
     mbar_init(&s.bar_dq_full, 1);
     mbar_init(&s.bar_a_done, 1);
+    mbar_init(&s.bar_b_done, 1);
     mbar_init(&s.bar_dq_empty, 256);
     mbar_init(&s.bar_delta[0], 128);
     mbar_init(&s.bar_delta[1], 128);
@@ -223,6 +241,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     setmaxnreg_dec<kRegsAux>();
     if (warp == 16) {
       // ================================================================ TMA producer
+      // Q(t) goes into a three-stage ring and is requested about one step before S^T(t) needs it; dO(t) goes
+      // into a single buffer that is free from the end of dV(t-1) until dP^T(t). Requests are issued in the
+      // order Q(0), dO(0), Q(1), dO(1), ...: the wait for the dO buffer is the one that paces the loop.
+      QRing qr;
       while (next_item()) {
         if (lane == 0) {
           const ItemCtx c = *cx;
@@ -237,23 +259,29 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           w.reset();
 #pragma unroll 1
           for (int vt = 0; vt < c.steps; ++vt) {
-            const uint32_t cs = gs + vt, st = cs & 1;
+            const uint32_t cs = gs + vt;
             if (*abort_flag) break;
-            if (!mbar_wait(&s.bar_q_empty[st][0], ((cs >> 1) & 1) ^ 1) ||
-                !mbar_wait(&s.bar_q_empty[st][1], ((cs >> 1) & 1) ^ 1)) {
+            int h, m, mode;
+            w.get(c, h, m, mode);
+            w.next(c);
+            if (!mbar_wait(&s.bar_q_empty[qr.st][0], qr.ph ^ 1) || !mbar_wait(&s.bar_q_empty[qr.st][1], qr.ph ^ 1)) {
               report_timeout(a.status, c.it, kWhereBwdQEmpty, vt);
               *abort_flag = 1;
               break;
             }
             NSP_TRACE_STAMP(14);
-            int h, m, mode;
-            w.get(c, h, m, mode);
-            w.next(c);
-            mbar_expect_tx(&s.bar_q_full[st], 2 * kTileBytes);
-            tma_load_3d(s.q[st][0], mq, &s.bar_q_full[st], 0, h, c.tok0 + m * kBM);
-            tma_load_3d(s.q[st][1], mq, &s.bar_q_full[st], 64, h, c.tok0 + m * kBM);
-            tma_load_3d(s.d_o[st][0], mdo, &s.bar_q_full[st], 0, h, c.tok0 + m * kBM);
-            tma_load_3d(s.d_o[st][1], mdo, &s.bar_q_full[st], 64, h, c.tok0 + m * kBM);
+            mbar_expect_tx(&s.bar_q_full[qr.st], kTileBytes);
+            tma_load_3d(s.q[qr.st][0], mq, &s.bar_q_full[qr.st], 0, h, c.tok0 + m * kBM);
+            tma_load_3d(s.q[qr.st][1], mq, &s.bar_q_full[qr.st], 64, h, c.tok0 + m * kBM);
+            qr.next();
+            if (!mbar_wait(&s.bar_do_empty[0], (cs & 1) ^ 1) || !mbar_wait(&s.bar_do_empty[1], (cs & 1) ^ 1)) {
+              report_timeout(a.status, c.it, kWhereBwdQEmpty, 100000 + vt);
+              *abort_flag = 1;
+              break;
+            }
+            mbar_expect_tx(&s.bar_do_full, kTileBytes);
+            tma_load_3d(s.d_o[0], mdo, &s.bar_do_full, 0, h, c.tok0 + m * kBM);
+            tma_load_3d(s.d_o[1], mdo, &s.bar_do_full, 64, h, c.tok0 + m * kBM);
           }
         }
         item_done();
@@ -266,6 +294,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       // the MMAs of the other. Each thread signals completion on barriers of its own (a tcgen05.commit covers
       // only the issuing thread's MMAs); whoever depends on both waits for both.
       const bool is_a = warp == 17;
+      QRing qr;
       while (next_item()) {
         if (lane == 0) {
           constexpr uint32_t idesc_kk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
@@ -277,92 +306,93 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           // MN-major operands step 16 rows = 2048 bytes. The high word is the same for both kinds.
           const uint32_t hi = static_cast<uint32_t>(make_smem_desc_sw128(0, 16, 1024) >> 32);
           constexpr uint32_t lbo_km = (16u >> 4) << 16, lbo_mn = (kHalfTileBytes >> 4) << 16;
-          constexpr uint32_t kStageStep = kTileBytes >> 4;  // descriptor distance between the two stages
+          constexpr uint32_t kStageStep = kTileBytes >> 4;  // descriptor distance between Q stages
           const int steps = cx->steps, item_it = cx->it;
           int where = 0;
           bool okm = mbar_wait(&s.bar_kv, gi & 1);
           if (!okm) where = kWhereBwdLoadKV;
+          const uint32_t q0_lo = smem_u32(s.q[0][0]) >> 4, do_lo = smem_u32(s.d_o[0]) >> 4;
           if (is_a) {
             const uint32_t k_km = (smem_u32(s.k[0]) >> 4) | lbo_km;
-            const uint32_t q0_lo = smem_u32(s.q[0][0]) >> 4, do0_lo = smem_u32(s.d_o[0][0]) >> 4;
-            // S^T of step vt -> R0 (A = K, B = Q of the step's stage, both K-major)
-            auto issue_s = [&](int vt) -> bool {
-              const uint32_t cs = gs + vt, st = cs & 1;
-              if (!mbar_wait(&s.bar_q_full[st], (cs >> 1) & 1)) { where = kWhereBwdLoadQ; return false; }
+            // S^T of the next step not yet issued -> R0 (A = K, B = Q of the ring stage, both K-major)
+            auto issue_s = [&]() -> bool {
+              if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph)) { where = kWhereBwdLoadQ; return false; }
               tc_fence_after_sync();
-              const uint32_t b_lo = (q0_lo + st * kStageStep) | lbo_km;
+              const uint32_t b_lo = (q0_lo + qr.st * kStageStep) | lbo_km;
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
                 umma_ss_lh(tR0, k_km + off, hi, b_lo + off, hi, idesc_kk, kk > 0);
               }
               umma_commit(&s.bar_s_full);
+              umma_commit(&s.bar_q_empty[qr.st][0]);  // this thread is done with the Q stage
+              qr.next();
               return true;
             };
-            okm = okm && issue_s(0);
+            okm = okm && issue_s();
 #pragma unroll 1
             for (int vt = 0; okm && vt < steps; ++vt) {
-              const uint32_t cs = gs + vt, st = cs & 1;
+              const uint32_t cs = gs + vt;
               if (*abort_flag) break;
+              if (!mbar_wait(&s.bar_do_full, cs & 1)) { okm = false; where = kWhereBwdLoadQ; break; }
               if (!mbar_wait(&s.bar_p_ready, cs & 1)) { okm = false; where = kWhereBwdPReady; break; }
               NSP_TRACE_STAMP(0);
               tc_fence_after_sync();
               const uint32_t acc = vt > 0;
-              const uint32_t do_mn = (do0_lo + st * kStageStep) | lbo_mn;
               // dV += P^T dO; packed P^T columns of K-step kk (16 query columns) sit at R0 + (kk/2)*32 + (kk%2)*8
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk)
-                umma_ts_lh(tDV, tR0 + (kk >> 1) * 32 + (kk & 1) * 8, do_mn + kk * 128, hi, idesc_kn, acc | (kk > 0));
-              umma_commit(&s.bar_a_done);          // S^T and dV of the step
-              umma_commit(&s.bar_q_empty[st][0]);
+                umma_ts_lh(tDV, tR0 + (kk >> 1) * 32 + (kk & 1) * 8, (do_lo | lbo_mn) + kk * 128, hi, idesc_kn,
+                           acc | (kk > 0));
+              umma_commit(&s.bar_a_done);       // S^T and dV of the step
+              umma_commit(&s.bar_do_empty[0]);  // this thread is done with the dO buffer
               NSP_TRACE_STAMP(15);
-#ifdef NSP_TRACE
-              if (vt + 1 < steps) mbar_wait(&s.bar_q_full[(cs + 1) & 1], ((cs + 1) >> 1) & 1);
-              NSP_TRACE_STAMP(13);
-#endif
-              if (vt + 1 < steps && !issue_s(vt + 1)) { okm = false; break; }
+              if (vt + 1 < steps && !issue_s()) { okm = false; break; }
               NSP_TRACE_STAMP(1);
             }
           } else {
             const uint32_t v_km = (smem_u32(s.v[0]) >> 4) | lbo_km, k_mn = (smem_u32(s.k[0]) >> 4) | lbo_mn;
             const uint32_t ds_km = (smem_u32(s.ds[0]) >> 4) | lbo_km, ds_mn = (smem_u32(s.ds[0]) >> 4) | lbo_mn;
-            const uint32_t q0_lo = smem_u32(s.q[0][0]) >> 4, do0_lo = smem_u32(s.d_o[0][0]) >> 4;
             // dP^T of step vt -> R1, once the dQ warps have drained dQ^T of the previous step from it
             auto issue_dp = [&](int vt) -> bool {
-              const uint32_t cs = gs + vt, st = cs & 1;
-              if (!mbar_wait(&s.bar_q_full[st], (cs >> 1) & 1)) { where = kWhereBwdLoadQ; return false; }
+              const uint32_t cs = gs + vt;
+              if (!mbar_wait(&s.bar_do_full, cs & 1)) { where = kWhereBwdLoadQ; return false; }
               if (!mbar_wait(&s.bar_dq_empty, (cs & 1) ^ 1)) { where = kWhereBwdDqEmpty; return false; }
               tc_fence_after_sync();
-              const uint32_t b_lo = (do0_lo + st * kStageStep) | lbo_km;
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
-                umma_ss_lh(tR1, v_km + off, hi, b_lo + off, hi, idesc_kk, kk > 0);
+                umma_ss_lh(tR1, v_km + off, hi, (do_lo | lbo_km) + off, hi, idesc_kk, kk > 0);
               }
               umma_commit(&s.bar_dp_full);
+              umma_commit(&s.bar_do_empty[1]);  // this thread is done with the dO buffer
               return true;
             };
             okm = okm && issue_dp(0);
 #pragma unroll 1
             for (int vt = 0; okm && vt < steps; ++vt) {
-              const uint32_t cs = gs + vt, st = cs & 1;
+              const uint32_t cs = gs + vt;
               if (*abort_flag) break;
+              if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph)) { okm = false; where = kWhereBwdLoadQ; break; }
               if (!mbar_wait(&s.bar_ds_ready, cs & 1)) { okm = false; where = kWhereBwdDsReady; break; }
               NSP_TRACE_STAMP(2);
               tc_fence_after_sync();
               const uint32_t acc = vt > 0;
-              const uint32_t q_mn = (q0_lo + st * kStageStep) | lbo_mn;
+              const uint32_t q_mn = (q0_lo + qr.st * kStageStep) | lbo_mn;
+              // dQ^T = K^T dS^T -> R1 (dP^T of this step has been consumed: ds_ready). It goes first: the dQ warps
+              // drain R1 while dK runs, so that dP^T of the next step can follow dK without a gap.
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk) umma_ss_lh(tR1, k_mn + kk * 128, hi, ds_mn + kk * 128, hi, idesc_nn, kk > 0);
+              umma_commit(&s.bar_dq_full);
               // dK += dS^T Q
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
                 umma_ss_lh(tDK, ds_km + off, hi, q_mn + kk * 128, hi, idesc_kn, acc | (kk > 0));
               }
-              // dQ^T = K^T dS^T -> R1 (dP^T of this step has been consumed: ds_ready)
-#pragma unroll
-              for (int kk = 0; kk < 8; ++kk) umma_ss_lh(tR1, k_mn + kk * 128, hi, ds_mn + kk * 128, hi, idesc_nn, kk > 0);
-              umma_commit(&s.bar_dq_full);         // dP^T, dK and dQ^T of the step
-              umma_commit(&s.bar_q_empty[st][1]);
+              umma_commit(&s.bar_b_done);              // dP^T, dQ^T and dK of the step
+              umma_commit(&s.bar_q_empty[qr.st][1]);  // this thread is done with the Q stage
+              qr.next();
               NSP_TRACE_STAMP(3);
               if (vt + 1 < steps && !issue_dp(vt + 1)) { okm = false; break; }
               NSP_TRACE_STAMP(4);
@@ -532,10 +562,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
 #pragma unroll
             for (int x = 0; x < 32; x += 4) {
               const float4 l4 = *reinterpret_cast<const float4*>(lse_s + cc * 32 + x);
-              const float p0 = ex2f(fmaf(__uint_as_float(pv[cc][x + 0]), a.scale_log2, -l4.x));
-              const float p1 = ex2f(fmaf(__uint_as_float(pv[cc][x + 1]), a.scale_log2, -l4.y));
-              const float p2 = ex2f(fmaf(__uint_as_float(pv[cc][x + 2]), a.scale_log2, -l4.z));
-              const float p3 = ex2f(fmaf(__uint_as_float(pv[cc][x + 3]), a.scale_log2, -l4.w));
+              float x0, x1, x2, x3;
+              fma2(x0, x1, __uint_as_float(pv[cc][x + 0]), __uint_as_float(pv[cc][x + 1]), a.scale_log2, a.scale_log2,
+                   -l4.x, -l4.y);
+              fma2(x2, x3, __uint_as_float(pv[cc][x + 2]), __uint_as_float(pv[cc][x + 3]), a.scale_log2, a.scale_log2,
+                   -l4.z, -l4.w);
+              const float p0 = ex2f(x0), p1 = ex2f(x1), p2 = ex2f(x2), p3 = ex2f(x3);
               pv[cc][x + 0] = __float_as_uint(p0);
               pv[cc][x + 1] = __float_as_uint(p1);
               pv[cc][x + 2] = __float_as_uint(p2);
@@ -544,12 +576,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               pp[(x >> 1) + 1] = pack_bf16x2(p2, p3);
             }
             tmem_st16(tS + cc * 32, pp);  // query columns [32cc, 32cc + 32) -> packed columns [32cc, 32cc + 16)
+            if (tid == 0) NSP_TRACE_STAMP(16 + cc);
           }
           tmem_wait_st();
+          if (tid == 0) NSP_TRACE_STAMP(18);
           tc_fence_before_sync();
           mbar_arrive(&s.bar_p_ready);
           if (tid == 0) NSP_TRACE_STAMP(7);
-          if (lane == 0) NSP_TRACE_STAMP(16 + warp);
           // Phase 2: dS^T = P^T o (dP^T - delta) -> swizzled shared memory. The dS buffer is free: dP^T of this
           // step was issued behind dK / dQ^T of the previous step, so bar_dp_full implies they have completed.
           oks = mbar_wait(&s.bar_dp_full, cs & 1);
@@ -562,13 +595,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             uint32_t dpv[32], dsp[16];
             tmem_ld32(tDP + cc * 32, dpv);
             tmem_wait_ld();
+            if (tid == 0) NSP_TRACE_STAMP(19 + 2 * cc);
 #pragma unroll
             for (int x = 0; x < 32; x += 4) {
               const float4 d4 = *reinterpret_cast<const float4*>(delta_s + cc * 32 + x);
-              const float d0 = __uint_as_float(pv[cc][x + 0]) * (__uint_as_float(dpv[x + 0]) - d4.x);
-              const float d1 = __uint_as_float(pv[cc][x + 1]) * (__uint_as_float(dpv[x + 1]) - d4.y);
-              const float d2 = __uint_as_float(pv[cc][x + 2]) * (__uint_as_float(dpv[x + 2]) - d4.z);
-              const float d3 = __uint_as_float(pv[cc][x + 3]) * (__uint_as_float(dpv[x + 3]) - d4.w);
+              float d0, d1, d2, d3;
+              sub2(d0, d1, __uint_as_float(dpv[x + 0]), __uint_as_float(dpv[x + 1]), d4.x, d4.y);
+              sub2(d2, d3, __uint_as_float(dpv[x + 2]), __uint_as_float(dpv[x + 3]), d4.z, d4.w);
+              mul2(d0, d1, d0, d1, __uint_as_float(pv[cc][x + 0]), __uint_as_float(pv[cc][x + 1]));
+              mul2(d2, d3, d2, d3, __uint_as_float(pv[cc][x + 2]), __uint_as_float(pv[cc][x + 3]));
               dsp[(x >> 1) + 0] = pack_bf16x2(d0, d1);
               dsp[(x >> 1) + 1] = pack_bf16x2(d2, d3);
             }
@@ -579,6 +614,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               *reinterpret_cast<uint4*>(ds_row + chunk * 16) =
                   make_uint4(dsp[ch * 4 + 0], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
             }
+            if (tid == 0) NSP_TRACE_STAMP(20 + 2 * cc);
           }
         } else {
           // ---- rare step (diagonal tile and/or one of the two first-tile passes): compact rolled loops, 16 query
@@ -661,7 +697,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       }
       // ---- epilogue: wait for the last MMAs of the item, then write dK (scaled) and dV of this key tile
       if (oks) {
-        oks = mbar_wait(&s.bar_dq_full, (gs + c.steps - 1) & 1) && mbar_wait(&s.bar_a_done, (gs + c.steps - 1) & 1);
+        oks = mbar_wait(&s.bar_b_done, (gs + c.steps - 1) & 1) && mbar_wait(&s.bar_a_done, (gs + c.steps - 1) & 1);
         oks = __all_sync(0xffffffffu, oks);
         if (!oks) where = kWhereBwdDqFull;
       }

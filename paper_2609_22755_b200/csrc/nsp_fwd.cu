@@ -48,7 +48,8 @@ struct FwdSmem {
   uint64_t bar_s_full[2];   // [A/B] S_x of a key tile is in TMEM
   uint64_t bar_p_ready[2];  // [A/B] 256 softmax threads: P_x written (and O_x rescaled if needed)
   uint64_t bar_pair[2][4];  // [A/B][lane quadrant] the two threads of every row have published their half-row value
-  float xchg[2][2][128];    // [A/B][column half][row] half-row maximum (or row sum) handed to the partner thread
+  float xchg[2][2][3][128];  // [A/B][column half][slot][row] half-row maximum (slots 0/1 by tile parity) or row sum
+                             // (slot 2) handed to the partner thread
   uint64_t bar_pv_done[2];  // [A/B] O_x += P_x V has completed
   uint32_t tmem_base;
   int32_t item_idx[2];
@@ -203,28 +204,31 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             const int joint = rd.joint;
             int where = 0;
             // S_x of key tile in stage kst -> TMEM columns [128*x, 128*x + 128)
-            // Descriptors are built once per round; inside the loops an operand advances by adding the byte
+            // Descriptors are {low word, high word}; inside the loops an operand advances by adding its byte
             // offset (in 16-byte units) to the low word, which keeps the single issuing thread fast.
-            const uint64_t dq[2] = {make_smem_desc_sw128(smem_u32(s.q[0][0]), 16, 1024),
-                                    make_smem_desc_sw128(smem_u32(s.q[1][0]), 16, 1024)};
-            const uint64_t dk[2] = {make_smem_desc_sw128(smem_u32(s.k[0][0]), 16, 1024),
-                                    make_smem_desc_sw128(smem_u32(s.k[1][0]), 16, 1024)};
-            const uint64_t dv[2] = {make_smem_desc_sw128(smem_u32(s.v[0][0]), kHalfTileBytes, 1024),
-                                    make_smem_desc_sw128(smem_u32(s.v[1][0]), kHalfTileBytes, 1024)};
+            const uint32_t hi = static_cast<uint32_t>(make_smem_desc_sw128(0, 16, 1024) >> 32);
+            constexpr uint32_t lbo_km = (16u >> 4) << 16, lbo_mn = (kHalfTileBytes >> 4) << 16;
+            const uint32_t q_lo = (smem_u32(s.q[0][0]) >> 4) | lbo_km;  // item B: + kTileBytes / 16
+            const uint32_t k_lo = (smem_u32(s.k[0][0]) >> 4) | lbo_km;  // stage 1: + kTileBytes / 16
+            const uint32_t v_lo = (smem_u32(s.v[0][0]) >> 4) | lbo_mn;
+            constexpr uint32_t kTileStep = kTileBytes >> 4;
+            // S_x of key tile in stage kst -> TMEM columns [128*x, 128*x + 128)
             auto issue_s = [&](int x, uint32_t kst) {
+              const uint32_t a_lo = q_lo + x * kTileStep, b_lo = k_lo + kst * kTileStep;
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
-                const uint64_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
-                umma_ss(tmem + 128 * x, dq[x] + off, dk[kst] + off, idesc_qk, kk > 0);
+                const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
+                umma_ss_lh(tmem + 128 * x, a_lo + off, hi, b_lo + off, hi, idesc_qk, kk > 0);
               }
               umma_commit(&s.bar_s_full[x]);
             };
-            // O_x += P_x V (P_x: bf16 pairs in the first 64 columns of S_x)
+            // O_x += P_x V (P_x: bf16 pairs in columns [0,32) and [64,96) of S_x)
             auto issue_pv = [&](int x, uint32_t vst, int j) {
+              const uint32_t b_lo = v_lo + vst * kTileStep;
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk)
-                umma_ts(tmem + 256 + 128 * x, tmem + 128 * x + kk * 8, dv[vst] + ((kk * 2048) >> 4), idesc_pv,
-                        (j > 0 || kk > 0));
+                umma_ts_lh(tmem + 256 + 128 * x, tmem + 128 * x + (kk >> 2) * 64 + (kk & 3) * 8, b_lo + kk * 128, hi, idesc_pv,
+                           (j > 0 || kk > 0));
               umma_commit(&s.bar_pv_done[x]);
             };
             bool ok = mbar_wait(&s.bar_q, qn & 1);
@@ -299,8 +303,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     uint32_t sn = 0;   // S tiles consumed so far
     uint32_t pvn = 0;  // PV products of this half issued before the current round
     uint32_t xn = 0;   // completed phases of this row pair's exchange barrier
-    float* my_slot = &s.xchg[x][ch][rl];
-    const float* partner_slot = &s.xchg[x][ch ^ 1][rl];
+    float* my_slot = &s.xchg[x][ch][0][rl];                   // slot k is my_slot[128 * k]
+    const float* partner_slot = &s.xchg[x][ch ^ 1][0][rl];
     uint64_t* pair_bar = &s.bar_pair[x][quad];
     while (next_pop()) {
       for (int r = 0; r < n_rounds; ++r) {
@@ -311,6 +315,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           const int h = ia.head, n_kv = ia.cost, q_row0 = ia.tile * kBM;
           float m_ref = -INFINITY;  // reference maximum (log2 domain) the stored P and l are relative to
           float l = 0.f;            // running sum of exp2(s - m_ref) over this thread's columns
+          float mx_posted = 0.f;    // this thread's half-row maximum of the previous tile (when `pending`)
+          bool pending = false;     // the previous tile's half-row maxima have been posted and not yet consumed
           bool ok = true;
           int where = 0;
           for (int j = 0; j < n_kv; ++j) {
@@ -326,61 +332,76 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             tmem_ld32(tS + lane_off + ch * 64 + 32, sr[1]);
             tmem_wait_ld();
             if (rl == 0 && ch == 0) NSP_FTRACE(5 + 8 * x);
-            float mx = -INFINITY;
-            if (j == n_kv - 1) {  // diagonal tile: keys past the query are masked
+            const bool last = (j == n_kv - 1);
+            if (last) {  // diagonal tile: keys past the query are masked
 #pragma unroll
               for (int c = 0; c < 2; ++c)
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                  float val = __uint_as_float(sr[c][e]);
-                  if (ch * 64 + c * 32 + e > rl) val = -INFINITY;
-                  sr[c][e] = __float_as_uint(val);
-                  mx = fmaxf(mx, val);
-                }
-            } else {
+                for (int e = 0; e < 32; ++e)
+                  if (ch * 64 + c * 32 + e > rl) sr[c][e] = __float_as_uint(-INFINITY);
+            }
+            // The reference maximum lags one tile behind: only the first tile of an item takes its row maximum
+            // before exponentiating. Every later tile is exponentiated against the reference it finds, and its
+            // own maximum is posted AFTER P has been handed to the MMA thread and folded in at the start of the
+            // next tile. The result is the same (any reference gives the same O and LSE as long as nothing
+            // overflows: a tile would have to exceed all earlier tiles of its row by 2^100 for that), but the
+            // maximum and its exchange between the two threads of a row leave the S -> P -> PV critical path.
+            bool need = false;
+            float alpha = 1.f;
+            if (j == 0) {
+              float mx = -INFINITY;
 #pragma unroll
               for (int c = 0; c < 2; ++c)
 #pragma unroll
                 for (int e = 0; e < 32; e += 2)
                   mx = max3f(mx, __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
+              my_slot[0] = mx;
+              mbar_arrive(pair_bar);
+              ok = mbar_wait(pair_bar, xn & 1);
+              ++xn;
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) { where = kWhereFwdPair; break; }
+              m_ref = fmaxf(mx, partner_slot[0]) * a.scale_log2;
+            } else if (pending) {
+              ok = mbar_wait(pair_bar, xn & 1);
+              if (rl == 0 && ch == 0) NSP_FTRACE(7 + 8 * x);
+              ++xn;
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) { where = kWhereFwdPair; break; }
+              const float mx = fmaxf(mx_posted, partner_slot[128 * ((j - 1) & 1)]) * a.scale_log2;
+              need = mx > m_ref + 8.f;
+              if (need) {
+                alpha = ex2f(m_ref - mx);
+                m_ref = mx;
+              }
+              pending = false;
             }
-            // row maximum = max of the two half rows (the partner has also finished reading its S columns by
-            // the time its value is visible, so P may then be written over any part of S_x)
-            *my_slot = mx;
-            mbar_arrive(pair_bar);
-            ok = mbar_wait(pair_bar, xn & 1);
-            ++xn;
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) { where = kWhereFwdPair; break; }
-            mx = fmaxf(mx, *partner_slot) * a.scale_log2;
             if (rl == 0 && ch == 0) NSP_FTRACE(6 + 8 * x);
-            const bool need = mx > m_ref + 8.f;
-            float alpha = 1.f;
-            if (need) {
-              alpha = ex2f(m_ref - mx);
-              m_ref = mx;
-            }
             l *= alpha;
-            float sum = 0.f;
+            float sum0 = 0.f, sum1 = 0.f;
+            float mx_tile = -INFINITY;  // this tile's half-row maximum (raw scores), for the next tile
+            const float neg_m = -m_ref;
             uint32_t pk[32];
 #pragma unroll
             for (int c = 0; c < 2; ++c)
 #pragma unroll
               for (int e = 0; e < 32; e += 2) {
-                const float p0 = ex2f(fmaf(__uint_as_float(sr[c][e]), a.scale_log2, -m_ref));
-                const float p1 = ex2f(fmaf(__uint_as_float(sr[c][e + 1]), a.scale_log2, -m_ref));
-                sum += p0 + p1;
+                float x0, x1;
+                mx_tile = max3f(mx_tile, __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
+                fma2(x0, x1, __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]), a.scale_log2, a.scale_log2, neg_m,
+                     neg_m);
+                const float p0 = ex2f(x0), p1 = ex2f(x1);
+                add2(sum0, sum1, sum0, sum1, p0, p1);
                 pk[c * 16 + (e >> 1)] = pack_bf16x2(p0, p1);
               }
-            l += sum;
-            tmem_st32(tS + lane_off + ch * 32, pk);  // packed columns [32*ch, 32*ch + 32) = score columns [64*ch, +64)
+            l += sum0 + sum1;
+            // packed columns [64*ch, 64*ch + 32) = score columns [64*ch, 64*ch + 64): inside this thread's own
+            // columns, so no other thread's unread scores are overwritten
+            tmem_st32(tS + lane_off + ch * 64, pk);
             if (rl == 0 && ch == 0) NSP_FTRACE(8 + 8 * x);
             // rescale this thread's 64 columns of O in place when some row of the warp moved its reference
             // maximum; the previous PV product of this half must have completed first (the next one is not
-            // issued before p_ready). The next exchange must not overwrite a slot the partner has not read yet:
-            // both threads of a pair pass the barrier of the NEXT tile only after this tile's read, which is
-            // ordered before their next write by the barrier itself (write -> arrive ... wait -> read; the next
-            // write of a slot follows the partner's next arrive only through bar_s_full, i.e. after p_ready).
+            // issued before p_ready).
             if (j > 0 && __any_sync(0xffffffffu, need)) {
               ok = mbar_wait(&s.bar_pv_done[x], (pvn + j - 1) & 1);
               ok = __all_sync(0xffffffffu, ok);
@@ -400,6 +421,15 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             tc_fence_before_sync();
             mbar_arrive(&s.bar_p_ready[x]);
             if (rl == 0 && ch == 0) NSP_FTRACE(9 + 8 * x);
+            if (j > 0 && !last) {
+              // post this tile's half-row maximum for the next tile. Slot by tile parity: the partner reads slot
+              // j & 1 at the start of tile j + 1, and this thread writes it again only at the end of tile j + 2,
+              // which it cannot reach before the partner has handed over P of tile j + 1.
+              mx_posted = mx_tile;
+              my_slot[128 * (j & 1)] = mx_tile;
+              mbar_arrive(pair_bar);
+              pending = true;
+            }
           }
           if (ok) {
             ok = mbar_wait(&s.bar_pv_done[x], (pvn + n_kv - 1) & 1);
@@ -408,7 +438,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           }
           pvn += n_kv;
           if (ok) {  // row sum = sum of the two half rows
-            *my_slot = l;
+            my_slot[256] = l;
             mbar_arrive(pair_bar);
             ok = mbar_wait(pair_bar, xn & 1);
             ++xn;
@@ -417,7 +447,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           }
           if (ok) {
             // ---- epilogue: O / l -> bf16 (this thread's 64 columns), LSE
-            l += *partner_slot;
+            l += partner_slot[256];
             tc_fence_after_sync();
             const int row = q_row0 + rl;
             const bool valid = row < sg.len;
