@@ -551,70 +551,82 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           // ---- common step (interior tile). Phase 1: P^T = exp2(S^T * c - LSE) for this thread's 64 query
           // columns, bf16 pairs over the S^T columns already read. The dV product needs only P^T, so it is
           // released to the MMA thread before dS^T is formed.
-          uint32_t pv[2][32];
-          tmem_ld32(tS, pv[0]);
-          tmem_ld32(tS + 32, pv[1]);
+          // Sixteen columns at a time; the LSE (delta) values of the next sixteen are requested before the
+          // arithmetic of the current ones, because a shared-memory load takes a long time here: the LSU is
+          // shared with the 64 KB of dQ reductions per step.
+          uint32_t sv[2][32];
+          float4 aux[2][4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) aux[0][i] = lds128(lse_s + 4 * i);
+          tmem_ld32(tS, sv[0]);
+          tmem_ld32(tS + 32, sv[1]);
           tmem_wait_ld();
           if (tid == 0) NSP_TRACE_STAMP(6);
+          uint32_t pp[2][16];  // P^T as bf16 pairs: what goes to R0, and what the dS^T product uses below
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            uint32_t pp[16];
+          for (int ch = 0; ch < 4; ++ch) {
+            if (ch < 3) {
 #pragma unroll
-            for (int x = 0; x < 32; x += 4) {
-              const float4 l4 = *reinterpret_cast<const float4*>(lse_s + cc * 32 + x);
-              float x0, x1, x2, x3;
-              fma2(x0, x1, __uint_as_float(pv[cc][x + 0]), __uint_as_float(pv[cc][x + 1]), a.scale_log2, a.scale_log2,
-                   -l4.x, -l4.y);
-              fma2(x2, x3, __uint_as_float(pv[cc][x + 2]), __uint_as_float(pv[cc][x + 3]), a.scale_log2, a.scale_log2,
-                   -l4.z, -l4.w);
-              const float p0 = ex2f(x0), p1 = ex2f(x1), p2 = ex2f(x2), p3 = ex2f(x3);
-              pv[cc][x + 0] = __float_as_uint(p0);
-              pv[cc][x + 1] = __float_as_uint(p1);
-              pv[cc][x + 2] = __float_as_uint(p2);
-              pv[cc][x + 3] = __float_as_uint(p3);
-              pp[(x >> 1) + 0] = pack_bf16x2(p0, p1);
-              pp[(x >> 1) + 1] = pack_bf16x2(p2, p3);
+              for (int i = 0; i < 4; ++i) aux[(ch + 1) & 1][i] = lds128(lse_s + (ch + 1) * 16 + 4 * i);
             }
-            tmem_st16(tS + cc * 32, pp);  // query columns [32cc, 32cc + 32) -> packed columns [32cc, 32cc + 16)
-            if (tid == 0) NSP_TRACE_STAMP(16 + cc);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float4 l4 = aux[ch & 1][i];
+              const int x = (ch & 1) * 16 + 4 * i;  // column inside the 32-column group ch / 2
+              float x0, x1, x2, x3;
+              fma2(x0, x1, __uint_as_float(sv[ch >> 1][x + 0]), __uint_as_float(sv[ch >> 1][x + 1]), a.scale_log2,
+                   a.scale_log2, -l4.x, -l4.y);
+              fma2(x2, x3, __uint_as_float(sv[ch >> 1][x + 2]), __uint_as_float(sv[ch >> 1][x + 3]), a.scale_log2,
+                   a.scale_log2, -l4.z, -l4.w);
+              pp[ch >> 1][(x >> 1) + 0] = pack_bf16x2(ex2f(x0), ex2f(x1));
+              pp[ch >> 1][(x >> 1) + 1] = pack_bf16x2(ex2f(x2), ex2f(x3));
+            }
+            if (ch & 1) tmem_st16(tS + (ch >> 1) * 32, pp[ch >> 1]);  // columns [32g, 32g + 32) -> packed [32g, +16)
+            if (tid == 0) NSP_TRACE_STAMP(16 + (ch >> 1));
           }
           tmem_wait_st();
           if (tid == 0) NSP_TRACE_STAMP(18);
           tc_fence_before_sync();
           mbar_arrive(&s.bar_p_ready);
           if (tid == 0) NSP_TRACE_STAMP(7);
-          // Phase 2: dS^T = P^T o (dP^T - delta) -> swizzled shared memory. The dS buffer is free: dP^T of this
-          // step was issued behind dK / dQ^T of the previous step, so bar_dp_full implies they have completed.
+          // Phase 2: dS^T = P^T o (dP^T - delta) -> swizzled shared memory; P enters with its bf16 value, the one
+          // the dV product uses. The dS buffer is free: dP^T of this step was issued behind dK / dQ^T of the
+          // previous step, so bar_dp_full implies they have completed.
+#pragma unroll
+          for (int i = 0; i < 4; ++i) aux[0][i] = lds128(delta_s + 4 * i);
           oks = mbar_wait(&s.bar_dp_full, cs & 1);
           oks = __all_sync(0xffffffffu, oks);
           if (!oks) { where = kWhereBwdDp; break; }
           tc_fence_after_sync();
           if (tid == 0) NSP_TRACE_STAMP(8);
+          uint32_t dpv[2][16];
+          tmem_ld16(tDP, dpv[0]);
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            uint32_t dpv[32], dsp[16];
-            tmem_ld32(tDP + cc * 32, dpv);
+          for (int ch = 0; ch < 4; ++ch) {
             tmem_wait_ld();
-            if (tid == 0) NSP_TRACE_STAMP(19 + 2 * cc);
+            if (ch < 3) {
+              tmem_ld16(tDP + (ch + 1) * 16, dpv[(ch + 1) & 1]);
 #pragma unroll
-            for (int x = 0; x < 32; x += 4) {
-              const float4 d4 = *reinterpret_cast<const float4*>(delta_s + cc * 32 + x);
+              for (int i = 0; i < 4; ++i) aux[(ch + 1) & 1][i] = lds128(delta_s + (ch + 1) * 16 + 4 * i);
+            }
+            if (tid == 0) NSP_TRACE_STAMP(19 + ch);
+            uint32_t dsp[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float4 d4 = aux[ch & 1][i];
+              const int x = 4 * i;
+              const uint32_t pa = pp[ch >> 1][(ch & 1) * 8 + (x >> 1)], pb = pp[ch >> 1][(ch & 1) * 8 + (x >> 1) + 1];
               float d0, d1, d2, d3;
-              sub2(d0, d1, __uint_as_float(dpv[x + 0]), __uint_as_float(dpv[x + 1]), d4.x, d4.y);
-              sub2(d2, d3, __uint_as_float(dpv[x + 2]), __uint_as_float(dpv[x + 3]), d4.z, d4.w);
-              mul2(d0, d1, d0, d1, __uint_as_float(pv[cc][x + 0]), __uint_as_float(pv[cc][x + 1]));
-              mul2(d2, d3, d2, d3, __uint_as_float(pv[cc][x + 2]), __uint_as_float(pv[cc][x + 3]));
+              sub2(d0, d1, __uint_as_float(dpv[ch & 1][x + 0]), __uint_as_float(dpv[ch & 1][x + 1]), d4.x, d4.y);
+              sub2(d2, d3, __uint_as_float(dpv[ch & 1][x + 2]), __uint_as_float(dpv[ch & 1][x + 3]), d4.z, d4.w);
+              mul2(d0, d1, d0, d1, __uint_as_float(pa << 16), __uint_as_float(pa & 0xffff0000u));
+              mul2(d2, d3, d2, d3, __uint_as_float(pb << 16), __uint_as_float(pb & 0xffff0000u));
               dsp[(x >> 1) + 0] = pack_bf16x2(d0, d1);
               dsp[(x >> 1) + 1] = pack_bf16x2(d2, d3);
             }
-            // dS^T row r, columns 32cc .. 32cc+31 of the half -> four 16-byte chunks of the swizzled row
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              const int chunk = (cc * 4 + ch) ^ (r & 7);
-              *reinterpret_cast<uint4*>(ds_row + chunk * 16) =
-                  make_uint4(dsp[ch * 4 + 0], dsp[ch * 4 + 1], dsp[ch * 4 + 2], dsp[ch * 4 + 3]);
-            }
-            if (tid == 0) NSP_TRACE_STAMP(20 + 2 * cc);
+            // sixteen query columns = two 16-byte chunks of the swizzled dS^T row
+            *reinterpret_cast<uint4*>(ds_row + ((2 * ch) ^ (r & 7)) * 16) = make_uint4(dsp[0], dsp[1], dsp[2], dsp[3]);
+            *reinterpret_cast<uint4*>(ds_row + ((2 * ch + 1) ^ (r & 7)) * 16) = make_uint4(dsp[4], dsp[5], dsp[6], dsp[7]);
           }
         } else {
           // ---- rare step (diagonal tile and/or one of the two first-tile passes): compact rolled loops, 16 query
