@@ -27,8 +27,8 @@
 // consecutive head-dimension values of one query row per register, and a plain red.global.add.f32 per register
 // is one fully coalesced 128-byte reduction into the fp32 accumulator. No shared-memory staging: shared-memory
 // bandwidth (MMA operand reads, TMA fills, dS^T) is a scarce resource of this kernel.
-// dK and dV accumulate in TMEM over the whole item in a fixed order (heads ascending, tiles ascending), so the
-// reduction over the query heads of a group is deterministic.
+// dK and dV accumulate in TMEM over the whole item in a fixed order (q tiles ascending, heads ascending inside
+// a tile), so the reduction over the query heads of a group is deterministic.
 // For the first q tile of a segment (rows 0..127, where P is O(1)) the step runs twice, once with the bf16
 // value of P and dS and once with the bf16 residual (hi + lo), and delta is recomputed in fp32 as
 // sum_j P_ij dP_ij instead of taking it from the bf16-rounded O; this keeps dK/dV/dQ inside the 2e-2 tolerance.
@@ -114,7 +114,9 @@ __device__ __forceinline__ void setmaxnreg_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
-// Walks the steps of an item: q heads of the group in ascending order, per head the q tiles in ascending order.
+// Walks the steps of an item: q tiles in ascending order, for every q tile the q heads of the group in ascending
+// order. With the heads innermost, CTAs that work on neighbouring key tiles stay one q tile apart for the whole
+// item, so the Q / dO tiles and the dQ accumulator rows they touch are still in L2 from their neighbour.
 // mode bit 0: recompute delta exactly; bit 1: residual (lo) pass of the hi/lo split.
 struct StepWalk {
   int hh, rr;
@@ -134,7 +136,7 @@ struct StepWalk {
     }
   }
   __device__ __forceinline__ void next(const ItemCtx& c) {
-    if (++rr == c.per_head) rr = 0, ++hh;
+    if (++hh == c.G) hh = 0, ++rr;
   }
 };
 
