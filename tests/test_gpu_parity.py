@@ -77,6 +77,32 @@ def test_scaled_down_twins_every_element(env, idx):
     _full_case(env, env["W"].config(idx, twin=True))
 
 
+def test_peaked_scores_exercise_the_rescale_path(env):
+    """Q and K three times larger than in the benchmark data: scores spread over +-40 in log2 units, so the running
+    maximum of a row keeps jumping by far more than the lazy-rescale threshold (2^8) from one key tile to the next.
+    This exercises what N(0,1) data hardly ever reaches: the in-place rescale of O, and tiles exponentiated against
+    a reference maximum that is one tile old (values of P far above 1). O and LSE keep the absolute tolerances.
+    The gradients are larger here and, with nearly one-hot P on every row, carry the error of delta = dO.O taken
+    from the bf16 O (the first-tile remedy of the kernel covers rows 0..127 only): they keep the relative-L2 bound,
+    and their max-abs bound is 1 % of max|ref|."""
+    W, P, torch = env["W"], env["P"], env["torch"]
+    w = W.custom([1536, 700, 300, 129], [4, 4, 8, 2], [1, 1, 2, 2], seed=9, name="peaked")
+    host = W.make_tensors(w)
+    host["q"] = (host["q"].float() * 3.0).to(torch.bfloat16)
+    host["k"] = (host["k"].float() * 3.0).to(torch.bfloat16)
+    run = P.GpuRun(w, tensors=host)
+    run.forward()
+    run.backward()
+    assert run.status()[0] == 0
+    res = run.results()
+    ref = P.oracle_full(w, run.host)
+    P.check("peaked:o", res["o"], ref["o"])
+    assert np.max(np.abs(res["lse"] - ref["lse"])) <= P.LSE_ABS_TOL * max(1.0, float(np.abs(ref["lse"]).max()) / 16)
+    for n in ("dq", "dk", "dv"):
+        ma, rl = P.check(f"peaked:{n}", res[n], ref[n], max_abs_tol=max(P.MAX_ABS_TOL, 1e-2 * float(np.abs(ref[n]).max())))
+        print(f"peaked:{n} max-abs {ma:.4g} (max|ref| {np.abs(ref[n]).max():.3g}) rel-L2 {rl:.3g}")
+
+
 def test_empty_and_degenerate_batches(env):
     B, W, P, torch = env["B"], env["W"], env["P"], env["torch"]
     # no segments at all
