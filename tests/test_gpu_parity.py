@@ -46,6 +46,11 @@ def test_tile_plan_bit_exact_full_size(env, idx):
         want = oracle.plan_tiles(w.cu_seqlens, w.hq, w.hkv, 128, 128, p)
         assert got.dtype == np.int32 and got.shape == want.shape
         assert np.array_equal(got, want)
+    # the order the backward kernel walks its items in is a permutation of the published backward list
+    exe = B.nsp_plan_get(plan, 2)
+    pub = B.nsp_plan_get(plan, 1)
+    key = lambda t: np.lexsort((t[:, 3], t[:, 2], t[:, 1], t[:, 0]))
+    assert exe.shape == pub.shape and np.array_equal(exe[key(exe)], pub[key(pub)])
     plan.destroy()
 
 
