@@ -33,9 +33,9 @@ from paper_2609_22755_b200 import workloads as W  # noqa: E402
 
 METRIC = "causal attention TFLOP/s fwd+bwd on 1 B200 and % of dense BF16 roofline"
 UNIT = "TFLOP/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one backward-main launch on the bench workload, from the ncu
-# capture summarised in profiles/bwd_kernel_nested_profile_case_64k.md (captured on a smaller case, scaled there).
-BWD_MAIN_DRAM_TRAFFIC_BYTES = int(6.373e9 * 5.0)  # 6.37 GB on the 64K profile case x 5.0 (ratio of Q elements)
+# dram__bytes_read.sum + dram__bytes_write.sum of one backward-main launch on the bench workload, from the
+# two-metric ncu capture summarised in profiles/bwd_kernel_nested_profile_case_64k.md.
+BWD_MAIN_DRAM_TRAFFIC_BYTES = int(36.02e9)  # measured on the bench workload itself (cfg4): 23.45 GB read + 12.57 GB written
 
 
 def measured_peaks():
