@@ -55,9 +55,13 @@ constexpr int kRegsSoftmax = 136, kRegsReduce = 80, kRegsAux = 48;
 // Optional step timeline (compiled in only with -DNSP_TRACE, for tuning): clock64 stamps of the first CTA's roles.
 #ifdef NSP_TRACE
 __device__ long long g_trace[64 * 24];
-#define NSP_TRACE_STAMP(slot)                                                                               \
-  do {                                                                                                      \
-    if (blockIdx.x == 0 && gi == 0 && vt >= 200 && vt < 264) g_trace[(vt - 200) * 24 + (slot)] = clock64(); \
+#ifndef NSP_TRACE_BASE
+#define NSP_TRACE_BASE 200
+#endif
+#define NSP_TRACE_STAMP(slot)                                                                  \
+  do {                                                                                         \
+    const uint32_t tix_ = gs + vt - NSP_TRACE_BASE;                                            \
+    if (blockIdx.x == 0 && tix_ < 64u) g_trace[tix_ * 24 + (slot)] = clock64();                \
   } while (0)
 #else
 #define NSP_TRACE_STAMP(slot)
@@ -646,24 +650,45 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           if (!oks) { where = kWhereBwdDp; break; }
           tc_fence_after_sync();
           const bool diag = (m == c.n);
+          if (tid == 0) NSP_TRACE_STAMP(6);
           if (mode & 1) {
             // delta_i = sum_j P_ij dP_ij over the keys of this tile (all keys of rows 0..127), fp32
             float* part = reinterpret_cast<float*>(s.ds[half]);  // [4 quadrants][64 columns]; free until dS is written
+            // Column sums over the 32 key rows of a warp by a butterfly: at every level a lane keeps the half of
+            // the columns its lane bit selects and adds the partner's partial sums of that half (16 shuffles for
+            // 16 columns); after the last level lane 2c (and 2c + 1) holds column c = lane / 2.
+            const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4, b1 = lane & 2;
 #pragma unroll 1
             for (int ch = 0; ch < 4; ++ch) {
               uint32_t sv[16], dpv[16];
+              float4 l4[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) l4[i] = lds128(lse_s + ch * 16 + 4 * i);
               tmem_ld16(tS + ch * 16, sv);
               tmem_ld16(tDP + ch * 16, dpv);
               tmem_wait_ld();
+              float v[16];
 #pragma unroll
               for (int x = 0; x < 16; ++x) {
-                float p = ex2f(fmaf(__uint_as_float(sv[x]), a.scale_log2, -lse_s[ch * 16 + x]));
+                const float lse_x = (x & 3) == 0 ? l4[x >> 2].x : (x & 3) == 1 ? l4[x >> 2].y
+                                  : (x & 3) == 2 ? l4[x >> 2].z : l4[x >> 2].w;
+                float p = ex2f(fmaf(__uint_as_float(sv[x]), a.scale_log2, -lse_x));
                 if (half * 64 + ch * 16 + x < r) p = 0.f;
-                float v = p * __uint_as_float(dpv[x]);
-#pragma unroll
-                for (int sft = 16; sft > 0; sft >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sft);
-                if (lane == 0) part[quad * 64 + ch * 16 + x] = v;
+                v[x] = p * __uint_as_float(dpv[x]);
               }
+              float w8[8], w4[4], w2[2];
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                w8[i] = (b4 ? v[i + 8] : v[i]) + __shfl_xor_sync(0xffffffffu, b4 ? v[i] : v[i + 8], 16);
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                w4[i] = (b3 ? w8[i + 4] : w8[i]) + __shfl_xor_sync(0xffffffffu, b3 ? w8[i] : w8[i + 4], 8);
+#pragma unroll
+              for (int i = 0; i < 2; ++i)
+                w2[i] = (b2 ? w4[i + 2] : w4[i]) + __shfl_xor_sync(0xffffffffu, b2 ? w4[i] : w4[i + 2], 4);
+              float w1 = (b1 ? w2[1] : w2[0]) + __shfl_xor_sync(0xffffffffu, b1 ? w2[0] : w2[1], 2);
+              w1 += __shfl_xor_sync(0xffffffffu, w1, 1);
+              if ((lane & 1) == 0) part[quad * 64 + ch * 16 + (lane >> 1)] = w1;
             }
             mbar_arrive(&s.bar_delta[half]);
             oks = mbar_wait(&s.bar_delta[half], nd & 1);
@@ -677,22 +702,31 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             oks = __all_sync(0xffffffffu, oks);
             if (!oks) { where = kWhereBwdDelta; break; }
           }
+          if (tid == 0) NSP_TRACE_STAMP(16);
 #pragma unroll 1
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t sv[16], dpv[16], pp[8], dsp[8];
+            float4 l4[4], e4[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              l4[i] = lds128(lse_s + ch * 16 + 4 * i);
+              e4[i] = lds128(delta_s + ch * 16 + 4 * i);
+            }
             tmem_ld16(tS + ch * 16, sv);
             tmem_ld16(tDP + ch * 16, dpv);
             tmem_wait_ld();
 #pragma unroll
             for (int x = 0; x < 16; x += 2) {
-              float p0 = ex2f(fmaf(__uint_as_float(sv[x + 0]), a.scale_log2, -lse_s[ch * 16 + x + 0]));
-              float p1 = ex2f(fmaf(__uint_as_float(sv[x + 1]), a.scale_log2, -lse_s[ch * 16 + x + 1]));
+              const float lse0 = (x & 2) ? l4[x >> 2].z : l4[x >> 2].x, lse1 = (x & 2) ? l4[x >> 2].w : l4[x >> 2].y;
+              const float del0 = (x & 2) ? e4[x >> 2].z : e4[x >> 2].x, del1 = (x & 2) ? e4[x >> 2].w : e4[x >> 2].y;
+              float p0 = ex2f(fmaf(__uint_as_float(sv[x + 0]), a.scale_log2, -lse0));
+              float p1 = ex2f(fmaf(__uint_as_float(sv[x + 1]), a.scale_log2, -lse1));
               if (diag) {  // query index must be >= key index
                 if (half * 64 + ch * 16 + x + 0 < r) p0 = 0.f;
                 if (half * 64 + ch * 16 + x + 1 < r) p1 = 0.f;
               }
-              const float d0 = p0 * (__uint_as_float(dpv[x + 0]) - delta_s[ch * 16 + x + 0]);
-              const float d1 = p1 * (__uint_as_float(dpv[x + 1]) - delta_s[ch * 16 + x + 1]);
+              const float d0 = p0 * (__uint_as_float(dpv[x + 0]) - del0);
+              const float d1 = p1 * (__uint_as_float(dpv[x + 1]) - del1);
               uint32_t pa = pack_bf16x2(p0, p1), da = pack_bf16x2(d0, d1);
               if (mode & 2) {  // residual pass: what the bf16 value left behind
                 pa = pack_bf16x2(p0 - __uint_as_float(pa << 16), p1 - __uint_as_float(pa & 0xffff0000u));
@@ -708,6 +742,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             *reinterpret_cast<uint4*>(ds_row + ((2 * ch + 1) ^ (r & 7)) * 16) = make_uint4(dsp[4], dsp[5], dsp[6], dsp[7]);
           }
           tmem_wait_st();
+          if (tid == 0) NSP_TRACE_STAMP(17);
           tc_fence_before_sync();
           mbar_arrive(&s.bar_p_ready);
         }
@@ -771,37 +806,64 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   if (warp == 0) tmem_dealloc(s.tmem_base, kBwdTmemCols);
 }
 
-// delta[h, i] = <dO[i,h,:], O[i,h,:]>; one warp per (token, head) row, rows in packed order.
-__global__ void bwd_preprocess_kernel(const SegInfo* __restrict__ seg, int n_seg, const int64_t* __restrict__ row_base,
-                                      int64_t total_rows, const __nv_bfloat16* __restrict__ o,
-                                      const __nv_bfloat16* __restrict__ d_o, float* __restrict__ delta) {
-  const int lane = threadIdx.x & 31;
-  const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-  if (row >= total_rows) return;
-  // row_base[s] = first packed row of segment s (ascending, row_base[n_seg] = total_rows)
-  int lo = 0, hi = n_seg - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (row_base[mid] <= row) lo = mid; else hi = mid - 1;
-  }
-  const SegInfo sg = seg[lo];
-  const int64_t rl = row - row_base[lo];
-  const int i = static_cast<int>(rl / sg.hq), h = static_cast<int>(rl % sg.hq);
-  const int64_t e = sg.q_off + rl * kHeadDim + lane * 4;
-  const uint2 a = *reinterpret_cast<const uint2*>(o + e);
-  const uint2 b = *reinterpret_cast<const uint2*>(d_o + e);
-  const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
-  const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
-  float acc = 0.f;
+// delta[h, i] = <dO[i,h,:], O[i,h,:]>. Rows (token, head) are packed one after the other, 256 bytes each, so the
+// kernel streams O and dO as flat arrays: a warp takes eight consecutive rows per pass, sixteen lanes per row with
+// one 16-byte load per tensor (eight loads in flight per thread), and only the index of the result needs the
+// segment table (delta is stored [head][token] inside a segment): lanes 0..7 look up one row each.
+__global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __restrict__ seg, int n_seg,
+                                                             const int64_t* __restrict__ row_base, int64_t total_rows,
+                                                             const __nv_bfloat16* __restrict__ o,
+                                                             const __nv_bfloat16* __restrict__ d_o,
+                                                             float* __restrict__ delta) {
+  const int lane = threadIdx.x & 31, sub = lane >> 4, l16 = lane & 15;
+  const int64_t n_groups = (total_rows + 7) >> 3;
+  const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+  for (int64_t grp = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; grp < n_groups; grp += n_warps) {
+    const int64_t row0 = grp * 8;
+    uint4 va[4], vb[4];
 #pragma unroll
-  for (int x = 0; x < 2; ++x) {
-    const float2 fa = __bfloat1622float2(pa[x]), fb = __bfloat1622float2(pb[x]);
-    acc = fmaf(fa.x, fb.x, acc);
-    acc = fmaf(fa.y, fb.y, acc);
-  }
+    for (int p = 0; p < 4; ++p) {
+      const int64_t row = row0 + 2 * p + sub;
+      if (row < total_rows) {
+        va[p] = __ldg(reinterpret_cast<const uint4*>(o + row * kHeadDim) + l16);
+        vb[p] = __ldg(reinterpret_cast<const uint4*>(d_o + row * kHeadDim) + l16);
+      } else {
+        va[p] = vb[p] = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+    // where the result of row row0 + (lane & 7) goes
+    int64_t dst = -1;
+    {
+      const int64_t row = row0 + (lane & 7);
+      if (row < total_rows) {
+        int lo = 0, hi = n_seg - 1;  // row_base[s] = first packed row of segment s (ascending)
+        while (lo < hi) {
+          const int mid = (lo + hi + 1) >> 1;
+          if (row_base[mid] <= row) lo = mid; else hi = mid - 1;
+        }
+        const SegInfo sg = seg[lo];
+        const int64_t rl = row - row_base[lo];
+        const int64_t i = rl / sg.hq, h = rl - i * sg.hq;
+        dst = sg.lse_off + h * sg.len + i;
+      }
+    }
 #pragma unroll
-  for (int sft = 16; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
-  if (lane == 0) delta[sg.lse_off + static_cast<int64_t>(h) * sg.len + i] = acc;
+    for (int p = 0; p < 4; ++p) {
+      const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&va[p]);
+      const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&vb[p]);
+      float acc = 0.f;
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const float2 fa = __bfloat1622float2(pa[x]), fb = __bfloat1622float2(pb[x]);
+        acc = fmaf(fa.x, fb.x, acc);
+        acc = fmaf(fa.y, fb.y, acc);
+      }
+#pragma unroll
+      for (int sft = 8; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+      const int64_t dst_p = __shfl_sync(0xffffffffu, dst, 2 * p + sub);
+      if (l16 == 0 && dst_p >= 0) delta[dst_p] = acc;
+    }
+  }
 }
 
 __global__ void bwd_postprocess_kernel(const float* __restrict__ acc, void* __restrict__ dq, int64_t n4, int dq_f32,
@@ -831,7 +893,8 @@ extern "C" int nsp_debug_trace_read(long long* host, int n) {
 cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
                                   const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, cudaStream_t st) {
   if (total_rows == 0) return cudaSuccess;
-  const int64_t blocks = (total_rows * 32 + 255) / 256;
+  int64_t blocks = ((total_rows + 7) / 8 * 32 + 255) / 256;  // one warp per eight rows, grid-stride beyond 16 waves
+  if (blocks > 148 * 8 * 16) blocks = 148 * 8 * 16;
   bwd_preprocess_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows, o, d_o,
                                                                        delta);
   count_launches(1);

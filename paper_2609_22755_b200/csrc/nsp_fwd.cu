@@ -39,6 +39,14 @@ __device__ long long g_ftrace[64 * 24];
 #define NSP_FTRACE(slot)
 #endif
 
+// One pop of the work list, decoded by thread 0 into shared memory (two slots: the next pop is fetched while the
+// current one runs).
+struct FwdPop {
+  SegInfo sa, sb;  // segments of items a and b
+  nsp_tile_t a, b;
+  int32_t it0, joint, n_rounds, pad_;
+};
+
 struct FwdSmem {
   uint8_t q[2][2][kHalfTileBytes];  // [A/B][64-column half]
   uint8_t k[2][2][kHalfTileBytes];  // [stage][half]
@@ -52,7 +60,7 @@ struct FwdSmem {
                              // (slot 2) handed to the partner thread
   uint64_t bar_pv_done[2];  // [A/B] O_x += P_x V has completed
   uint32_t tmem_base;
-  int32_t item_idx[2];
+  FwdPop pop[2];
   int32_t abort;
 };
 static_assert(sizeof(FwdSmem) <= 232448, "shared memory budget (227 KB)");
@@ -79,7 +87,6 @@ struct FwdRound {
   nsp_tile_t a, b;
   int joint;
 };
-
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   FwdSmem& s = *reinterpret_cast<FwdSmem*>(smem_raw);
@@ -118,21 +125,42 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   // ---- work decoding shared by all roles (every role runs its own copy of the loops, see the backward kernel)
   FwdRound rd;
   int n_rounds = 0, it0 = 0;
+  const FwdPop* pp = nullptr;
+  // Thread 0 only. The atomic on the cursor and the dependent loads of the items and their segments take about as
+  // long as a whole single-tile item, so after a short item they are done one pop ahead (after a long one the
+  // cursor is read when the item ends, which keeps the work list's balance at the end of the launch).
+  bool fetched_ahead = false;
+  auto fetch_pop = [&](FwdPop& p) {
+    const int it = atomicAdd(a.counter, 2);
+    p.it0 = it;
+    if (it < a.n_items) {
+      const bool have_b = it + 1 < a.n_items;
+      const nsp_tile_t ia = a.items[it];
+      const nsp_tile_t ib = have_b ? a.items[it + 1] : ia;
+      const SegInfo sa = a.seg[ia.seg];
+      p.a = ia, p.b = ib, p.sa = sa;
+      p.sb = ib.seg == ia.seg ? sa : a.seg[ib.seg];
+      const int G = sa.hq / sa.hkv;
+      p.joint = have_b && ib.seg == ia.seg && ib.tile == ia.tile && (ia.head / G == ib.head / G);
+      p.n_rounds = p.joint ? 1 : (have_b ? 2 : 1);
+    }
+  };
   auto next_pop = [&]() -> bool {
-    if (tid == 0) s.item_idx[gp & 1] = atomicAdd(a.counter, 2);
+    if (tid == 0 && !fetched_ahead) fetch_pop(s.pop[gp & 1]);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    it0 = s.item_idx[gp & 1];
+    pp = &s.pop[gp & 1];
+    it0 = pp->it0;
     ++gp;
     if (it0 >= a.n_items || *abort_flag) return false;
-    rd.a = a.items[it0];
-    const bool have_b = it0 + 1 < a.n_items;
-    rd.b = have_b ? a.items[it0 + 1] : rd.a;
-    const SegInfo sg = a.seg[rd.a.seg];
-    const int G = sg.hq / sg.hkv;
-    rd.joint = have_b && rd.b.seg == rd.a.seg && rd.b.tile == rd.a.tile && (rd.a.head / G == rd.b.head / G);
-    n_rounds = rd.joint ? 1 : (have_b ? 2 : 1);
+    rd.a = pp->a, rd.b = pp->b, rd.joint = pp->joint;
+    n_rounds = pp->n_rounds;
+    // the other slot held the previous pop: every role left it before it came to the barrier above
+    if (tid == 0) {
+      fetched_ahead = rd.a.cost <= 8;
+      if (fetched_ahead) fetch_pop(s.pop[gp & 1]);
+    }
     return true;
   };
   // end of a round: every warp has finished with the Q tiles, the K/V rings and the TMEM accumulators
@@ -151,7 +179,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
         for (int r = 0; r < n_rounds; ++r) {
           if (lane == 0 && !*abort_flag) {
             const nsp_tile_t ia = r == 0 ? rd.a : rd.b;
-            const SegInfo sg = a.seg[ia.seg];
+            const SegInfo sg = r == 0 ? pp->sa : pp->sb;
             const int g = ia.head / (sg.hq / sg.hkv);
             const int tok0 = sg.tok_in_run, q_row0 = ia.tile * kBM, n_kv = ia.cost;
             const CUtensorMap* mq = &maps.q[sg.run];
@@ -311,7 +339,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
         const bool active = (x == 0 || rd.joint) && !*abort_flag;
         if (active) {
           const nsp_tile_t ia = x == 0 ? (r == 0 ? rd.a : rd.b) : rd.b;
-          const SegInfo sg = a.seg[ia.seg];
+          const SegInfo sg = (x == 0 && r == 0) ? pp->sa : pp->sb;
           const int h = ia.head, n_kv = ia.cost, q_row0 = ia.tile * kBM;
           float m_ref = -INFINITY;  // reference maximum (log2 domain) the stored P and l are relative to
           float l = 0.f;            // running sum of exp2(s - m_ref) over this thread's columns
