@@ -144,6 +144,36 @@ int nsp_attn_bwd_static(const nsp_plan_t* plan, const void* q, const void* k, co
                         const void* d_o, const float* lse, void* dq, void* dk, void* dv, int dq_dtype, int dkv_dtype,
                         float softmax_scale, void* stream);
 
+/*
+ * Tree-level recomputation (paper Sec. 4.2, "Tree-Level Recomputation"): the backward pass of a shard in which the
+ * attention output of some segments was not kept after the forward pass.
+ *
+ * nsp_recompute_mark derives the save / recompute marking of this GPU's segments from an activation budget, the way
+ * the paper's executor walks its tree: segments (cu_seqlens [n_seg + 1], hq [n_seg], as for nsp_plan_tiles; all
+ * host) are visited from the upper levels down (level[s], host, larger =
+ * closer to the root, e.g. the SP degree of the segment's node; inside a level the segment that is more expensive to
+ * recompute first, cost = hq * L(L+1)/2), the bytes a saved segment keeps alive (its O slice in bf16 and its LSE in
+ * fp32: L * hq * (2 * head_dim + 4)) are accumulated, and from the first segment that no longer fits under
+ * budget_bytes on, everything is marked for recomputation. recompute (host, [n_seg], written): 0 = save,
+ * 1 = recompute. saved_bytes (may be NULL): bytes of the saved segments. Host-only, no CUDA call.
+ * Errors: INVALID_ARG (null pointer, negative size or budget, decreasing cu_seqlens, hq <= 0).
+ *
+ * nsp_attn_bwd_recompute is nsp_attn_bwd with such a marking (recompute: host, [n_seg]; if it is pinned memory it
+ * must stay unchanged until the stream has passed the call). For a marked segment the contents of o and lse are
+ * never read: a forward launch restricted to the marked segments recomputes their LSE and forms
+ * delta = rowsum(dO o O) from the accumulator in the same kernel, so the recomputed O never travels to memory; for
+ * the other segments o and lse are used as in nsp_attn_bwd. Outputs as nsp_attn_bwd. ws: at least
+ * nsp_plan_recompute_ws_bytes (the backward workspace plus an LSE copy and the flags), 256-byte aligned.
+ * Errors: as nsp_attn_bwd.
+ */
+int nsp_recompute_mark(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* level, int32_t n_seg,
+                       int32_t head_dim, int64_t budget_bytes, uint8_t* recompute, int64_t* saved_bytes);
+int nsp_plan_recompute_ws_bytes(const nsp_plan_t* plan, size_t* bytes);
+int nsp_attn_bwd_recompute(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, const void* k,
+                           const void* v, const void* o, const void* d_o, const float* lse, void* dq, void* dk,
+                           void* dv, int dq_dtype, int dkv_dtype, float softmax_scale, void* ws, size_t ws_bytes,
+                           void* stream);
+
 /* Read the sticky device status {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
 int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
 

@@ -1,8 +1,9 @@
 """TEST INFRASTRUCTURE: ctypes front-end of the fp64 CPU oracle (``nsp_oracle.c``).
 
 Only tests, the smoke check and the benchmark's CPU-baseline / reference legs import this package. It never
-imports the CUDA package and shares nothing with it. All arithmetic lives in the C file; this module only
-compiles it with gcc, marshals numpy arrays and reshapes results.
+imports the CUDA package and shares nothing with it. The attention and tile-plan arithmetic lives in the C file;
+this module compiles it with gcc, marshals numpy arrays and reshapes results. The one function written here in
+plain Python loops is ``recompute_mark`` (the save / recompute walk of the paper's tree-level recomputation).
 
 Conventions (identical to the C file header): packed ragged token-major tensors, bf16 inputs passed as
 ``uint16`` bit patterns (or ``float64`` arrays for finite-difference checks), float64 outputs.
@@ -157,3 +158,30 @@ def plan_tiles(cu, hq, hkv, bm=128, bn=128, pass_=0):
                             ctypes.c_int(pass_), _p(out), ctypes.c_int64(n.value), ctypes.byref(n))
     _check(rc, "plan_tiles")
     return out[: n.value]
+
+
+def recompute_mark(lengths, hq, level, budget_bytes, head_dim=128):
+    """Save / recompute marking of one GPU's segments (paper Sec. 4.2, "Tree-Level Recomputation"): walk the tree
+    from the upper levels toward the leaves, add up the bytes of the attention-output slices that are saved, and
+    once the budget is reached mark everything that is left for recomputation; inside the level where the cut
+    falls, the samples that cost more to recompute are saved first.
+
+    lengths, hq, level: one entry per segment (level: larger = closer to the root). A saved segment keeps its O
+    slice (2 bytes per element) and its LSE (4 bytes per row) alive; its recomputation cost is hq * L(L+1)/2.
+    Returns (flags, saved_bytes): flags[s] = 1 for recompute, 0 for save. Ties keep the segment order."""
+    n = len(lengths)
+    visit = []
+    for lv in sorted(set(int(x) for x in level), reverse=True):  # root first
+        members = [s for s in range(n) if int(level[s]) == lv]
+        # inside a level: larger recomputation cost first; Python's sort is stable, so ties keep their order
+        members.sort(key=lambda s: -(int(hq[s]) * (int(lengths[s]) * (int(lengths[s]) + 1) // 2)))
+        visit += members
+    flags = [1] * n
+    used = 0
+    for s in visit:
+        need = int(lengths[s]) * int(hq[s]) * (2 * head_dim + 4)
+        if used + need > budget_bytes:
+            break  # the budget is reached: this segment and all later ones are recomputed
+        used += need
+        flags[s] = 0
+    return np.asarray(flags, dtype=np.uint8), used

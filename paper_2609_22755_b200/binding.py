@@ -25,7 +25,7 @@ NSP_MAX_RUNS = 32
 EXPORTS = [
     "nsp_plan_tiles", "nsp_plan_sizes", "nsp_plan_get", "nsp_attn_fwd", "nsp_attn_bwd", "nsp_device_status",
     "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string", "nsp_plan_set_profiling", "nsp_plan_kernel_ms",
-    "nsp_attn_bwd_static",
+    "nsp_attn_bwd_static", "nsp_recompute_mark", "nsp_plan_recompute_ws_bytes", "nsp_attn_bwd_recompute",
 ]
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
 KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST = 0, 1, 2, 3
@@ -70,6 +70,13 @@ def lib() -> ctypes.CDLL:
         L.nsp_attn_bwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_float, vp]
         L.nsp_attn_bwd_static.restype = ctypes.c_int
+        L.nsp_recompute_mark.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, vp, i64p]
+        L.nsp_recompute_mark.restype = ctypes.c_int
+        L.nsp_plan_recompute_ws_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+        L.nsp_plan_recompute_ws_bytes.restype = ctypes.c_int
+        L.nsp_attn_bwd_recompute.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int,
+                                             ctypes.c_float, vp, ctypes.c_size_t, vp]
+        L.nsp_attn_bwd_recompute.restype = ctypes.c_int
         L.nsp_device_status.argtypes = [vp, i32p]
         L.nsp_device_status.restype = ctypes.c_int
         L.nsp_launch_count.argtypes = []
@@ -197,6 +204,56 @@ def nsp_attn_bwd(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, softmax_scale, ws
                             _stream_ptr(stream))
     if rc != NSP_OK:
         raise NspError(rc, "nsp_attn_bwd")
+
+
+def nsp_recompute_mark(cu_seqlens, hq, level, budget_bytes: int, head_dim: int = 128):
+    """Save / recompute marking of a shard's segments under an activation budget (host only); returns
+    (flags uint8 [n_seg], bytes of the saved segments)."""
+    import numpy as np
+
+    cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    hq = np.ascontiguousarray(hq, dtype=np.int32)
+    level = np.ascontiguousarray(level, dtype=np.int32)
+    n = len(hq)
+    if cu.shape != (n + 1,) or level.shape != (n,):
+        raise ValueError("cu_seqlens needs n_seg + 1 entries, hq and level n_seg")
+    flags = np.zeros(max(n, 1), dtype=np.uint8)
+    saved = ctypes.c_int64()
+    vp = ctypes.c_void_p
+    rc = lib().nsp_recompute_mark(cu.ctypes.data_as(vp), hq.ctypes.data_as(vp), level.ctypes.data_as(vp), n,
+                                  int(head_dim), int(budget_bytes), flags.ctypes.data_as(vp), ctypes.byref(saved))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_recompute_mark")
+    return flags[:n], int(saved.value)
+
+
+def nsp_plan_recompute_ws_bytes(plan: Plan) -> int:
+    n = ctypes.c_size_t()
+    rc = lib().nsp_plan_recompute_ws_bytes(plan.handle, ctypes.byref(n))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_plan_recompute_ws_bytes")
+    return int(n.value)
+
+
+def nsp_attn_bwd_recompute(plan: Plan, recompute, q, k, v, o, d_o, lse, dq, dk, dv, softmax_scale, ws, dq_dtype=None,
+                           dkv_dtype=None, stream=None):
+    """nsp_attn_bwd with per-segment flags (uint8 [n_seg], host): o and lse of a flagged segment are never read."""
+    import numpy as np
+    import torch
+
+    recompute = np.ascontiguousarray(recompute, dtype=np.uint8)
+    if recompute.shape != (plan.n_seg,):
+        raise ValueError("recompute must have one entry per segment")
+    if dq_dtype is None:
+        dq_dtype = NSP_F32 if dq.dtype == torch.float32 else NSP_BF16
+    if dkv_dtype is None:
+        dkv_dtype = NSP_F32 if dk.dtype == torch.float32 else NSP_BF16
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    rc = lib().nsp_attn_bwd_recompute(plan.handle, recompute.ctypes.data_as(ctypes.c_void_p), _ptr(q), _ptr(k), _ptr(v),
+                                      _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv), dq_dtype, dkv_dtype,
+                                      float(softmax_scale), _ptr(ws), ws_bytes, _stream_ptr(stream))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_attn_bwd_recompute")
 
 
 def nsp_device_status(plan: Plan):

@@ -369,15 +369,28 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  a.seg_mask = nullptr;
+  a.d_o = nullptr;
+  a.delta = nullptr;
   prof_mark(plan, NSP_KERNEL_FWD, 0, st);
   if (launch_fwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_FWD, 1, st);
   return NSP_OK;
 }
 
-int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const void* v, const void* o, const void* d_o,
-                 const float* lse, void* dq, void* dk, void* dv, int dq_dtype, int dkv_dtype, float softmax_scale,
-                 void* ws, size_t ws_bytes, void* stream) {
+namespace {
+
+size_t recompute_ws_bytes(const nsp_plan_t* plan) {
+  size_t base = 0;
+  nsp_plan_sizes(plan, nullptr, nullptr, nullptr, nullptr, &base);
+  return base + align_up(static_cast<size_t>(plan->lse_elems) * 4, 256) + align_up(static_cast<size_t>(plan->n_seg), 256);
+}
+
+// Backward pass. recompute == nullptr: the plain pass. Otherwise host flags per segment: for a marked segment o and
+// lse are not read; its LSE and delta are recomputed by a forward launch restricted to the marked segments.
+int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, const void* k, const void* v,
+             const void* o, const void* d_o, const float* lse, void* dq, void* dk, void* dv, int dq_dtype,
+             int dkv_dtype, float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
   if (!plan) return NSP_ERR_INVALID_ARG;
   if (plan->sticky) return plan->sticky;
   if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return NSP_ERR_INVALID_ARG;
@@ -388,15 +401,21 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
       !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
     return NSP_ERR_INVALID_ARG;
-  size_t need = 0;
-  nsp_plan_sizes(plan, nullptr, nullptr, nullptr, nullptr, &need);
+  size_t base = 0;
+  nsp_plan_sizes(plan, nullptr, nullptr, nullptr, nullptr, &base);
+  const size_t need = recompute ? recompute_ws_bytes(plan) : base;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < need) return NSP_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* wsb = static_cast<char*>(ws);
   float* dq_acc = static_cast<float*>(ws);
-  float* delta = reinterpret_cast<float*>(static_cast<char*>(ws) + align_up(static_cast<size_t>(plan->q_elems) * 4, 256));
+  float* delta = reinterpret_cast<float*>(wsb + align_up(static_cast<size_t>(plan->q_elems) * 4, 256));
+  float* lse_ws = reinterpret_cast<float*>(wsb + base);
+  uint8_t* d_mask = reinterpret_cast<uint8_t*>(wsb + base + align_up(static_cast<size_t>(plan->lse_elems) * 4, 256));
 
   BwdMaps maps;
   std::memset(&maps, 0, sizeof(maps));
+  FwdMaps fmaps;
+  if (recompute) std::memset(&fmaps, 0, sizeof(fmaps));
   for (size_t r = 0; r < plan->runs.size(); ++r) {
     const RunInfo& run = plan->runs[r];
     if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq) ||
@@ -404,12 +423,36 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
         !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv) ||
         !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv))
       return NSP_ERR_CUDA;
+    if (recompute) fmaps.q[r] = maps.q[r], fmaps.k[r] = maps.k[r], fmaps.v[r] = maps.v[r];
   }
   if (cudaMemsetAsync(plan->d_counters + 1, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
   if (cudaMemsetAsync(dq_acc, 0, static_cast<size_t>(plan->q_elems) * 4, st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (recompute) {
+    // from pageable memory the runtime stages the flags before it returns; a pinned array must stay unchanged until
+    // the stream has passed this copy
+    if (cudaMemcpyAsync(d_mask, recompute, static_cast<size_t>(plan->n_seg), cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return NSP_ERR_CUDA;
+    if (cudaMemsetAsync(plan->d_counters, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
+    FwdArgs fa;
+    fa.seg = plan->d_seg;
+    fa.items = plan->d_fwd;
+    fa.n_items = static_cast<int32_t>(plan->n_fwd);
+    fa.counter = plan->d_counters;
+    fa.status = plan->d_status;
+    fa.o = nullptr;
+    fa.lse = lse_ws;
+    fa.scale_log2 = softmax_scale * 1.4426950408889634f;
+    fa.seg_mask = d_mask;
+    fa.d_o = static_cast<const __nv_bfloat16*>(d_o);
+    fa.delta = delta;
+    prof_mark(plan, NSP_KERNEL_FWD, 0, st);
+    if (launch_fwd(fmaps, fa, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+    prof_mark(plan, NSP_KERNEL_FWD, 1, st);
+  }
   prof_mark(plan, NSP_KERNEL_BWD_PRE, 0, st);
   if (launch_bwd_preprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems,
                             static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta,
+                            recompute ? d_mask : nullptr, recompute ? lse : nullptr, recompute ? lse_ws : nullptr,
                             st) != cudaSuccess)
     return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_PRE, 1, st);
@@ -419,7 +462,7 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.n_items = static_cast<int32_t>(plan->n_bwd);
   a.counter = plan->d_counters + 1;
   a.status = plan->d_status;
-  a.lse = lse;
+  a.lse = recompute ? lse_ws : lse;
   a.delta = delta;
   a.dq_acc = dq_acc;
   a.dk = dk;
@@ -438,6 +481,62 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   if (launch_bwd_postprocess(dq_acc, dq, plan->q_elems, dq_dtype == NSP_F32, softmax_scale, st) != cudaSuccess)
     return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_POST, 1, st);
+  return NSP_OK;
+}
+
+}  // namespace
+
+int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                 const float* lse, void* dq, void* dk, void* dv, int dq_dtype, int dkv_dtype, float softmax_scale,
+                 void* ws, size_t ws_bytes, void* stream) {
+  return bwd_impl(plan, nullptr, q, k, v, o, d_o, lse, dq, dk, dv, dq_dtype, dkv_dtype, softmax_scale, ws, ws_bytes,
+                  stream);
+}
+
+int nsp_plan_recompute_ws_bytes(const nsp_plan_t* plan, size_t* bytes) {
+  if (!plan || !bytes) return NSP_ERR_INVALID_ARG;
+  *bytes = recompute_ws_bytes(plan);
+  return NSP_OK;
+}
+
+int nsp_attn_bwd_recompute(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, const void* k,
+                           const void* v, const void* o, const void* d_o, const float* lse, void* dq, void* dk,
+                           void* dv, int dq_dtype, int dkv_dtype, float softmax_scale, void* ws, size_t ws_bytes,
+                           void* stream) {
+  if (!plan || !recompute) return NSP_ERR_INVALID_ARG;
+  return bwd_impl(plan, recompute, q, k, v, o, d_o, lse, dq, dk, dv, dq_dtype, dkv_dtype, softmax_scale, ws, ws_bytes,
+                  stream);
+}
+
+int nsp_recompute_mark(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* level, int32_t n_seg,
+                       int32_t head_dim, int64_t budget_bytes, uint8_t* recompute, int64_t* saved_bytes) {
+  if (n_seg < 0 || head_dim <= 0 || budget_bytes < 0) return NSP_ERR_INVALID_ARG;
+  if (n_seg > 0 && (!cu_seqlens || !hq || !level || !recompute)) return NSP_ERR_INVALID_ARG;
+  for (int s = 0; s < n_seg; ++s)
+    if (cu_seqlens[s + 1] < cu_seqlens[s] || hq[s] <= 0) return NSP_ERR_INVALID_ARG;
+  std::vector<int> order(n_seg);
+  for (int s = 0; s < n_seg; ++s) order[s] = s;
+  auto len = [&](int s) { return static_cast<int64_t>(cu_seqlens[s + 1]) - cu_seqlens[s]; };
+  // recomputation cost of a segment: its causal (query, key) pairs times its query heads
+  auto cost = [&](int s) { return static_cast<int64_t>(hq[s]) * (len(s) * (len(s) + 1) / 2); };
+  std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
+    if (level[x] != level[y]) return level[x] > level[y];
+    return cost(x) > cost(y);
+  });
+  int64_t used = 0;
+  bool cut = false;
+  for (int s : order) {
+    // what saving the segment keeps alive: its slice of O (bf16) and of the LSE (fp32)
+    const int64_t bytes = len(s) * hq[s] * (static_cast<int64_t>(head_dim) * 2 + 4);
+    if (!cut && used + bytes <= budget_bytes) {
+      used += bytes;
+      recompute[s] = 0;
+    } else {
+      cut = true;
+      recompute[s] = 1;
+    }
+  }
+  if (saved_bytes) *saved_bytes = used;
   return NSP_OK;
 }
 

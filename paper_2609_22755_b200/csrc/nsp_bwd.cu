@@ -810,11 +810,16 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
 // kernel streams O and dO as flat arrays: a warp takes eight consecutive rows per pass, sixteen lanes per row with
 // one 16-byte load per tensor (eight loads in flight per thread), and only the index of the result needs the
 // segment table (delta is stored [head][token] inside a segment): lanes 0..7 look up one row each.
+// With seg_skip, the rows of marked segments are read but nothing is written for them; with lse_out, the LSE of every
+// row that is processed is copied from lse_in (same index as delta).
 __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __restrict__ seg, int n_seg,
                                                              const int64_t* __restrict__ row_base, int64_t total_rows,
                                                              const __nv_bfloat16* __restrict__ o,
                                                              const __nv_bfloat16* __restrict__ d_o,
-                                                             float* __restrict__ delta) {
+                                                             float* __restrict__ delta,
+                                                             const uint8_t* __restrict__ seg_skip,
+                                                             const float* __restrict__ lse_in,
+                                                             float* __restrict__ lse_out) {
   const int lane = threadIdx.x & 31, sub = lane >> 4, l16 = lane & 15;
   const int64_t n_groups = (total_rows + 7) >> 3;
   const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
@@ -844,7 +849,11 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
         const SegInfo sg = seg[lo];
         const int64_t rl = row - row_base[lo];
         const int64_t i = rl / sg.hq, h = rl - i * sg.hq;
-        dst = sg.lse_off + h * sg.len + i;
+        // rows of a skipped segment (its delta and LSE come from the recomputation) are left alone
+        if (seg_skip == nullptr || seg_skip[lo] == 0) {
+          dst = sg.lse_off + h * sg.len + i;
+          if (lse_out != nullptr && lane < 8) lse_out[dst] = lse_in[dst];
+        }
       }
     }
 #pragma unroll
@@ -891,12 +900,13 @@ extern "C" int nsp_debug_trace_read(long long* host, int n) {
 #endif
 
 cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
-                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, cudaStream_t st) {
+                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta,
+                                  const uint8_t* seg_skip, const float* lse_in, float* lse_out, cudaStream_t st) {
   if (total_rows == 0) return cudaSuccess;
   int64_t blocks = ((total_rows + 7) / 8 * 32 + 255) / 256;  // one warp per eight rows, grid-stride beyond 16 waves
   if (blocks > 148 * 8 * 16) blocks = 148 * 8 * 16;
   bwd_preprocess_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows, o, d_o,
-                                                                       delta);
+                                                                       delta, seg_skip, lse_in, lse_out);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -56,7 +56,8 @@ struct FwdSmem {
   uint64_t bar_s_full[2];   // [A/B] S_x of a key tile is in TMEM
   uint64_t bar_p_ready[2];  // [A/B] 256 softmax threads: P_x written (and O_x rescaled if needed)
   uint64_t bar_pair[2][4];  // [A/B][lane quadrant] the two threads of every row have published their half-row value
-  float xchg[2][2][3][128];  // [A/B][column half][slot][row] half-row maximum (slots 0/1 by tile parity) or row sum
+  float xchg[2][2][4][128];  // [A/B][column half][slot][row] half-row maximum (slots 0/1 by tile parity), row sum (2),
+                             // half-row dot product of O and dO (3, recomputation only)
                              // (slot 2) handed to the partner thread
   uint64_t bar_pv_done[2];  // [A/B] O_x += P_x V has completed
   uint32_t tmem_base;
@@ -131,18 +132,26 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   // cursor is read when the item ends, which keeps the work list's balance at the end of the launch).
   bool fetched_ahead = false;
   auto fetch_pop = [&](FwdPop& p) {
-    const int it = atomicAdd(a.counter, 2);
-    p.it0 = it;
-    if (it < a.n_items) {
-      const bool have_b = it + 1 < a.n_items;
-      const nsp_tile_t ia = a.items[it];
-      const nsp_tile_t ib = have_b ? a.items[it + 1] : ia;
+    for (;;) {
+      const int it = atomicAdd(a.counter, 2);
+      p.it0 = it;
+      if (it >= a.n_items) break;
+      bool have_b = it + 1 < a.n_items;
+      nsp_tile_t ia = a.items[it];
+      nsp_tile_t ib = have_b ? a.items[it + 1] : ia;
+      if (a.seg_mask != nullptr) {  // recomputation: only the marked segments
+        const bool fa = a.seg_mask[ia.seg] != 0, fb = have_b && a.seg_mask[ib.seg] != 0;
+        if (!fa && !fb) continue;
+        if (!fa) ia = ib;
+        if (!fa || !fb) ib = ia, have_b = false;
+      }
       const SegInfo sa = a.seg[ia.seg];
       p.a = ia, p.b = ib, p.sa = sa;
       p.sb = ib.seg == ia.seg ? sa : a.seg[ib.seg];
       const int G = sa.hq / sa.hkv;
       p.joint = have_b && ib.seg == ia.seg && ib.tile == ia.tile && (ia.head / G == ib.head / G);
       p.n_rounds = p.joint ? 1 : (have_b ? 2 : 1);
+      break;
     }
   };
   auto next_pop = [&]() -> bool {
@@ -465,6 +474,55 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             if (!ok) where = kWhereFwdO;
           }
           pvn += n_kv;
+          const int row = q_row0 + rl;
+          const bool valid = row < sg.len;
+          if (ok && a.delta != nullptr) {
+            // ---- epilogue of a recomputation: LSE and delta = <dO, O> of the row, O itself is not written.
+            // The half-row dot product is taken with the unnormalised O and handed over together with the half-row
+            // sum.
+            tc_fence_after_sync();
+            const __nv_bfloat16* dptr =
+                a.d_o + sg.q_off + (static_cast<int64_t>(valid ? row : 0) * sg.hq + h) * kHeadDim + ch * 64;
+            float part = 0.f;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              uint32_t orow[32];
+              tmem_ld32(tO + lane_off + ch * 64 + c * 32, orow);
+              uint4 dv4[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) dv4[e] = __ldg(reinterpret_cast<const uint4*>(dptr + c * 32) + e);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t w[4] = {dv4[e].x, dv4[e].y, dv4[e].z, dv4[e].w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                  part = fmaf(__uint_as_float(orow[8 * e + 2 * t]), __uint_as_float(w[t] << 16), part);
+                  part = fmaf(__uint_as_float(orow[8 * e + 2 * t + 1]), __uint_as_float(w[t] & 0xffff0000u), part);
+                }
+              }
+            }
+            my_slot[256] = l;
+            my_slot[384] = part;
+            mbar_arrive(pair_bar);
+            ok = mbar_wait(pair_bar, xn & 1);
+            ++xn;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) where = kWhereFwdPair;
+            if (ok && valid && ch == 0) {
+              l += partner_slot[256];
+              part += partner_slot[384];
+              const int64_t at = sg.lse_off + static_cast<int64_t>(h) * sg.len + row;
+              a.lse[at] = (m_ref + log2f(l)) * 0.6931471805599453f;
+              a.delta[at] = part / l;
+            }
+            if (!ok && lane == 0) {
+              report_timeout(a.status, it0, where, 0);
+              *abort_flag = 1;
+            }
+            round_end();
+            continue;
+          }
           if (ok) {  // row sum = sum of the two half rows
             my_slot[256] = l;
             mbar_arrive(pair_bar);
@@ -477,8 +535,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             // ---- epilogue: O / l -> bf16 (this thread's 64 columns), LSE
             l += partner_slot[256];
             tc_fence_after_sync();
-            const int row = q_row0 + rl;
-            const bool valid = row < sg.len;
             const float inv_l = 1.f / l;
             __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim + ch * 64;
 #pragma unroll

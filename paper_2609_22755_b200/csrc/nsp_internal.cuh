@@ -82,6 +82,11 @@ struct FwdArgs {
   __nv_bfloat16* o;
   float* lse;
   float scale_log2;  // softmax_scale * log2(e)
+  // Recomputation inside the backward pass (all three null in a plain forward): only items of segments with
+  // seg_mask[seg] != 0 run, and instead of O the kernel writes delta = rowsum(dO o O) next to the LSE.
+  const uint8_t* seg_mask;
+  const __nv_bfloat16* d_o;
+  float* delta;
 };
 
 struct BwdArgs {
@@ -108,8 +113,11 @@ cudaError_t launch_plan_build(const SegInfo* d_seg, int n_seg, int bm, int bn, n
                               cudaStream_t st);
 size_t plan_sort_tmp_bytes(int64_t max_items);
 cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st);
+// seg_skip (may be null): segments whose rows are left alone; lse_in / lse_out (may be null): LSE copied for the rows
+// that are processed.
 cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
-                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, cudaStream_t st);
+                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta,
+                                  const uint8_t* seg_skip, const float* lse_in, float* lse_out, cudaStream_t st);
 cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st);
 cudaError_t launch_bwd_postprocess(const float* dq_acc, void* dq, int64_t n, int dq_f32, float scale, cudaStream_t st);
 void count_launches(int n);

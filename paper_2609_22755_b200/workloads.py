@@ -106,7 +106,7 @@ def _mk(name, lengths, hq, hkv, seed, note=""):
 
 
 def config(idx: int, seed: int | None = None, twin: bool = False) -> Workload:
-    """The five benchmark configurations (idx 1..5) or their scaled-down twins (same head structure,
+    """The five benchmark configurations (idx 1..5; idx 6 is the mixed-degree shard of `full_tree_shard`) or their scaled-down twins (same head structure,
     lengths divided by 16..32, sized so the fp64 oracle evaluates every element in seconds to a minute)."""
     if seed is None:
         seed = idx - 1
@@ -137,7 +137,26 @@ def config(idx: int, seed: int | None = None, twin: bool = False) -> Workload:
         short = lognormal_lengths(seed, 262144 - 131072, 4096, 1.0, 64, 65536)
         return _mk("cfg5_largehead_longtail", [131072] + short, [16] + [64] * len(short), [1] + [4] * len(short), seed,
                    "one 131,072-token segment at degree 4 (16q/1kv) + degree-1 tail (64q/4kv)")
-    raise ValueError("config index must be 1..5")
+    if idx == 6:
+        return full_tree_shard(seed, twin)
+    raise ValueError("config index must be 1..6")
+
+
+def full_tree_shard(seed: int = 5, twin: bool = False) -> Workload:
+    """One GPU's chain in a full binary SP tree over eight GPUs (paper Sec. 4.1, Def. 1) for a 32q/4kv model: the
+    root's segment at degree 8 (4q/1kv), two at degree 4 (8q/1kv), four at degree 2 (16q/2kv) and a long-tailed
+    degree-1 leaf batch (32q/4kv). Four runs with four different head counts in one shard. Not one of the five
+    benchmark configurations (index 6); the twin divides the lengths by 32."""
+    if twin:
+        leaf = lognormal_lengths(seed, 1024, 64, 1.2, 16, 512)
+        lens = [4096] + [1024, 528] + [256, 304, 128, 200] + leaf
+    else:
+        leaf = lognormal_lengths(seed, 16384, 1024, 1.2, 64, 8192)
+        lens = [131072] + [32768, 16400] + [8192, 9744, 4096, 6160] + leaf
+    hq = [4] + [8] * 2 + [16] * 4 + [32] * len(leaf)
+    hkv = [1] + [1] * 2 + [2] * 4 + [4] * len(leaf)
+    return _mk("full_tree_shard_twin" if twin else "full_tree_shard", lens, hq, hkv, seed,
+               "degrees 8 / 4 / 2 / 1 of a 32q/4kv model in one shard")
 
 
 def profile_case(seed: int = 3) -> Workload:

@@ -36,7 +36,7 @@ def _full_case(env, w, **kw):
     return P.compare_full(w, res, ref), run, res, ref
 
 
-@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5, 6])
 def test_tile_plan_bit_exact_full_size(env, idx):
     B, W, oracle = env["B"], env["W"], env["oracle"]
     w = W.config(idx)
@@ -77,7 +77,7 @@ def test_bf16_gradients_and_fp32_dq_variants(env):
         assert P.errors(res[n], ref[n])[1] <= P.REL_L2_TOL
 
 
-@pytest.mark.parametrize("idx", [2, 3, 4, 5])
+@pytest.mark.parametrize("idx", [2, 3, 4, 5, 6])
 def test_scaled_down_twins_every_element(env, idx):
     _full_case(env, env["W"].config(idx, twin=True))
 
@@ -106,6 +106,55 @@ def test_peaked_scores_exercise_the_rescale_path(env):
     for n in ("dq", "dk", "dv"):
         ma, rl = P.check(f"peaked:{n}", res[n], ref[n], max_abs_tol=max(P.MAX_ABS_TOL, 1e-2 * float(np.abs(ref[n]).max())))
         print(f"peaked:{n} max-abs {ma:.4g} (max|ref| {np.abs(ref[n]).max():.3g}) rel-L2 {rl:.3g}")
+
+
+@pytest.mark.parametrize("which", ["all", "budget", "alternate", "none"])
+@pytest.mark.parametrize("case", ["full_tree_twin", "ragged"])
+def test_backward_with_recomputation(env, case, which):
+    """Tree-level recomputation: for the flagged segments O and LSE are poisoned with NaN before the backward call,
+    which must recompute what it needs; the gradients are compared with the oracle element by element, and with the
+    plain backward of the same run."""
+    torch, P, B, W = env["torch"], env["P"], env["B"], env["W"]
+    w = W.config(6, twin=True) if case == "full_tree_twin" else W.ragged()
+    run = P.GpuRun(w)
+    run.forward()
+    run.backward()
+    plain = {n: getattr(run, n).clone() for n in ("dq", "dk", "dv")}
+    n = w.n_seg
+    if which == "all":
+        flags = np.ones(n, np.uint8)
+    elif which == "none":
+        flags = np.zeros(n, np.uint8)
+    elif which == "alternate":
+        flags = (np.arange(n) % 2).astype(np.uint8)
+    else:  # the marking of an activation budget that holds about half of the shard's attention output
+        total = int((w.lengths * w.hq).sum()) * (2 * w.head_dim + 4)
+        level = (w.hq.max() // w.hq).astype(np.int32)  # SP degree of the segment's node
+        flags, saved = B.nsp_recompute_mark(w.cu_seqlens, w.hq, level, total // 2)
+        assert 0 < saved <= total // 2 and 0 < flags.sum() < n
+    qo, lo = w.q_offsets(), w.lse_offsets()
+    o, lse = run.o.clone(), run.lse.clone()
+    for s in range(n):
+        if flags[s]:
+            o[qo[s]:qo[s + 1]] = float("nan")
+            lse[lo[s]:lo[s + 1]] = float("nan")
+    for t in (run.dq, run.dk, run.dv):
+        t.fill_(float("nan"))
+    ws = torch.empty(B.nsp_plan_recompute_ws_bytes(run.plan), dtype=torch.uint8, device=run.dev)
+    B.nsp_attn_bwd_recompute(run.plan, flags, run.q, run.k, run.v, o, run.do, lse, run.dq, run.dk, run.dv,
+                             w.softmax_scale, ws)
+    assert run.status()[0] == 0
+    res = run.results()
+    ref = P.oracle_full(w, run.host)
+    for name in ("dq", "dk", "dv"):
+        P.check(f"{w.name}:recompute[{which}]:{name}", res[name], ref[name])
+    if which == "none":  # nothing recomputed: the very same kernels on the very same inputs
+        for name in ("dk", "dv"):
+            assert torch.equal(getattr(run, name), plain[name])
+    # too small a workspace is refused
+    with pytest.raises(B.NspError):
+        B.nsp_attn_bwd_recompute(run.plan, flags, run.q, run.k, run.v, o, run.do, lse, run.dq, run.dk, run.dv,
+                                 w.softmax_scale, run.ws[:max(run.plan.bwd_ws_bytes - 256, 0)])
 
 
 def test_empty_and_degenerate_batches(env):
@@ -213,7 +262,7 @@ def _sample_rows(w, rng, per_seg):
     return rows
 
 
-@pytest.mark.parametrize("idx,per_seg,last_cols", [(2, 2, 32), (3, 3, 32), (4, 6, 48), (5, 3, 24)])
+@pytest.mark.parametrize("idx,per_seg,last_cols", [(2, 2, 32), (3, 3, 32), (4, 6, 48), (5, 3, 24), (6, 3, 32)])
 def test_full_size_configs_sampled(env, idx, per_seg, last_cols):
     """Full benchmark sizes in the launch configuration the benchmark times."""
     W, P, oracle, torch = env["W"], env["P"], env["oracle"], env["torch"]

@@ -55,7 +55,7 @@ def test_matches_bruteforce_enumeration(lengths, hq, hkv, bm, bn):
     assert len({(x[0], x[1], x[2]) for x in f.tolist()}) == len(f)
 
 
-@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5, 6])
 def test_counts_and_cost_sums_on_benchmark_configs(idx):
     w = W.config(idx)
     L = w.lengths
