@@ -151,8 +151,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4,
-                    help="benchmark configuration 1..5 (default 4: the nested-plan shard); 0 = the scaled-down nested "
-                         "case used for profiler captures")
+                    help="benchmark configuration 1..5 (default 4: the nested-plan shard); 6 = the mixed-degree "
+                         "full-tree shard; 0 = the scaled-down nested case used for profiler captures")
+    ap.add_argument("--uniform", type=int, default=0, metavar="L",
+                    help="instead of --config: 131,072 tokens at 32q/4kv in segments of L tokens each (short-segment "
+                         "studies; not a bench value)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile-mode", action="store_true",
@@ -187,7 +190,10 @@ def main():
         torch.cuda.synchronize()
 
     # one shard per GPU: same configuration, its own seed (lengths and values)
-    if args.config == 0:
+    if args.uniform > 0:
+        n = max(1, 131072 // args.uniform)
+        w = W.custom([args.uniform] * n, 32, 4, seed=1000 * rank, name=f"uniform_{n}x{args.uniform}_32q4kv")
+    elif args.config == 0:
         w = W.profile_case()
     else:
         w = W.config(args.config, seed=(args.config - 1) + 1000 * rank)
