@@ -56,7 +56,8 @@ enum {
   NSP_ERR_ALLOC = 3,          /* host or device allocation failed (plan construction only) */
   NSP_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (including: no device) */
   NSP_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait expired (sticky, see nsp_device_status) */
-  NSP_ERR_WORKSPACE = 6       /* workspace pointer null/misaligned or ws_bytes too small */
+  NSP_ERR_WORKSPACE = 6,      /* workspace pointer null/misaligned or ws_bytes too small */
+  NSP_ERR_INFEASIBLE = 7      /* nsp_route_sp_tree: no placement of the searched prefix fits the token budget */
 };
 
 enum { NSP_BF16 = 0, NSP_F32 = 1 }; /* output dtypes of the gradients */
@@ -173,6 +174,42 @@ int nsp_attn_bwd_recompute(const nsp_plan_t* plan, const uint8_t* recompute, con
                            const void* v, const void* o, const void* d_o, const float* lse, void* dq, void* dk,
                            void* dv, int dq_dtype, int dkv_dtype, float softmax_scale, void* ws, size_t ws_bytes,
                            void* stream);
+
+/*
+ * Planner (paper Sec. 4.2, "Routing Objective and Cost Model" and Algorithm 1, "Prefix-Completion SP-Tree Routing").
+ * Host only, no CUDA call.
+ *
+ * The SP tree is the full binary tree over P = 2^(n_levels-1) GPUs: node (l, i) covers GPUs [i*2^l, (i+1)*2^l) and
+ * runs its samples at SP degree 2^l.
+ *
+ * nsp_cost_table fills cost_out [n_samples * n_levels] (row j, column l: the load, in nanoseconds, that sample j
+ * puts on EVERY GPU of a level-l node, forward + backward) from profiled coefficients, level by level as the paper's
+ * cost model: compute = L(L+1)/2 causal pairs x hq/2^l local q heads x tcomp_ns[l * NSP_COST_BUCKETS + b] (profiled
+ * nanoseconds per pair and head at level l for the length class b = clip(floor(log2 L), 5, 20) - 5); prologue +
+ * epilogue = (L/d)(d-1)/d tokens x 4 * head_dim * (2 hq + 2 hkv) bytes (Q, K, V in and O out, forward and backward,
+ * bf16) / link_gbs[l] (GB/s of the fabric a level-l group communicates over; unused for l = 0); non-attention
+ * work = L/d tokens x other_ns_per_token. The sum is rounded to the nearest integer. hq, hkv: heads of the whole
+ * model. Errors: INVALID_ARG.
+ *
+ * nsp_route_sp_tree routes a batch: samples are visited by nonincreasing length (equal lengths keep their order);
+ * the first prefix_k are placed by a beam search over all tree nodes (root first, left to right; with monotone != 0
+ * a sample may not sit above the level of the previous, longer one), dropping states in which a GPU's token load
+ * Tok_p = sum of L/d exceeds b_tok and keeping the beam_w states with the smallest critical load max_p C_p (ties:
+ * order of generation); every surviving state is then completed greedily, each remaining sample going to the
+ * least-loaded single-GPU leaf that stays within b_tok, or to the leaf with the smallest token load when none
+ * does; the completed state with the smallest critical load is returned, states within the budget first.
+ * Outputs (host): level_out / index_out [n_samples] = the node of every sample; load_out [P] = C_p; tok_out [P] =
+ * Tok_p in units of 1/P token; feasible_out = 1 if every GPU is within b_tok (the last three may be NULL).
+ * Cost is O(prefix_k * beam_w * (2P-1) * P). Errors: INVALID_ARG (negative sizes, lengths or costs, n_levels not
+ * in 1..11, beam_w < 1), INFEASIBLE (no token-feasible placement of the prefix; nothing is written).
+ */
+#define NSP_COST_BUCKETS 16
+int nsp_cost_table(const int32_t* lengths, int32_t n_samples, int32_t n_levels, int32_t hq, int32_t hkv,
+                   int32_t head_dim, const double* tcomp_ns, const double* link_gbs, double other_ns_per_token,
+                   int64_t* cost_out);
+int nsp_route_sp_tree(const int32_t* lengths, const int64_t* cost, int32_t n_samples, int32_t n_levels,
+                      int32_t prefix_k, int32_t beam_w, int64_t b_tok, int32_t monotone, int32_t* level_out,
+                      int32_t* index_out, int64_t* load_out, int64_t* tok_out, int32_t* feasible_out);
 
 /* Read the sticky device status {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
 int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);

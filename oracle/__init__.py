@@ -3,7 +3,8 @@
 Only tests, the smoke check and the benchmark's CPU-baseline / reference legs import this package. It never
 imports the CUDA package and shares nothing with it. The attention and tile-plan arithmetic lives in the C file;
 this module compiles it with gcc, marshals numpy arrays and reshapes results. The one function written here in
-plain Python loops is ``recompute_mark`` (the save / recompute walk of the paper's tree-level recomputation).
+plain Python loops are ``recompute_mark`` (the save / recompute walk of the paper's tree-level recomputation) and
+``route_sp_tree`` (the paper's Algorithm 1, prefix-completion SP-tree routing) with its ``cost_table``.
 
 Conventions (identical to the C file header): packed ragged token-major tensors, bf16 inputs passed as
 ``uint16`` bit patterns (or ``float64`` arrays for finite-difference checks), float64 outputs.
@@ -185,3 +186,88 @@ def recompute_mark(lengths, hq, level, budget_bytes, head_dim=128):
         used += need
         flags[s] = 0
     return np.asarray(flags, dtype=np.uint8), used
+
+
+def route_sp_tree(lengths, cost, n_levels, k, w, b_tok, monotone=False):
+    """Prefix-completion SP-tree routing (paper Algorithm 1), step by step in the paper's order.
+
+    The SP tree is the full binary tree over P = 2**(n_levels-1) GPUs: node (l, i) covers GPUs
+    [i * 2**l, (i + 1) * 2**l) and runs its samples at SP degree 2**l. cost[j][l] is the load the cost model
+    attributes to EVERY GPU of a level-l node when sample j is placed there (any integer unit); the model is
+    additive, so CostModel(a) is the per-GPU sum. Token loads follow the paper's Tok_p: a sample of length L on a
+    degree-d node adds L / d to each of its GPUs; they are kept in units of 1/P token so that they stay integers.
+
+    State S = (a, C, T). FeasibleNodes = all tree nodes, root first, left to right (with ``monotone``: no level
+    above the level given to the previous, longer sample of the state). Beam and final choice break ties by order
+    of generation. The tail goes to the leaves ("effective leaf units" = the single-GPU nodes).
+
+    Returns None if the prefix search runs out of token-feasible states, else
+    (level[j], index[j], C[p], T[p] in 1/P tokens, feasible) with feasible = every GPU within b_tok."""
+    M = len(lengths)
+    K = n_levels - 1
+    P = 1 << K
+    order = sorted(range(M), key=lambda j: -int(lengths[j]))  # stable: equal lengths keep their order
+    H, R = order[:k], order[k:]
+    Q = [({}, [0] * P, [0] * P, K)]  # (a, C, T, level of the last placed sample)
+    for j in H:
+        N = []
+        for (a, C, T, last) in Q:
+            for l in range(K, -1, -1):
+                if monotone and l > last:
+                    continue
+                for i in range(P >> l):
+                    a2 = dict(a)
+                    a2[j] = (l, i)
+                    C2, T2 = list(C), list(T)
+                    for p in range(i << l, (i + 1) << l):
+                        C2[p] += int(cost[j][l])
+                        T2[p] += int(lengths[j]) * (P >> l)
+                    if max(T2) <= b_tok * P:
+                        N.append((a2, C2, T2, l))
+        if not N:
+            return None
+        N.sort(key=lambda S: max(S[1]))  # stable
+        Q = N[:w]
+    done = []
+    for (a, C, T, _) in Q:
+        a, C, T = dict(a), list(C), list(T)
+        for j in R:
+            Lj = int(lengths[j])
+            fits = [p for p in range(P) if T[p] + Lj * P <= b_tok * P]
+            if fits:
+                u = min(fits, key=lambda p: C[p])  # least-loaded unit that satisfies the budget (first on ties)
+            else:
+                u = min(range(P), key=lambda p: T[p])  # none does: the unit with the smallest token load
+            a[j] = (0, u)
+            C[u] += int(cost[j][0])
+            T[u] += Lj * P
+        done.append((a, C, T))
+    feas = [S for S in done if max(S[2]) <= b_tok * P] if done else []
+    pool = feas if feas else done
+    a, C, T = min(pool, key=lambda S: max(S[1]))
+    level = [a[j][0] for j in range(M)]
+    index = [a[j][1] for j in range(M)]
+    return level, index, C, T, bool(feas)
+
+
+def cost_table(lengths, n_levels, hq, hkv, head_dim, tcomp_ns, link_gbs, other_ns_per_token):
+    """The paper's hierarchical cost model (Sec. 4.2) for one sample on a level-l node, per covered GPU, forward +
+    backward, in nanoseconds: SP-backend level = compute (causal pairs x local q heads x profiled ns per pair and
+    head for the sample's length class) + prologue / epilogue all-to-alls (the (d-1)/d share of the GPU's L/d
+    tokens; Q, K, V in and O out, both passes, bf16) over the level's link bandwidth; model level = non-attention
+    time per resident token. tcomp_ns[l][b], b = clip(floor(log2 L), 5, 20) - 5. Returns int64 [n, n_levels]."""
+    import math
+
+    out = np.zeros((len(lengths), n_levels), dtype=np.int64)
+    for j, L in enumerate(int(x) for x in lengths):
+        b = min(max(L.bit_length() - 1, 5), 20) - 5 if L > 0 else 0
+        pairs = L * (L + 1) / 2.0
+        for l in range(n_levels):
+            d = float(1 << l)
+            comp = pairs * (hq / d) * float(tcomp_ns[l][b])
+            comm = 0.0
+            if l > 0:
+                comm = (L / d) * ((d - 1.0) / d) * (4.0 * head_dim * (2.0 * hq + 2.0 * hkv)) / float(link_gbs[l])
+            other = (L / d) * float(other_ns_per_token)
+            out[j, l] = math.floor(comp + comm + other + 0.5)
+    return out

@@ -18,6 +18,7 @@ NSP_ERR_ALLOC = 3
 NSP_ERR_CUDA = 4
 NSP_ERR_DEVICE_TIMEOUT = 5
 NSP_ERR_WORKSPACE = 6
+NSP_ERR_INFEASIBLE = 7
 NSP_BF16 = 0
 NSP_F32 = 1
 NSP_MAX_RUNS = 32
@@ -26,7 +27,9 @@ EXPORTS = [
     "nsp_plan_tiles", "nsp_plan_sizes", "nsp_plan_get", "nsp_attn_fwd", "nsp_attn_bwd", "nsp_device_status",
     "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string", "nsp_plan_set_profiling", "nsp_plan_kernel_ms",
     "nsp_attn_bwd_static", "nsp_recompute_mark", "nsp_plan_recompute_ws_bytes", "nsp_attn_bwd_recompute",
+    "nsp_cost_table", "nsp_route_sp_tree",
 ]
+NSP_COST_BUCKETS = 16
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
 KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST = 0, 1, 2, 3
 
@@ -77,6 +80,12 @@ def lib() -> ctypes.CDLL:
         L.nsp_attn_bwd_recompute.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int,
                                              ctypes.c_float, vp, ctypes.c_size_t, vp]
         L.nsp_attn_bwd_recompute.restype = ctypes.c_int
+        L.nsp_cost_table.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                     vp, vp, ctypes.c_double, vp]
+        L.nsp_cost_table.restype = ctypes.c_int
+        L.nsp_route_sp_tree.argtypes = [vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                        ctypes.c_int64, ctypes.c_int32, vp, vp, vp, vp, i32p]
+        L.nsp_route_sp_tree.restype = ctypes.c_int
         L.nsp_device_status.argtypes = [vp, i32p]
         L.nsp_device_status.restype = ctypes.c_int
         L.nsp_launch_count.argtypes = []
@@ -225,6 +234,51 @@ def nsp_recompute_mark(cu_seqlens, hq, level, budget_bytes: int, head_dim: int =
     if rc != NSP_OK:
         raise NspError(rc, "nsp_recompute_mark")
     return flags[:n], int(saved.value)
+
+
+def nsp_cost_table(lengths, n_levels, hq, hkv, head_dim, tcomp_ns, link_gbs, other_ns_per_token):
+    """Cost table [n_samples, n_levels] (int64 ns per covered GPU) from profiled coefficients (host only)."""
+    import numpy as np
+
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    tcomp = np.ascontiguousarray(tcomp_ns, dtype=np.float64)
+    link = np.ascontiguousarray(link_gbs, dtype=np.float64)
+    if tcomp.shape != (n_levels, NSP_COST_BUCKETS) or link.shape != (n_levels,):
+        raise ValueError("tcomp_ns must be [n_levels, NSP_COST_BUCKETS], link_gbs [n_levels]")
+    out = np.zeros((len(lengths), n_levels), dtype=np.int64)
+    vp = ctypes.c_void_p
+    rc = lib().nsp_cost_table(lengths.ctypes.data_as(vp), len(lengths), int(n_levels), int(hq), int(hkv), int(head_dim),
+                              tcomp.ctypes.data_as(vp), link.ctypes.data_as(vp), float(other_ns_per_token),
+                              out.ctypes.data_as(vp))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_cost_table")
+    return out
+
+
+def nsp_route_sp_tree(lengths, cost, n_levels, prefix_k, beam_w, b_tok, monotone=False):
+    """Algorithm 1 (host only). Returns (level[n], index[n], load[P], tok[P] in 1/P tokens, feasible) or raises
+    NspError(NSP_ERR_INFEASIBLE)."""
+    import numpy as np
+
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    cost = np.ascontiguousarray(cost, dtype=np.int64)
+    n = len(lengths)
+    if cost.shape != (n, n_levels):
+        raise ValueError("cost must be [n_samples, n_levels]")
+    P = 1 << (n_levels - 1)
+    level = np.zeros(max(n, 1), np.int32)
+    index = np.zeros(max(n, 1), np.int32)
+    load = np.zeros(P, np.int64)
+    tok = np.zeros(P, np.int64)
+    feas = ctypes.c_int32()
+    vp = ctypes.c_void_p
+    rc = lib().nsp_route_sp_tree(lengths.ctypes.data_as(vp), cost.ctypes.data_as(vp), n, int(n_levels), int(prefix_k),
+                                 int(beam_w), int(b_tok), int(bool(monotone)), level.ctypes.data_as(vp),
+                                 index.ctypes.data_as(vp), load.ctypes.data_as(vp), tok.ctypes.data_as(vp),
+                                 ctypes.byref(feas))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_route_sp_tree")
+    return level[:n], index[:n], load, tok, bool(feas.value)
 
 
 def nsp_plan_recompute_ws_bytes(plan: Plan) -> int:

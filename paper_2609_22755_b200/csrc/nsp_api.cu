@@ -144,6 +144,7 @@ const char* nsp_status_string(int code) {
     case NSP_ERR_CUDA: return "CUDA call failed";
     case NSP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
     case NSP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case NSP_ERR_INFEASIBLE: return "no plan within the token budget";
     default: return "unknown status";
   }
 }
