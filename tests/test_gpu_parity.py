@@ -157,6 +157,25 @@ def test_backward_with_recomputation(env, case, which):
                                  w.softmax_scale, run.ws[:max(run.plan.bwd_ws_bytes - 256, 0)])
 
 
+def test_routed_shards_run_through_the_kernels(env):
+    """Planner output instead of a hand-made shard: a scaled-down long-tailed batch is routed over eight GPUs (cost
+    table from the shipped measured coefficients, Algorithm 1), and the shards of the first GPU and of the GPU with
+    the most segments go through the kernels and are compared with the oracle element by element."""
+    W = env["W"]
+    from paper_2609_22755_b200 import planner
+
+    tail = W.lognormal_lengths(3, 8 * 2048 - 12288, 48, 1.3, 16, 1024)
+    lengths = [12288] + tail
+    r = planner.route_batch(lengths, 4, 2300, prefix_k=6, beam_w=4)
+    assert r["feasible"] and int(r["level"][0]) == 3
+    shards = r["shards"]
+    pick = {0, int(np.argmax([s.n_seg for s in shards]))}
+    for p in sorted(pick):
+        w = shards[p]
+        assert w.n_seg >= 2 and int(w.hq[0]) == 4
+        _full_case(env, w)
+
+
 def test_empty_and_degenerate_batches(env):
     B, W, P, torch = env["B"], env["W"], env["P"], env["torch"]
     # no segments at all

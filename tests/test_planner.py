@@ -200,3 +200,29 @@ def test_shards_from_routing():
     # every (sample, query head) pair is computed exactly once across the GPUs
     total = sum(int((s.lengths * s.hq).sum()) for s in shards)
     assert total == 32 * sum(lengths)
+
+
+def test_route_batch_on_a_long_tailed_batch(B):
+    """Eight GPUs, 65,536 tokens each: one 393,216-token sample plus a long tail, the shape of the nested-plan
+    benchmark shard. The token budget forces the long sample onto the root; the measured cost table balances the
+    rest."""
+    from paper_2609_22755_b200 import planner
+    from paper_2609_22755_b200 import workloads as W
+
+    tail = W.lognormal_lengths(0, 8 * 65536 - 393216, 1024, 1.3, 16, 32768)
+    lengths = [393216] + tail
+    r = planner.route_batch(lengths, 4, 70000)
+    assert r["feasible"] and int(r["level"][0]) == 3
+    assert r["tok"].max() <= 70000 * 8 and int(r["tok"].sum()) == 8 * sum(lengths)
+    load = r["load_ns"].astype(np.float64)
+    assert load.max() / load.mean() < 1.01
+    order = np.argsort(-np.asarray(lengths), kind="stable")
+    lv = r["level"][order][:8]
+    assert all(a >= b for a, b in zip(lv, lv[1:]))  # monotone SP over the searched prefix
+    # greedy alone (no prefix search) cannot place the long sample and is far worse
+    g = planner.route_batch(lengths, 4, 70000, prefix_k=0, beam_w=1)
+    assert not g["feasible"] and g["load_ns"].max() > 5 * load.max()
+    # GPU 0's shard: the long sample with 4 of the 32 query heads and one (replicated) KV head comes first
+    w = r["shards"][0]
+    assert int(w.lengths[0]) == 393216 and int(w.hq[0]) == 4 and int(w.hkv[0]) == 1
+    assert sum(int((s.lengths * s.hq).sum()) for s in r["shards"]) == 32 * sum(lengths)
