@@ -97,7 +97,7 @@ int nsp_plan_sizes(const nsp_plan_t* plan, int64_t* q_elems, int64_t* kv_elems, 
 
 /* Copy a work list to the host (pass 0 = forward, 1 = backward: the lists defined above, bit-exact; pass 2 = the
  * backward items in the order the backward kernel actually walks them: the same items grouped by (segment, kv
- * head), shorter segments first, key tiles ascending inside a group, which keeps the dQ accumulator rows of a q
+ * head), longer segments first, key tiles ascending inside a group, which keeps the dQ accumulator rows of a q
  * tile in L2 while all key tiles of the group add to them). Writes min(cap, n) items, stores n in *n_items
  * (host_out may be NULL to query). Synchronises the plan's build stream. */
 int nsp_plan_get(const nsp_plan_t* plan, int pass, nsp_tile_t* host_out, int64_t cap, int64_t* n_items);

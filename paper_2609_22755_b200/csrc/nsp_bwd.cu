@@ -51,6 +51,9 @@ constexpr uint32_t kBwdTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 // setmaxnreg redistributes the launch-time allocation (96 per thread): 256*136 + 256*80 + 128*48 = 640*96
 constexpr int kRegsSoftmax = 136, kRegsReduce = 80, kRegsAux = 48;
+constexpr int kFrontMinSteps = 2048;          // items shorter than this start at once
+constexpr int kFrontMinGroup = 8;             // so do items of groups with fewer q heads per kv head
+constexpr long long kFrontWaitClk = 1500000;  // ~0.9 ms: upper bound of the start alignment (also: 1/16 of the item)
 
 // Optional step timeline (compiled in only with -DNSP_TRACE, for tuning): clock64 stamps of the first CTA's roles.
 #ifdef NSP_TRACE
@@ -238,6 +241,27 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         x.mode_first = (a.debug_flags & 2) == 0 ? 1 : 0;
         x.per_head = (sg.len + kBM - 1) / kBM - item.tile + x.two_pass;  // q tiles n .. Mt-1 (bm == bn)
         x.steps = x.G * x.per_head;
+        // Start alignment. kFrontBlock consecutive items are neighbouring key tiles of one (segment, kv head) and
+        // walk the same (q tile, head) sequence from the segment's last q tile down. CTAs that start them at the
+        // same moment stay on the same q tile for the whole item and find its Q, dO and dQ-accumulator tiles in
+        // L2; left alone they start one q tile apart (items end G steps apart), and 148 CTAs on 148 different q
+        // tiles need 148 * G * 128 KB of L2: more than there is from G = 8 on (measured at G = 16: 900 GB of DRAM
+        // traffic for tensors of 15 GB). So the CTA of a long item of such a group waits here, for at most
+        // kFrontWaitClk, until the other items of its block have been popped as well (the CTAs that pop them are
+        // the next ones to finish, G steps apart). A timeout is not an error: the CTA just starts.
+        {
+          const int blk = idx / kFrontBlock;
+          const int rest = a.n_items - blk * kFrontBlock;
+          const int expect = rest < kFrontBlock ? rest : kFrontBlock;
+          atomicAdd(a.front + blk, 1);
+          if (x.steps >= kFrontMinSteps && x.G >= kFrontMinGroup) {
+            const long long t0 = clock64();
+            const long long own = static_cast<long long>(x.steps) * 340;  // about 1/16 of what the item takes
+            const long long limit = own < kFrontWaitClk ? own : kFrontWaitClk;
+            while (*reinterpret_cast<volatile int32_t*>(a.front + blk) < expect && clock64() - t0 < limit)
+              __nanosleep(200);
+          }
+        }
       }
     }
     tc_fence_before_sync();

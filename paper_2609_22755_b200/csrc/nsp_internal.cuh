@@ -10,6 +10,7 @@ namespace nsp {
 constexpr int kHeadDim = NSP_HEAD_DIM;
 constexpr int kBM = 128;  // query rows per tile
 constexpr int kBN = 128;  // key rows per tile
+constexpr int kFrontBlock = 16;  // backward: consecutive work items whose CTAs start together
 
 // Per-segment table entry (device + host copy).
 struct SegInfo {
@@ -104,6 +105,7 @@ struct BwdArgs {
   float scale;
   float scale_log2;
   int32_t debug_flags;  // experiments only: bit 0 = no hi/lo split, bit 1 = no exact delta
+  int32_t* front;       // [ceil(n_items / kFrontBlock)] arrival counters, zeroed before the launch (see next_item)
 };
 
 // Host-side launchers implemented next to their kernels.
