@@ -211,6 +211,27 @@ int nsp_route_sp_tree(const int32_t* lengths, const int64_t* cost, int32_t n_sam
                       int32_t prefix_k, int32_t beam_w, int64_t b_tok, int32_t monotone, int32_t* level_out,
                       int32_t* index_out, int64_t* load_out, int64_t* tok_out, int32_t* feasible_out);
 
+/*
+ * Layout steps of the Ulysses all-to-all around the attention compute (paper Sec. 2.2; the prologue and epilogue
+ * phases of a tree node, Sec. 4.2). The exchange itself (NCCL send / receive between the GPUs of the node) is issued
+ * by the caller; see ulysses.py for the schedule. Tensors are device pointers, rows of head_dim elements of dtype
+ * NSP_BF16 or NSP_F32, head_dim * element size a multiple of 16 bytes, pointers 16-byte aligned; first_head is a
+ * host array [n_blocks], n_blocks <= NSP_A2A_MAX_PEERS.
+ *
+ * nsp_a2a_gather_heads: src [tokens, heads, head_dim] (this GPU's token slice, all heads) -> dst [n_blocks][tokens,
+ * heads_per_block, head_dim], block p = heads [first_head[p], first_head[p] + heads_per_block): the contiguous block
+ * peer p receives. Blocks may overlap (a KV head replicated over several peers).
+ * nsp_a2a_scatter_heads: the inverse, src [n_blocks][tokens, heads_per_block, head_dim] -> dst [tokens, heads,
+ * head_dim]; where several blocks carry the same head (partial dK / dV of a replicated KV head) they are added in
+ * block order in fp32; heads no block carries are left untouched.
+ * Errors: INVALID_ARG, UNSUPPORTED (row size not a multiple of 16 bytes), CUDA.
+ */
+#define NSP_A2A_MAX_PEERS 64
+int nsp_a2a_gather_heads(const void* src, void* dst, int64_t tokens, int32_t heads, int32_t heads_per_block,
+                         int32_t n_blocks, int32_t head_dim, int32_t dtype, const int32_t* first_head, void* stream);
+int nsp_a2a_scatter_heads(const void* src, void* dst, int64_t tokens, int32_t heads, int32_t heads_per_block,
+                          int32_t n_blocks, int32_t head_dim, int32_t dtype, const int32_t* first_head, void* stream);
+
 /* Read the sticky device status {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
 int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
 

@@ -27,7 +27,7 @@ EXPORTS = [
     "nsp_plan_tiles", "nsp_plan_sizes", "nsp_plan_get", "nsp_attn_fwd", "nsp_attn_bwd", "nsp_device_status",
     "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string", "nsp_plan_set_profiling", "nsp_plan_kernel_ms",
     "nsp_attn_bwd_static", "nsp_recompute_mark", "nsp_plan_recompute_ws_bytes", "nsp_attn_bwd_recompute",
-    "nsp_cost_table", "nsp_route_sp_tree",
+    "nsp_cost_table", "nsp_route_sp_tree", "nsp_a2a_gather_heads", "nsp_a2a_scatter_heads",
 ]
 NSP_COST_BUCKETS = 16
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
@@ -86,6 +86,10 @@ def lib() -> ctypes.CDLL:
         L.nsp_route_sp_tree.argtypes = [vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                         ctypes.c_int64, ctypes.c_int32, vp, vp, vp, vp, i32p]
         L.nsp_route_sp_tree.restype = ctypes.c_int
+        for f in (L.nsp_a2a_gather_heads, L.nsp_a2a_scatter_heads):
+            f.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                          ctypes.c_int32, vp, vp]
+            f.restype = ctypes.c_int
         L.nsp_device_status.argtypes = [vp, i32p]
         L.nsp_device_status.restype = ctypes.c_int
         L.nsp_launch_count.argtypes = []
@@ -279,6 +283,30 @@ def nsp_route_sp_tree(lengths, cost, n_levels, prefix_k, beam_w, b_tok, monotone
     if rc != NSP_OK:
         raise NspError(rc, "nsp_route_sp_tree")
     return level[:n], index[:n], load, tok, bool(feas.value)
+
+
+def _a2a(fn_name, src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream):
+    import numpy as np
+    import torch
+
+    dtype = NSP_F32 if src.dtype == torch.float32 else NSP_BF16
+    if dst.dtype != src.dtype:
+        raise ValueError("source and destination must have the same dtype")
+    fh = np.ascontiguousarray(first_head, dtype=np.int32)
+    rc = getattr(lib(), fn_name)(_ptr(src), _ptr(dst), int(tokens), int(heads), int(heads_per_block), len(fh),
+                                 int(head_dim), dtype, fh.ctypes.data_as(ctypes.c_void_p), _stream_ptr(stream))
+    if rc != NSP_OK:
+        raise NspError(rc, fn_name)
+
+
+def nsp_a2a_gather_heads(src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream=None):
+    """[tokens, heads, D] -> [len(first_head)][tokens, heads_per_block, D] (device tensors, flat or shaped)."""
+    _a2a("nsp_a2a_gather_heads", src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream)
+
+
+def nsp_a2a_scatter_heads(src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream=None):
+    """[len(first_head)][tokens, heads_per_block, D] -> [tokens, heads, D], adding blocks that share a head."""
+    _a2a("nsp_a2a_scatter_heads", src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream)
 
 
 def nsp_plan_recompute_ws_bytes(plan: Plan) -> int:

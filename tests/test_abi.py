@@ -22,7 +22,7 @@ def B():
 
 def test_header_symbols_are_exported(B):
     header = (ROOT / "include" / "nsp.h").read_text()
-    declared = set(re.findall(r"\b(nsp_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(nsp_[a-z0-9_]+)\s*\(", header))
     assert {"nsp_plan_tiles", "nsp_attn_fwd", "nsp_attn_bwd"} <= declared
     lib = ctypes.CDLL(str(B.LIB_PATH))
     for name in sorted(declared):

@@ -1,0 +1,157 @@
+"""Ulysses prologue / epilogue (paper Sec. 2.2, Sec. 4.2): the exchange schedule on CPU ranks (gloo, world sizes 2 and
+4, layout steps by a plain torch stand-in), and the library's CUDA layout kernels on one GPU against the same
+stand-in, including an emulation of all ranks of a node in one process."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+
+
+class TorchLayoutOps:
+    """Plain torch indexing with the semantics of nsp_a2a_gather_heads / nsp_a2a_scatter_heads."""
+
+    def gather(self, src, dst, tokens, heads, hpb, D, first, stream=None):
+        src = src.reshape(tokens, heads, D)
+        dst = dst.reshape(len(first), tokens, hpb, D)
+        for p, f in enumerate(first):
+            dst[p].copy_(src[:, f:f + hpb])
+
+    def scatter(self, src, dst, tokens, heads, hpb, D, first, stream=None):
+        src = src.reshape(len(first), tokens, hpb, D)
+        dst = dst.reshape(tokens, heads, D)
+        for h in range(heads):
+            parts = [src[p][:, h - f] for p, f in enumerate(first) if f <= h < f + hpb]
+            if len(parts) == 1:
+                dst[:, h] = parts[0]
+            elif parts:
+                acc = torch.zeros_like(parts[0], dtype=torch.float32)
+                for x in parts:  # block order, fp32
+                    acc = acc + x.float()
+                dst[:, h] = acc.to(dst.dtype)
+
+
+def _global(lengths, H, D, seed, dtype=torch.float32):
+    g = torch.Generator().manual_seed(seed)
+    return [torch.randn(L, H, D, generator=g).to(dtype) for L in lengths]
+
+
+def _local(xs, d, r):
+    return torch.cat([x[r * (x.shape[0] // d):(r + 1) * (x.shape[0] // d)] for x in xs])
+
+
+def _worker(rank, world, port, hq, hkv):
+    import torch.distributed as dist
+
+    from paper_2609_22755_b200.ulysses import NodeLayout, UlyssesExchange
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        D = 16
+        lengths = [8 * world, 0, 3 * world, 20 * world]
+        lay = NodeLayout(lengths, world, rank, hq, hkv, D)
+        ex = UlyssesExchange(lay, list(range(world)), ops=TorchLayoutOps())
+        q = _global(lengths, hq, D, 1)
+        kv = _global(lengths, hkv, D, 2)
+        # prologue: complete sequences, this rank's heads
+        got_q = ex.to_attention_layout(_local(q, world, rank), "q")
+        want_q = torch.cat([x[:, lay.q_first[rank]:lay.q_first[rank] + lay.hq_loc] for x in q])
+        assert torch.equal(got_q, want_q)
+        got_k = ex.to_attention_layout(_local(kv, world, rank), "kv")
+        want_k = torch.cat([x[:, lay.kv_first[rank]:lay.kv_first[rank] + lay.hkv_loc] for x in kv])
+        assert torch.equal(got_k, want_k)
+        # epilogue of a q-shaped tensor: the exact inverse
+        back = ex.from_attention_layout(got_q, "q")
+        assert torch.equal(back, _local(q, world, rank))
+        # epilogue of dK: rank s contributes (s + 1) * its block; shared heads are summed over the sharing ranks
+        part = got_k * float(rank + 1)
+        got_dk = ex.from_attention_layout(part, "kv")
+        want = torch.zeros(lay.t_loc, hkv, D)
+        for s in range(world):
+            f = lay.kv_first[s]
+            blk = torch.cat([x[:, f:f + lay.hkv_loc] for x in kv]) * float(s + 1)  # what rank s holds, full length
+            mine = torch.cat([blk[lay.full_off[j] + rank * lay.tok_loc[j]:lay.full_off[j] + (rank + 1) * lay.tok_loc[j]]
+                              for j in range(len(lengths))])
+            want[:, f:f + lay.hkv_loc] += mine
+        assert torch.allclose(got_dk, want, rtol=0, atol=1e-5)
+    finally:
+        dist.destroy_process_group()
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+@pytest.mark.parametrize("world,hq,hkv", [(2, 8, 4), (2, 4, 1), (4, 8, 2), (4, 8, 8)])
+def test_exchange_schedule_on_cpu_ranks(world, hq, hkv):
+    import torch.multiprocessing as mp
+
+    mp.spawn(_worker, args=(world, _free_port(), hq, hkv), nprocs=world, join=True)
+
+
+def test_layout_rejects_bad_shapes():
+    from paper_2609_22755_b200.ulysses import NodeLayout
+
+    with pytest.raises(ValueError):
+        NodeLayout([10], 4, 0, 8, 2)  # length not a multiple of the degree
+    with pytest.raises(ValueError):
+        NodeLayout([16], 4, 0, 6, 2)  # degree does not divide the query heads
+    with pytest.raises(ValueError):
+        NodeLayout([16], 4, 4, 8, 2)  # rank outside the group
+    lay = NodeLayout([16, 32], 4, 1, 8, 2)
+    assert lay.kv_first == [0, 0, 1, 1] and lay.hkv_loc == 1 and lay.q_first == [0, 2, 4, 6]
+    assert lay.t_loc == 12 and lay.t_full == 48
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("d,hq,hkv", [(2, 8, 4), (4, 8, 2), (8, 32, 4)])
+def test_cuda_layout_kernels_and_one_process_emulation(d, hq, hkv, dtype):
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2609_22755_b200.ulysses import CudaLayoutOps, NodeLayout
+
+    D = 128
+    dev = torch.device("cuda:0")
+    lengths = [64 * d, 8 * d, 0, 1000 * d]
+    q = [x.to(dev) for x in _global(lengths, hq, D, 3, dtype)]
+    kv = [x.to(dev) for x in _global(lengths, hkv, D, 4, dtype)]
+    cuda_ops, ref_ops = CudaLayoutOps(), TorchLayoutOps()
+    lays = [NodeLayout(lengths, d, r, hq, hkv, D) for r in range(d)]
+    sends = {}
+    for kind, xs in (("q", q), ("kv", kv)):
+        for r, lay in enumerate(lays):
+            H, h_loc, first = lay.heads(kind)
+            x_loc = _local(xs, d, r).contiguous()
+            got = torch.empty((d, lay.t_loc, h_loc, D), dtype=dtype, device=dev)
+            want = torch.empty_like(got)
+            cuda_ops.gather(x_loc, got, lay.t_loc, H, h_loc, D, first)
+            ref_ops.gather(x_loc, want, lay.t_loc, H, h_loc, D, first)
+            assert torch.equal(got, want)
+            sends[kind, r] = got
+    # all ranks in one process: move the blocks the way the exchange does and compare with the global slicing
+    for kind, xs in (("q", q), ("kv", kv)):
+        for r, lay in enumerate(lays):
+            H, h_loc, first = lay.heads(kind)
+            full = torch.empty((lay.t_full, h_loc, D), dtype=dtype, device=dev)
+            for s in range(d):
+                for j in range(len(lengths)):
+                    a = int(lay.full_off[j]) + s * lay.tok_loc[j]
+                    full[a:a + lay.tok_loc[j]] = sends[kind, s][r, int(lay.loc_off[j]):int(lay.loc_off[j + 1])]
+            assert torch.equal(full, torch.cat([x[:, first[r]:first[r] + h_loc] for x in xs]))
+    # scatter: inverse for q; sums for shared KV heads
+    for kind in ("q", "kv"):
+        lay = lays[0]
+        H, h_loc, first = lay.heads(kind)
+        g = torch.Generator(device=dev).manual_seed(5)
+        blocks = torch.randn((d, lay.t_loc, h_loc, D), device=dev, generator=g).to(dtype)
+        got = torch.full((lay.t_loc, H, D), 7.0, dtype=dtype, device=dev)
+        want = got.clone()
+        cuda_ops.scatter(blocks, got, lay.t_loc, H, h_loc, D, first)
+        ref_ops.scatter(blocks, want, lay.t_loc, H, h_loc, D, first)
+        assert torch.equal(got, want)
