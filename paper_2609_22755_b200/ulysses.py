@@ -160,7 +160,8 @@ def phase_streams(nodes, prologue, compute, epilogue):
     """Two-queue phase streaming over the nodes of a GPU's chain: the prologue of node i + 1 and the epilogue of node
     i - 1 run on a communication stream while node i computes. prologue(i) / compute(i, inputs) / epilogue(i, outputs)
     are callables; each is issued under the stream it belongs to and ordered with CUDA events. Returns the list of
-    epilogue results. Without CUDA (CPU tensors) the phases simply run in order."""
+    epilogue results. Tensors a phase allocates cross streams: the caller keeps them alive until the returned results
+    have been consumed (as the lists here do). Without CUDA (CPU tensors) the phases simply run in order."""
     import torch
 
     if not torch.cuda.is_available():

@@ -155,3 +155,52 @@ def test_cuda_layout_kernels_and_one_process_emulation(d, hq, hkv, dtype):
         cuda_ops.scatter(blocks, got, lay.t_loc, H, h_loc, D, first)
         ref_ops.scatter(blocks, want, lay.t_loc, H, h_loc, D, first)
         assert torch.equal(got, want)
+
+
+@pytest.mark.gpu
+def test_phase_streams_orders_the_phases_on_one_gpu():
+    """Two-queue phase streaming with the exchange replaced by its layout step alone (one GPU, no peers): every
+    node's result must equal what the three phases give when run one after the other on one stream."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2609_22755_b200 import binding as B
+    from paper_2609_22755_b200 import workloads as W
+    from paper_2609_22755_b200.ulysses import phase_streams
+
+    dev = torch.device("cuda:0")
+    D = 128
+    nodes = [W.custom([2048, 512], 8, 2, seed=1), W.custom([4096], 4, 1, seed=2), W.custom([256] * 6, 16, 4, seed=3)]
+    plans = [B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, D) for w in nodes]
+    host = [W.make_tensors(w, which=("q", "k", "v")) for w in nodes]
+    staged = [{n: t.to(dev) for n, t in h.items() if n in ("q", "k", "v")} for h in host]
+
+    def prologue(i):  # stands for the all-to-all: a head gather of the whole tensor into one block
+        w, out = nodes[i], {}
+        T = int(w.lengths.sum())
+        for name, H in (("q", int(w.hq[0])), ("k", int(w.hkv[0])), ("v", int(w.hkv[0]))):
+            dst = torch.empty_like(staged[i][name])
+            B.nsp_a2a_gather_heads(staged[i][name], dst, T, H, H, D, [0], torch.cuda.current_stream())
+            out[name] = dst
+        return out
+
+    def compute(i, x):
+        w = nodes[i]
+        o = torch.empty_like(x["q"])
+        lse = torch.empty(w.lse_elems(), dtype=torch.float32, device=dev)
+        B.nsp_attn_fwd(plans[i], x["q"], x["k"], x["v"], o, lse, w.softmax_scale, stream=torch.cuda.current_stream())
+        return o
+
+    def epilogue(i, o):
+        w = nodes[i]
+        out = torch.empty_like(o)
+        B.nsp_a2a_scatter_heads(o, out, int(w.lengths.sum()), int(w.hq[0]), int(w.hq[0]), D, [0],
+                                torch.cuda.current_stream())
+        return out
+
+    want = [epilogue(i, compute(i, prologue(i))) for i in range(len(nodes))]
+    torch.cuda.synchronize()
+    got = phase_streams(nodes, prologue, compute, epilogue)
+    torch.cuda.synchronize()
+    for g, w_ in zip(got, want):
+        assert torch.equal(g, w_)
+    assert all(B.nsp_device_status(p)[0] == 0 for p in plans)
