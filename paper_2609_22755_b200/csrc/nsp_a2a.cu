@@ -23,96 +23,107 @@ struct HeadMap {
   int32_t first_head[NSP_A2A_MAX_PEERS];
 };
 
-// one thread per 16 bytes of the packed side
+// Both kernels are launched with a thread count that is a multiple of the 16-byte vectors of one token row of the
+// side they iterate over, so a thread keeps its (head, vector) position for the whole grid-stride loop and only the
+// token (and, for the gather, the block) advances: no division inside the loop.
+
+// one thread per 16 bytes of the packed side [n][T, Hd, D]
 __global__ void __launch_bounds__(256) gather_heads_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
                                                            int64_t T, int H, int Hd, int n, int vec_per_row,
                                                            const __grid_constant__ HeadMap map) {
-  const int64_t per_block = T * Hd * vec_per_row;
-  const int64_t total = per_block * n;
-  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
-       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-    const int p = static_cast<int>(i / per_block);
-    const int64_t r = i - p * per_block;
-    const int64_t tok = r / (Hd * vec_per_row);
-    const int rem = static_cast<int>(r - tok * (Hd * vec_per_row));
-    const int hh = rem / vec_per_row, v = rem - hh * vec_per_row;
-    dst[i] = __ldg(src + (tok * H + map.first_head[p] + hh) * vec_per_row + v);
+  const int row = Hd * vec_per_row;  // vectors of one token inside a block
+  const int64_t threads = static_cast<int64_t>(gridDim.x) * blockDim.x;  // a multiple of `row`
+  const int64_t t0 = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int in_row = static_cast<int>(t0 % row);
+  const int hh = in_row / vec_per_row, v = in_row - hh * vec_per_row;
+  const int64_t tok_step = threads / row;
+  int64_t tok = t0 / row;
+  int p = 0;
+  for (;;) {
+    while (tok >= T && p < n) tok -= T, ++p;
+    if (p >= n) break;
+    dst[(p * T + tok) * row + in_row] = __ldg(src + (tok * H + map.first_head[p] + hh) * vec_per_row + v);
+    tok += tok_step;
   }
 }
 
-// one thread per 16 bytes of the [T, H, D] side; the blocks that cover the head are added in block order.
-// The blocks that carry a head are found first (no memory access); the common case of exactly one is a plain copy,
-// two elements per thread and pass so that two loads are in flight.
+// one thread per 16 bytes of the [T, H, D] side; the blocks that carry the thread's head are found once, the common
+// case of exactly one is a plain copy (two tokens per pass, so that two loads are in flight), several are added in
+// block order in fp32
 template <bool kF32>
 __global__ void __launch_bounds__(256) scatter_heads_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
                                                             int64_t T, int H, int Hd, int n, int vec_per_row,
                                                             const __grid_constant__ HeadMap map) {
-  const int64_t total = T * H * vec_per_row;
+  const int row = H * vec_per_row;
+  const int64_t threads = static_cast<int64_t>(gridDim.x) * blockDim.x;  // a multiple of `row`
+  const int64_t t0 = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int in_row = static_cast<int>(t0 % row);
+  const int h = in_row / vec_per_row, v = in_row - h * vec_per_row;
+  const int64_t tok_step = threads / row;
   const int64_t per_block = T * Hd * vec_per_row;
-  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-  for (int64_t i0 = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i0 < total; i0 += 2 * stride) {
-    uint64_t hits[2] = {0, 0};
-    int64_t off[2] = {0, 0};  // offset of the element inside a block
-    int h2[2] = {0, 0};
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int64_t i = i0 + u * stride;
-      if (i >= total) continue;
-      const int64_t tok = i / (H * vec_per_row);
-      const int rem = static_cast<int>(i - tok * (H * vec_per_row));
-      const int h = rem / vec_per_row, v = rem - h * vec_per_row;
-      h2[u] = h;
-      off[u] = tok * Hd * vec_per_row + v;
-      for (int p = 0; p < n; ++p) {
-        const int hh = h - map.first_head[p];
-        if (hh >= 0 && hh < Hd) hits[u] |= 1ull << p;
-      }
+  uint64_t hits = 0;
+  for (int p = 0; p < n; ++p) {
+    const int hh = h - map.first_head[p];
+    if (hh >= 0 && hh < Hd) hits |= 1ull << p;
+  }
+  const int cnt = __popcll(hits);
+  if (cnt == 0) return;  // a head no block carries is left as it is
+  if (cnt == 1) {
+    const int p = __ffsll(static_cast<long long>(hits)) - 1;
+    const uint4* s1 = src + p * per_block + static_cast<int64_t>(h - map.first_head[p]) * vec_per_row + v;
+    const int64_t srow = static_cast<int64_t>(Hd) * vec_per_row;
+    int64_t tok = t0 / row;
+    for (; tok + tok_step < T; tok += 2 * tok_step) {
+      const uint4 a = __ldg(s1 + tok * srow), b = __ldg(s1 + (tok + tok_step) * srow);
+      dst[tok * row + in_row] = a;  // a plain copy keeps the bits
+      dst[(tok + tok_step) * row + in_row] = b;
     }
-    uint4 one[2];
+    if (tok < T) dst[tok * row + in_row] = __ldg(s1 + tok * srow);
+    return;
+  }
+  for (int64_t tok = t0 / row; tok < T; tok += tok_step) {
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    uint64_t left = hits;
+    while (left) {  // up to four loads in flight, added in block order
+      uint4 x[4];
+      int m = 0;
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (__popcll(hits[u]) == 1) {
-        const int p = __ffsll(static_cast<long long>(hits[u])) - 1;
-        one[u] = __ldg(src + p * per_block + off[u] + static_cast<int64_t>(h2[u] - map.first_head[p]) * vec_per_row);
+      for (int u = 0; u < 4; ++u) {
+        if (left) {
+          const int p = __ffsll(static_cast<long long>(left)) - 1;
+          left &= left - 1;
+          x[u] = __ldg(src + p * per_block + (tok * Hd + (h - map.first_head[p])) * vec_per_row + v);
+          m = u + 1;
+        }
       }
-    }
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int64_t i = i0 + u * stride;
-      const int cnt = __popcll(hits[u]);
-      if (cnt == 0) continue;  // a head no block carries is left as it is
-      if (cnt == 1) {
-        dst[i] = one[u];  // a plain copy keeps the bits
-        continue;
-      }
-      float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      for (int p = 0; p < n; ++p) {
-        if (!((hits[u] >> p) & 1ull)) continue;
-        const uint4 x = __ldg(src + p * per_block + off[u] + static_cast<int64_t>(h2[u] - map.first_head[p]) * vec_per_row);
-        if (kF32) {
-          acc[0] += __uint_as_float(x.x), acc[1] += __uint_as_float(x.y);
-          acc[2] += __uint_as_float(x.z), acc[3] += __uint_as_float(x.w);
-        } else {
-          const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+      for (int u = 0; u < 4; ++u) {
+        if (u < m) {
+          if (kF32) {
+            acc[0] += __uint_as_float(x[u].x), acc[1] += __uint_as_float(x[u].y);
+            acc[2] += __uint_as_float(x[u].z), acc[3] += __uint_as_float(x[u].w);
+          } else {
+            const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
 #pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            acc[2 * t] += __uint_as_float(w[t] << 16);
-            acc[2 * t + 1] += __uint_as_float(w[t] & 0xffff0000u);
+            for (int t = 0; t < 4; ++t) {
+              acc[2 * t] += __uint_as_float(w[t] << 16);
+              acc[2 * t + 1] += __uint_as_float(w[t] & 0xffff0000u);
+            }
           }
         }
       }
-      if (kF32) {
-        dst[i] = make_uint4(__float_as_uint(acc[0]), __float_as_uint(acc[1]), __float_as_uint(acc[2]),
-                            __float_as_uint(acc[3]));
-      } else {
-        uint32_t w[4];
+    }
+    if (kF32) {
+      dst[tok * row + in_row] = make_uint4(__float_as_uint(acc[0]), __float_as_uint(acc[1]), __float_as_uint(acc[2]),
+                                           __float_as_uint(acc[3]));
+    } else {
+      uint32_t w[4];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[2 * t], acc[2 * t + 1]);
-          w[t] = *reinterpret_cast<const uint32_t*>(&b2);
-        }
-        dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int t = 0; t < 4; ++t) {
+        const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[2 * t], acc[2 * t + 1]);
+        w[t] = *reinterpret_cast<const uint32_t*>(&b2);
       }
+      dst[tok * row + in_row] = make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
 }
@@ -135,10 +146,16 @@ int check(const void* src, void* dst, int64_t tokens, int heads, int heads_per_b
   return NSP_OK;
 }
 
-int grid_for(int64_t total) {
+// Blocks of 256 threads whose total is a multiple of `row` (the vectors of one token row), about `total` threads but
+// no more than 32 blocks per SM.
+int grid_for(int64_t total, int row) {
+  int a = row, b = 256;
+  while (b) { const int t = a % b; a = b; b = t; }
+  const int unit = row / a;  // blocks per multiple of `row`
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 32) blocks = 148 * 32;
-  return static_cast<int>(blocks < 1 ? 1 : blocks);
+  blocks = (blocks + unit - 1) / unit * unit;
+  return static_cast<int>(blocks < unit ? unit : blocks);
 }
 
 }  // namespace
@@ -152,7 +169,7 @@ extern "C" int nsp_a2a_gather_heads(const void* src, void* dst, int64_t tokens, 
   const int vec = head_dim * (dtype == NSP_F32 ? 4 : 2) / 16;
   const int64_t total = tokens * heads_per_block * vec * n_blocks;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  gather_heads_kernel<<<grid_for(total), 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
+  gather_heads_kernel<<<grid_for(total, heads_per_block * vec), 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
                                                           tokens, heads, heads_per_block, n_blocks, vec, map);
   nsp::count_launches(1);
   return cudaGetLastError() == cudaSuccess ? NSP_OK : NSP_ERR_CUDA;
@@ -168,10 +185,10 @@ extern "C" int nsp_a2a_scatter_heads(const void* src, void* dst, int64_t tokens,
   const int64_t total = tokens * heads * vec;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (dtype == NSP_F32)
-    scatter_heads_kernel<true><<<grid_for(total), 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
+    scatter_heads_kernel<true><<<grid_for(total, heads * vec), 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
                                                                 tokens, heads, heads_per_block, n_blocks, vec, map);
   else
-    scatter_heads_kernel<false><<<grid_for(total), 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
+    scatter_heads_kernel<false><<<grid_for(total, heads * vec), 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
                                                                  tokens, heads, heads_per_block, n_blocks, vec, map);
   nsp::count_launches(1);
   return cudaGetLastError() == cudaSuccess ? NSP_OK : NSP_ERR_CUDA;
