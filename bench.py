@@ -144,6 +144,34 @@ def reference_arm(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def rank_workload(config: int, uniform: int, rank: int):
+    """The shard a rank runs: every GPU gets the same configuration with its own seed (lengths and values), so N
+    GPUs are N independent replicas and the job's work grows with N (weak scaling)."""
+    if uniform > 0:
+        n = max(1, 131072 // uniform)
+        return W.custom([uniform] * n, 32, 4, seed=1000 * rank, name=f"uniform_{n}x{uniform}_32q4kv")
+    if config == 0:
+        return W.profile_case()
+    return W.config(config, seed=(config - 1) + 1000 * rank)
+
+
+def max_over_ranks(ms: float, world: int, device: str) -> float:
+    """The step time of the job is the slowest rank's."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_rank: float, world: int, ms: float) -> float:
+    """TFLOP/s of the whole job: what all ranks processed divided by the slowest rank's time."""
+    return world * flops_per_rank / (ms * 1e-3) / 1e12
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -190,13 +218,7 @@ def main():
         torch.cuda.synchronize()
 
     # one shard per GPU: same configuration, its own seed (lengths and values)
-    if args.uniform > 0:
-        n = max(1, 131072 // args.uniform)
-        w = W.custom([args.uniform] * n, 32, 4, seed=1000 * rank, name=f"uniform_{n}x{args.uniform}_32q4kv")
-    elif args.config == 0:
-        w = W.profile_case()
-    else:
-        w = W.config(args.config, seed=(args.config - 1) + 1000 * rank)
+    w = rank_workload(args.config, args.uniform, rank)
     host = W.make_tensors(w)
     host = {k: v.pin_memory() for k, v in host.items()}
     eng = NspAttention(w, device=f"cuda:{local_rank}")
@@ -228,12 +250,8 @@ def main():
     barrier()
     launches = B.launch_count() - launches0
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1) / args.steps
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * flops / (ms * 1e-3) / 1e12
+    ms = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, "cuda")
+    value = whole_job_value(flops, world, ms)
     assert eng.status()[0] == 0, f"device status {eng.status()}"
 
     # ---- end to end: host buffers in, host buffers out
@@ -247,12 +265,8 @@ def main():
             h2d, d2h = eng.step_host(host, host_out)
         e1.record()
         barrier()
-        ms_e2e = e0.elapsed_time(e1) / args.steps
-        if world > 1:
-            t = torch.tensor([ms_e2e], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, "cuda")
+        e2e = {"value": whole_job_value(flops, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e}
 
     if rank == 0:
