@@ -55,9 +55,18 @@ class NspAttention:
     def forward(self):
         B.nsp_attn_fwd(self.plan, self.q, self.k, self.v, self.o, self.lse, self.scale, stream=self.stream)
 
-    def backward(self):
-        B.nsp_attn_bwd(self.plan, self.q, self.k, self.v, self.o, self.do, self.lse, self.dq, self.dk, self.dv,
-                       self.scale, self.ws, stream=self.stream)
+    def backward(self, recompute=None):
+        """recompute: optional uint8 flags per segment (see nsp_recompute_mark): O and LSE of a flagged segment are
+        not read, the backward pass recomputes what it needs of them."""
+        if recompute is None:
+            B.nsp_attn_bwd(self.plan, self.q, self.k, self.v, self.o, self.do, self.lse, self.dq, self.dk, self.dv,
+                           self.scale, self.ws, stream=self.stream)
+            return
+        need = B.nsp_plan_recompute_ws_bytes(self.plan)
+        if self.ws.numel() < need:
+            self.ws = self.torch.empty(need, dtype=self.torch.uint8, device=self.dev)
+        B.nsp_attn_bwd_recompute(self.plan, recompute, self.q, self.k, self.v, self.o, self.do, self.lse, self.dq,
+                                 self.dk, self.dv, self.scale, self.ws, stream=self.stream)
 
     def step_device(self):
         self.forward()

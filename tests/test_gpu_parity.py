@@ -155,6 +155,19 @@ def test_backward_with_recomputation(env, case, which):
     with pytest.raises(B.NspError):
         B.nsp_attn_bwd_recompute(run.plan, flags, run.q, run.k, run.v, o, run.do, lse, run.dq, run.dk, run.dv,
                                  w.softmax_scale, run.ws[:max(run.plan.bwd_ws_bytes - 256, 0)])
+    if which == "alternate":  # the same through the user-facing wrapper
+        from paper_2609_22755_b200.api import NspAttention
+
+        eng = NspAttention(w)
+        eng.load(run.host)
+        eng.forward()
+        eng.o.copy_(o)
+        eng.lse.copy_(lse)
+        eng.backward(recompute=flags)
+        torch.cuda.synchronize()
+        assert eng.status()[0] == 0
+        for name in ("dk", "dv"):
+            assert torch.equal(getattr(eng, name), getattr(run, name))
 
 
 def test_routed_shards_run_through_the_kernels(env):
