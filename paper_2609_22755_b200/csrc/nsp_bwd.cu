@@ -37,6 +37,7 @@
 // together do not fit in it runs at the speed of instruction fetch. So the common step (an interior tile) has
 // its own lean, fully unrolled path; everything rare (diagonal tile, first-tile passes, ragged tail, item
 // epilogue) goes through compact rolled loops; an item is decoded once, by one thread, into shared memory.
+#include <type_traits>
 #include <cuda_bf16.h>
 #include "nsp_internal.cuh"
 #include "sm100_ptx.cuh"
@@ -585,8 +586,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         if (tid == 0) NSP_TRACE_STAMP(5);
         const float* lse_s = s.lse[st] + half * 64;
         float* delta_s = s.delta[st] + half * 64;
-        if (mode == 0 && m != c.n) {
-          // ---- common step (interior tile). Phase 1: P^T = exp2(S^T * c - LSE) for this thread's 64 query
+        // ---- common step (interior tile; the diagonal tile runs a second copy of the same code with a mask on P,
+        // kept apart so that the interior copy's instructions stay as they are)
+        auto common_step = [&](auto diag_tag) -> bool {
+          // Phase 1: P^T = exp2(S^T * c - LSE) for this thread's 64 query
           // columns, bf16 pairs over the S^T columns already read. The dV product needs only P^T, so it is
           // released to the MMA thread before dS^T is formed.
           // Sixteen columns at a time; the LSE (delta) values of the next sixteen are requested before the
@@ -619,6 +622,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               pp[ch >> 1][(x >> 1) + 0] = pack_bf16x2(ex2f(x0), ex2f(x1));
               pp[ch >> 1][(x >> 1) + 1] = pack_bf16x2(ex2f(x2), ex2f(x3));
             }
+            if constexpr (decltype(diag_tag)::value) {
+              // diagonal tile: a key sees only the queries at or after it. Element e of this chunk (query column
+              // 64 * half + 16 * ch + e) survives iff e >= t; P = 0 also zeroes dS^T below. Rows and columns past
+              // the end of a ragged segment fall under the same mask (their LSE is +inf).
+              const int t = r - (half * 64 + ch * 16);
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t keep = t <= 2 * kk ? 0xffffffffu : (t == 2 * kk + 1 ? 0xffff0000u : 0u);
+                pp[ch >> 1][(ch & 1) * 8 + kk] &= keep;
+              }
+            }
             if (ch & 1) tmem_st16(tS + (ch >> 1) * 32, pp[ch >> 1]);  // columns [32g, 32g + 32) -> packed [32g, +16)
             if (tid == 0) NSP_TRACE_STAMP(16 + (ch >> 1));
           }
@@ -634,7 +648,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           for (int i = 0; i < 4; ++i) aux[0][i] = lds128(delta_s + 4 * i);
           oks = mbar_wait(&s.bar_dp_full, cs & 1);
           oks = __all_sync(0xffffffffu, oks);
-          if (!oks) { where = kWhereBwdDp; break; }
+          if (!oks) { where = kWhereBwdDp; return false; }
           tc_fence_after_sync();
           if (tid == 0) NSP_TRACE_STAMP(8);
           uint32_t dpv[2][16];
@@ -666,8 +680,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             *reinterpret_cast<uint4*>(ds_row + ((2 * ch) ^ (r & 7)) * 16) = make_uint4(dsp[0], dsp[1], dsp[2], dsp[3]);
             *reinterpret_cast<uint4*>(ds_row + ((2 * ch + 1) ^ (r & 7)) * 16) = make_uint4(dsp[4], dsp[5], dsp[6], dsp[7]);
           }
+          return true;
+        };
+        if (mode == 0 && m != c.n) {
+          if (!common_step(std::false_type{})) break;
+        } else if (mode == 0) {
+          if (!common_step(std::true_type{})) break;
         } else {
-          // ---- rare step (diagonal tile and/or one of the two first-tile passes): compact rolled loops, 16 query
+          // ---- rare step (one of the two first-tile passes): compact rolled loops, 16 query
           // columns at a time; P^T and dS^T are handed over together at the end.
           oks = mbar_wait(&s.bar_dp_full, cs & 1);
           oks = __all_sync(0xffffffffu, oks);
