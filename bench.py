@@ -280,6 +280,13 @@ def main():
             "frac_of_burst_peak": achieved / peaks["burst"], "burst_peak": peaks["burst"],
             "launch_ms": bwd_ms, "flops_per_launch": f_bwd,
         }
+        fwd_ms = statistics.mean(k_fwd)
+        roofline_fwd = {
+            "kernel": "fwd_kernel", "bound": "tensor", "achieved": f_fwd / (fwd_ms * 1e-3) / 1e12, "peak": peaks["sustained"],
+            "unit": "TFLOP/s", "frac": f_fwd / (fwd_ms * 1e-3) / 1e12 / peaks["sustained"],
+            "frac_of_burst_peak": f_fwd / (fwd_ms * 1e-3) / 1e12 / peaks["burst"], "launch_ms": fwd_ms,
+            "flops_per_launch": f_fwd,
+        }
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
             tf, dt, cores, desc = run_oracle_sample(w)
@@ -293,7 +300,7 @@ def main():
                        "longest_segment": int(w.lengths.max()), "head_dim": w.head_dim, "note": w.note,
                        "grad_dtypes": "dQ bf16, dK/dV fp32", "l2": "inputs exceed L2 (no flush needed)",
                        "parallelism": "replicas" if world > 1 else "1 GPU"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "roofline_fwd": roofline_fwd, "cpu_baseline": cpu,
             "fraction_of_burst_peak": value / world / peaks["burst"],
             "fraction_of_sustained_peak": value / world / peaks["sustained"],
             "kernels_ms": {"fwd": statistics.mean(k_fwd), "bwd_preprocess": statistics.mean(k_pre),
