@@ -235,6 +235,14 @@ int nsp_a2a_scatter_heads(const void* src, void* dst, int64_t tokens, int32_t he
 /* Read the sticky device status {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
 int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
 
+/* Failure-detection self test: enqueues a one-warp kernel that waits, with the library's bounded wait, on a barrier
+ * nothing arrives at. After limit_clk SM cycles (1 .. 2^31; a million is well under a millisecond) the wait gives
+ * up and the kernel records NSP_ERR_DEVICE_TIMEOUT in the plan's status word, the way a stalled attention kernel
+ * would; nothing traps, the context stays usable, other plans are unaffected. nsp_device_status then reads
+ * {NSP_ERR_DEVICE_TIMEOUT, -1, 90, limit_clk / 1024} and the plan answers every later call with that code.
+ * Errors: INVALID_ARG, CUDA, or the plan's sticky status. */
+int nsp_selftest_wait_timeout(const nsp_plan_t* plan, int64_t limit_clk, void* stream);
+
 /* Kernels of the path, for nsp_plan_kernel_ms. */
 enum { NSP_KERNEL_FWD = 0, NSP_KERNEL_BWD_PRE = 1, NSP_KERNEL_BWD_MAIN = 2, NSP_KERNEL_BWD_POST = 3, NSP_KERNEL_COUNT = 4 };
 

@@ -28,6 +28,7 @@ EXPORTS = [
     "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string", "nsp_plan_set_profiling", "nsp_plan_kernel_ms",
     "nsp_attn_bwd_static", "nsp_recompute_mark", "nsp_plan_recompute_ws_bytes", "nsp_attn_bwd_recompute",
     "nsp_cost_table", "nsp_route_sp_tree", "nsp_a2a_gather_heads", "nsp_a2a_scatter_heads",
+    "nsp_selftest_wait_timeout",
 ]
 NSP_COST_BUCKETS = 16
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
@@ -90,6 +91,8 @@ def lib() -> ctypes.CDLL:
             f.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                           ctypes.c_int32, vp, vp]
             f.restype = ctypes.c_int
+        L.nsp_selftest_wait_timeout.argtypes = [vp, ctypes.c_int64, vp]
+        L.nsp_selftest_wait_timeout.restype = ctypes.c_int
         L.nsp_device_status.argtypes = [vp, i32p]
         L.nsp_device_status.restype = ctypes.c_int
         L.nsp_launch_count.argtypes = []
@@ -336,6 +339,13 @@ def nsp_attn_bwd_recompute(plan: Plan, recompute, q, k, v, o, d_o, lse, dq, dk, 
                                       float(softmax_scale), _ptr(ws), ws_bytes, _stream_ptr(stream))
     if rc != NSP_OK:
         raise NspError(rc, "nsp_attn_bwd_recompute")
+
+
+def nsp_selftest_wait_timeout(plan: Plan, limit_clk: int = 1_000_000, stream=None):
+    """Let one bounded device-side wait run out on purpose; the plan's status word then holds NSP_ERR_DEVICE_TIMEOUT."""
+    rc = lib().nsp_selftest_wait_timeout(plan.handle, int(limit_clk), _stream_ptr(stream))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_selftest_wait_timeout")
 
 
 def nsp_device_status(plan: Plan):

@@ -9,6 +9,7 @@
 #include <vector>
 #include <cuda_bf16.h>
 #include "nsp_internal.cuh"
+#include "sm100_ptx.cuh"
 
 namespace nsp {
 static std::atomic<int64_t> g_launches{0};
@@ -547,6 +548,29 @@ int nsp_recompute_mark(const int32_t* cu_seqlens, const int32_t* hq, const int32
   }
   if (saved_bytes) *saved_bytes = used;
   return NSP_OK;
+}
+
+namespace {
+// One warp waits on a barrier nothing ever arrives at; the bounded wait runs out after limit_clk SM cycles and the
+// warp records it in the status word exactly as the attention kernels would.
+__global__ void selftest_wait_kernel(int32_t* status, long long limit_clk) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
+  const bool ok = mbar_wait(&bar, 0, limit_clk);
+  if (!ok && threadIdx.x == 0) report_timeout(status, -1, kWhereSelfTest, static_cast<int32_t>(limit_clk >> 10));
+}
+}  // namespace
+
+int nsp_selftest_wait_timeout(const nsp_plan_t* plan, int64_t limit_clk, void* stream) {
+  if (!plan || limit_clk < 1 || limit_clk > (1ll << 31)) return NSP_ERR_INVALID_ARG;
+  if (plan->sticky) return plan->sticky;
+  selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(plan->d_status, limit_clk);
+  count_launches(1);
+  return cudaGetLastError() == cudaSuccess ? NSP_OK : NSP_ERR_CUDA;
 }
 
 int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]) {

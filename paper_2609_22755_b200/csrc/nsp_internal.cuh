@@ -64,6 +64,7 @@ enum DeviceWhere : int32_t {
   kWhereBwdDsReady = 24,
   kWhereBwdItemBarrier = 25,
   kWhereBwdTmemBase = 26,
+  kWhereSelfTest = 90,
 };
 
 __device__ __forceinline__ void report_timeout(int32_t* status, int32_t item, int32_t where, int32_t aux) {

@@ -189,6 +189,22 @@ def test_routed_shards_run_through_the_kernels(env):
         _full_case(env, w)
 
 
+def test_bounded_wait_runs_out_and_is_reported(env):
+    """Failure detection without a fault: a one-warp kernel waits on a barrier nothing arrives at; the library's
+    bounded wait gives up, the status word carries the record, the plan refuses further work, and the context is
+    still good for another plan."""
+    B, W, P = env["B"], env["W"], env["P"]
+    w = W.config(1)
+    run = P.GpuRun(w)
+    B.nsp_selftest_wait_timeout(run.plan, 1_000_000)
+    code, item, where, aux = B.nsp_device_status(run.plan)
+    assert (code, item, where, aux) == (B.NSP_ERR_DEVICE_TIMEOUT, -1, 90, 1_000_000 >> 10)
+    with pytest.raises(B.NspError) as e:
+        run.forward()
+    assert e.value.code == B.NSP_ERR_DEVICE_TIMEOUT
+    _full_case(env, w)  # a fresh plan on the same context runs and matches the oracle
+
+
 def test_empty_and_degenerate_batches(env):
     B, W, P, torch = env["B"], env["W"], env["P"], env["torch"]
     # no segments at all
