@@ -189,6 +189,37 @@ def test_routed_shards_run_through_the_kernels(env):
         _full_case(env, w)
 
 
+def test_one_gpu_of_a_routed_batch_with_recomputation(env):
+    """The pieces in the order an iteration uses them, for the first GPU of an eight-GPU tree at reduced scale: route
+    the batch (cost table, Algorithm 1), take the GPU's shard, mark its segments under an activation budget that
+    holds the root segment only, run forward, drop O and LSE of the marked segments, run the recomputing backward,
+    compare with the oracle."""
+    torch, P, B, W = env["torch"], env["P"], env["B"], env["W"]
+    from paper_2609_22755_b200 import planner
+
+    tail = W.lognormal_lengths(7, 8 * 2048 - 12288, 48, 1.3, 16, 1024)
+    lengths = [12288] + tail
+    r = planner.route_batch(lengths, 4, 2300, prefix_k=6, beam_w=4)
+    w = r["shards"][0]
+    level = np.asarray([int(r["level"][j]) for j in r["sample_ids"][0]], dtype=np.int32)
+    root_bytes = int(w.lengths[0]) * int(w.hq[0]) * (2 * w.head_dim + 4)
+    flags, saved = B.nsp_recompute_mark(w.cu_seqlens, w.hq, level, root_bytes)
+    assert saved == root_bytes and flags[0] == 0 and flags[1:].all()
+    run = P.GpuRun(w)
+    run.forward()
+    qo, lo = w.q_offsets(), w.lse_offsets()
+    for s in np.nonzero(flags)[0]:
+        run.o[qo[s]:qo[s + 1]] = float("nan")
+        run.lse[lo[s]:lo[s + 1]] = float("nan")
+    ws = torch.empty(B.nsp_plan_recompute_ws_bytes(run.plan), dtype=torch.uint8, device=run.dev)
+    B.nsp_attn_bwd_recompute(run.plan, flags, run.q, run.k, run.v, run.o, run.do, run.lse, run.dq, run.dk, run.dv,
+                             w.softmax_scale, ws)
+    assert run.status()[0] == 0
+    res, ref = run.results(), P.oracle_full(w, run.host)
+    for name in ("dq", "dk", "dv"):
+        P.check(f"{w.name}:{name}", res[name], ref[name])
+
+
 def test_bounded_wait_runs_out_and_is_reported(env):
     """Failure detection without a fault: a one-warp kernel waits on a barrier nothing arrives at; the library's
     bounded wait gives up, the status word carries the record, the plan refuses further work, and the context is
