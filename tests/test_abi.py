@@ -91,3 +91,31 @@ def test_no_device_means_an_error_not_a_fallback(B):
     if torch.cuda.is_available():
         pytest.skip("a device is present")
     assert _plan_rc(B, [0, 4, 9], [4, 4], [2, 2]) in (B.NSP_ERR_CUDA, B.NSP_ERR_UNSUPPORTED)
+
+
+def test_layout_and_selftest_calls_reject_bad_arguments_without_a_device(B):
+    lib = ctypes.CDLL(str(B.LIB_PATH))
+    fh = (ctypes.c_int32 * 4)(0, 2, 4, 6)
+    buf = ctypes.c_void_p(256)  # never dereferenced: every case below is refused first
+    for fn in (lib.nsp_a2a_gather_heads, lib.nsp_a2a_scatter_heads):
+        fn.restype = ctypes.c_int
+        fn.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                       ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+        args = lambda **kw: [kw.get("src", buf), kw.get("dst", buf), kw.get("tokens", 8), kw.get("heads", 8),
+                             kw.get("hpb", 2), kw.get("n", 4), kw.get("D", 128), kw.get("dtype", B.NSP_BF16),
+                             kw.get("fh", fh), None]
+        assert fn(*args(tokens=-1)) == B.NSP_ERR_INVALID_ARG
+        assert fn(*args(hpb=0)) == B.NSP_ERR_INVALID_ARG
+        assert fn(*args(hpb=3)) == B.NSP_ERR_INVALID_ARG  # block 3 would reach past the last head
+        assert fn(*args(n=65)) == B.NSP_ERR_INVALID_ARG
+        assert fn(*args(dtype=7)) == B.NSP_ERR_INVALID_ARG
+        assert fn(*args(fh=None)) == B.NSP_ERR_INVALID_ARG
+        assert fn(*args(D=4)) == B.NSP_ERR_UNSUPPORTED  # 8-byte rows
+        assert fn(*args(src=ctypes.c_void_p(260))) == B.NSP_ERR_INVALID_ARG  # misaligned
+        assert fn(*args(src=None)) == B.NSP_ERR_INVALID_ARG
+        assert fn(*args(tokens=0, src=None, dst=None)) == B.NSP_OK  # nothing to move
+    lib.nsp_selftest_wait_timeout.restype = ctypes.c_int
+    lib.nsp_selftest_wait_timeout.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
+    assert lib.nsp_selftest_wait_timeout(None, 1000, None) == B.NSP_ERR_INVALID_ARG
+    lib.nsp_attn_bwd_recompute.restype = ctypes.c_int
+    assert lib.nsp_plan_recompute_ws_bytes(None, None) == B.NSP_ERR_INVALID_ARG
