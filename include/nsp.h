@@ -4,13 +4,13 @@
  * nested plan.
  *
  * Where the operation comes from (paper sections):
- *   - Sec. 2.2 "Sequence Parallelism": after the Ulysses all-to-all a GPU holds the FULL-length sequence for
+ *   - Sec. 2.1, paragraph "Sequence Parallelism": after the Ulysses all-to-all a GPU holds the FULL-length sequence for
  *     H/d of the heads (d = the sequence's SP degree) and attends locally, with no communication.
- *   - Sec. 2.3 "Sequence Packing": a batch is a token budget of packed variable-length segments that never
+ *   - Sec. 2.2 "Sequence Packing": a batch is a token budget of packed variable-length segments that never
  *     attend to one another.
- *   - Sec. 4.1 (Def. 1, SP tree) and Sec. 4.2 "Tree level": a GPU takes part in every node of its
+ *   - Sec. 4.1.1 (Def. 1, SP tree) and Sec. 4.1.2 "Tree level": a GPU takes part in every node of its
  *     leaf-to-root chain, so one GPU's share mixes segments of different degrees, i.e. different head counts.
- *   - Sec. 4.2 "SP-backend level": the compute phase T^comp exists separately for forward and backward; this
+ *   - Sec. 4.1.2 "SP-backend level": the compute phase T^comp exists separately for forward and backward; this
  *     library is that phase. The paper hands it to standard softmax-attention kernels and prints no formula,
  *     so the semantics are the textbook ones:
  *         S_ij = scale * <Q[i,h], K[j,g]>  (j <= i, diagonal included; g = h / (Hq/Hkv), contiguous groups)
@@ -33,7 +33,10 @@
  * Outputs are fully overwritten. A plan may be in use by one stream at a time.
  *
  * Errors: every function returns an NSP_* code; nothing throws, aborts or traps. Device-side problems (a bounded
- * wait that ran out) are recorded in a sticky per-plan status word that nsp_device_status reads.
+ * wait that ran out) are recorded by the failing kernel in a per-plan status record that lives in device memory and in
+ * mapped pinned host memory. Every call that takes the plan looks at the host copy first (a host load, no
+ * synchronisation) and, once it is set, answers with that code and enqueues nothing: the failure surfaces at the
+ * first call made after the failing kernel has written it. nsp_device_status synchronises and returns the record.
  * There is no CPU fallback: without a CUDA device the compute calls return NSP_ERR_CUDA.
  */
 #ifndef NSP_H_
@@ -57,7 +60,9 @@ enum {
   NSP_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (including: no device) */
   NSP_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait expired (sticky, see nsp_device_status) */
   NSP_ERR_WORKSPACE = 6,      /* workspace pointer null/misaligned or ws_bytes too small */
-  NSP_ERR_INFEASIBLE = 7      /* nsp_route_sp_tree: no placement of the searched prefix fits the token budget */
+  NSP_ERR_DEVICE_ASSERT = 7,  /* an index check inside a kernel failed (only the checked build, libnsp_checked.so,
+                                 contains such checks; sticky like DEVICE_TIMEOUT) */
+  NSP_ERR_INFEASIBLE = 8      /* nsp_route_sp_tree: no placement of the searched prefix fits the token budget */
 };
 
 enum { NSP_BF16 = 0, NSP_F32 = 1 }; /* output dtypes of the gradients */
@@ -77,7 +82,7 @@ typedef struct {
 
 /*
  * Build the device-side work lists for one packed batch (the in-GPU counterpart of the paper's per-node
- * issue order, Sec. 5.1; the paper balances across GPUs, this list balances the SMs of one GPU).
+ * issue order, Sec. 4.2.1 "Inter-level Phase Streaming"; the paper balances across GPUs, this list balances the SMs of one GPU).
  *   forward  item (s, h, m), h in [0,hq[s]), m in [0, ceil(L_s/bm)):  cost = ceil(min(L_s,(m+1)*bm) / bn)
  *   backward item (s, g, n), g in [0,hkv[s]), n in [0, ceil(L_s/bn)): cost = (hq[s]/hkv[s]) * (ceil(L_s/bm) - floor(n*bn/bm))
  *   order: cost descending, then seg, tile, head ascending (a total order: the list is unique).
@@ -96,14 +101,15 @@ int nsp_plan_sizes(const nsp_plan_t* plan, int64_t* q_elems, int64_t* kv_elems, 
                    size_t* fwd_ws_bytes, size_t* bwd_ws_bytes);
 
 /* Copy a work list to the host (pass 0 = forward, 1 = backward: the lists defined above, bit-exact; pass 2 = the
- * backward items in the order the backward kernel actually walks them: the same items grouped by (segment, kv
- * head), longer segments first, key tiles ascending inside a group, which keeps the dQ accumulator rows of a q
- * tile in L2 while all key tiles of the group add to them). Writes min(cap, n) items, stores n in *n_items
- * (host_out may be NULL to query). Synchronises the plan's build stream. */
+ * backward items in the order the backward kernel actually walks them, a permutation of pass 1 that is just as
+ * unique: the (segment, kv head) groups by segment length descending, then segment, then kv head ascending; inside a
+ * group the key tiles ascending. Group-major order keeps the dQ accumulator rows of a q tile in L2 while all key tiles
+ * of the group add to them. Writes min(cap, n) items, stores n in *n_items (host_out may be NULL to query). The lists
+ * were complete when nsp_plan_tiles returned; this call only copies. */
 int nsp_plan_get(const nsp_plan_t* plan, int pass, nsp_tile_t* host_out, int64_t cap, int64_t* n_items);
 
 /*
- * Forward (paper Sec. 4.2, T^comp,fwd of every node on this GPU's chain, in one launch).
+ * Forward (paper Sec. 4.1.2, T^comp,fwd of every node on this GPU's chain, in one launch).
  * q [q_elems] bf16, k/v [kv_elems] bf16 (device, read-only); o [q_elems] bf16 and lse [lse_elems] fp32 (device,
  * written). softmax_scale: finite, > 0. ws / ws_bytes: device workspace of at least fwd_ws_bytes (may be NULL
  * when that is 0). Errors: INVALID_ARG, WORKSPACE, CUDA, DEVICE_TIMEOUT (sticky status from an earlier call).
@@ -112,7 +118,7 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
                  float softmax_scale, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * Backward (paper Sec. 4.2, T^comp,bwd). Inputs: q, k, v, o, d_o (bf16) and lse (fp32) as produced by
+ * Backward (paper Sec. 4.1.2, T^comp,bwd). Inputs: q, k, v, o, d_o (bf16) and lse (fp32) as produced by
  * nsp_attn_fwd. Outputs: dq [q_elems], dk/dv [kv_elems] in dq_dtype / dkv_dtype (NSP_BF16 or NSP_F32);
  * dk/dv hold the sum over the hq/hkv query heads that share a KV head on THIS GPU (with a replicated KV head
  * at high degree the cross-GPU sum belongs to the epilogue collective, outside this library).
@@ -146,7 +152,7 @@ int nsp_attn_bwd_static(const nsp_plan_t* plan, const void* q, const void* k, co
                         float softmax_scale, void* stream);
 
 /*
- * Tree-level recomputation (paper Sec. 4.2, "Tree-Level Recomputation"): the backward pass of a shard in which the
+ * Tree-level recomputation (paper Sec. 4.2.2 "Tree-Level Recomputation"): the backward pass of a shard in which the
  * attention output of some segments was not kept after the forward pass.
  *
  * nsp_recompute_mark derives the save / recompute marking of this GPU's segments from an activation budget, the way
@@ -176,7 +182,8 @@ int nsp_attn_bwd_recompute(const nsp_plan_t* plan, const uint8_t* recompute, con
                            void* stream);
 
 /*
- * Planner (paper Sec. 4.2, "Routing Objective and Cost Model" and Algorithm 1, "Prefix-Completion SP-Tree Routing").
+ * Planner (paper Sec. 4.1.2 "Routing Objective and Cost Model" and Sec. 4.1.3, Algorithm 1 "Prefix-Completion SP-Tree
+ * Routing").
  * Host only, no CUDA call.
  *
  * The SP tree is the full binary tree over P = 2^(n_levels-1) GPUs: node (l, i) covers GPUs [i*2^l, (i+1)*2^l) and
@@ -212,8 +219,8 @@ int nsp_route_sp_tree(const int32_t* lengths, const int64_t* cost, int32_t n_sam
                       int32_t* index_out, int64_t* load_out, int64_t* tok_out, int32_t* feasible_out);
 
 /*
- * Layout steps of the Ulysses all-to-all around the attention compute (paper Sec. 2.2; the prologue and epilogue
- * phases of a tree node, Sec. 4.2). The exchange itself (NCCL send / receive between the GPUs of the node) is issued
+ * Layout steps of the Ulysses all-to-all around the attention compute (paper Sec. 2.1; the prologue and epilogue
+ * phases of a tree node, Sec. 4.1.2). The exchange itself (NCCL send / receive between the GPUs of the node) is issued
  * by the caller; see ulysses.py for the schedule. Tensors are device pointers, rows of head_dim elements of dtype
  * NSP_BF16 or NSP_F32, head_dim * element size a multiple of 16 bytes, pointers 16-byte aligned; first_head is a
  * host array [n_blocks], n_blocks <= NSP_A2A_MAX_PEERS.
@@ -232,7 +239,7 @@ int nsp_a2a_gather_heads(const void* src, void* dst, int64_t tokens, int32_t hea
 int nsp_a2a_scatter_heads(const void* src, void* dst, int64_t tokens, int32_t heads, int32_t heads_per_block,
                           int32_t n_blocks, int32_t head_dim, int32_t dtype, const int32_t* first_head, void* stream);
 
-/* Read the sticky device status {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
+/* Read the device status record {code, item, where, aux}; code 0 = healthy. Synchronises the device. */
 int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
 
 /* Failure-detection self test: enqueues a one-warp kernel that waits, with the library's bounded wait, on a barrier
@@ -246,7 +253,7 @@ int nsp_selftest_wait_timeout(const nsp_plan_t* plan, int64_t limit_clk, void* s
 /* Kernels of the path, for nsp_plan_kernel_ms. */
 enum { NSP_KERNEL_FWD = 0, NSP_KERNEL_BWD_PRE = 1, NSP_KERNEL_BWD_MAIN = 2, NSP_KERNEL_BWD_POST = 3, NSP_KERNEL_COUNT = 4 };
 
-/* Measurement aid (the paper's cost model is fed by offline profiles of the compute phase, Sec. 4.2): when
+/* Measurement aid (the paper's cost model is fed by offline profiles of the compute phase, Sec. 4.1.2): when
  * enabled, every later nsp_attn_fwd / nsp_attn_bwd on this plan brackets each of its kernels with a pair of CUDA
  * events recorded on the launching stream. Errors: INVALID_ARG (null plan), CUDA. */
 int nsp_plan_set_profiling(nsp_plan_t* plan, int enable);

@@ -162,7 +162,7 @@ def plan_tiles(cu, hq, hkv, bm=128, bn=128, pass_=0):
 
 
 def recompute_mark(lengths, hq, level, budget_bytes, head_dim=128):
-    """Save / recompute marking of one GPU's segments (paper Sec. 4.2, "Tree-Level Recomputation"): walk the tree
+    """Save / recompute marking of one GPU's segments (paper Sec. 4.2.2 "Tree-Level Recomputation"): walk the tree
     from the upper levels toward the leaves, add up the bytes of the attention-output slices that are saved, and
     once the budget is reached mark everything that is left for recomputation; inside the level where the cut
     falls, the samples that cost more to recompute are saved first.
@@ -251,7 +251,7 @@ def route_sp_tree(lengths, cost, n_levels, k, w, b_tok, monotone=False):
 
 
 def cost_table(lengths, n_levels, hq, hkv, head_dim, tcomp_ns, link_gbs, other_ns_per_token):
-    """The paper's hierarchical cost model (Sec. 4.2) for one sample on a level-l node, per covered GPU, forward +
+    """The paper's hierarchical cost model (Sec. 4.1.2) for one sample on a level-l node, per covered GPU, forward +
     backward, in nanoseconds: SP-backend level = compute (causal pairs x local q heads x profiled ns per pair and
     head for the sample's length class) + prologue / epilogue all-to-alls (the (d-1)/d share of the GPU's L/d
     tokens; Q, K, V in and O out, both passes, bf16) over the level's link bandwidth; model level = non-attention

@@ -5,9 +5,9 @@
  * this file. It shares no code, header, table or helper with the CUDA library and never calls it.
  *
  * What it evaluates is the plain definition of the local attention compute phase of an Ulysses-style
- * sequence-parallel backend (paper Sec. 2.2 "Sequence Parallelism": after the all-to-all every GPU holds
- * complete sequences for a subset of heads and attends locally; Sec. 2.3 "Sequence Packing": packed segments
- * never attend to one another; Sec. 4.2 "SP-backend level": the compute phase exists for forward and for
+ * sequence-parallel backend (paper Sec. 2.1, paragraph "Sequence Parallelism": after the all-to-all every GPU holds
+ * complete sequences for a subset of heads and attends locally; Sec. 2.2 "Sequence Packing": packed segments
+ * never attend to one another; Sec. 4.1.2 "SP-backend level": the compute phase exists for forward and for
  * backward). The paper delegates the arithmetic to standard softmax attention kernels and prints no
  * formula of its own, so the oracle is the textbook definition written out, in double precision:
  *
@@ -442,7 +442,7 @@ int orc_attn_cols(const void* q, const void* k, const void* v, const void* d_o, 
 
 /* ------------------------------------------------------------------------------------------------ tile plan
  * Work list of the in-GPU schedule (the paper balances load across GPUs and issues a GPU's nodes one after
- * the other, Sec. 5.1; the in-GPU list is this build's reading). Tile sizes bm (query rows), bn (key rows).
+ * the other, Sec. 4.2.1; the in-GPU list is this build's reading). Tile sizes bm (query rows), bn (key rows).
  *   pass 0 (forward):  one item per (segment s, q head h, q tile m);  cost = ceil(min(L, (m+1)*bm) / bn),
  *                      the number of key tiles the q tile visits.
  *   pass 1 (backward): one item per (segment s, kv head g, key tile n); cost = G * (Mt - floor(n*bn / bm)),

@@ -18,7 +18,8 @@ NSP_ERR_ALLOC = 3
 NSP_ERR_CUDA = 4
 NSP_ERR_DEVICE_TIMEOUT = 5
 NSP_ERR_WORKSPACE = 6
-NSP_ERR_INFEASIBLE = 7
+NSP_ERR_DEVICE_ASSERT = 7
+NSP_ERR_INFEASIBLE = 8
 NSP_BF16 = 0
 NSP_F32 = 1
 NSP_MAX_RUNS = 32

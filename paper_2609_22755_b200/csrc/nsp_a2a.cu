@@ -1,4 +1,4 @@
-// Layout kernels of the Ulysses all-to-all around the attention compute (paper Sec. 2.2 and Sec. 4.2, the prologue /
+// Layout kernels of the Ulysses all-to-all around the attention compute (paper Sec. 2.1 and Sec. 4.1.2, the prologue /
 // epilogue phases of an SP-tree node). HBM-bound copies: 16 bytes per thread and access, rows of head_dim elements.
 //
 // Before the prologue a GPU of a degree-d node holds its 1/d token slice of the node's samples with ALL heads,

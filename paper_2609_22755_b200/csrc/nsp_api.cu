@@ -33,7 +33,8 @@ struct nsp_plan {
   int32_t* d_front = nullptr;        // [n_bwd / kFrontBlock + 1] start-alignment counters of the backward kernel
   int32_t* d_counters = nullptr;  // [0] forward cursor, [1] backward cursor
   int32_t* d_status = nullptr;    // {code, item, where, aux}
-  cudaStream_t build_stream = nullptr;
+  int32_t* h_status = nullptr;    // the same record in mapped pinned host memory (written by the failing kernel)
+  int32_t* h_status_dev = nullptr;  // device pointer to h_status
   int sticky = 0;
   // optional per-kernel timing (CUDA events on the launching stream)
   bool profiling = false;
@@ -79,17 +80,18 @@ bool encode_run_map(CUtensorMap* out, const void* base, int64_t elem_off, int64_
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Order in which the backward kernel walks its work items. The published work list (nsp_plan_get, pass 1) is
-// sorted by cost alone; walked in that order, the CTAs that run at the same time hold key tiles of MANY (segment,
+// Order in which the backward kernel walks its work items (nsp_plan_get, pass 2). The published work list (pass 1)
+// is sorted by cost alone; walked in that order, the CTAs that run at the same time hold key tiles of MANY (segment,
 // kv head) groups, a q tile's fp32 dQ accumulator rows are touched by a few CTAs now and by the others much later,
 // and they travel to DRAM and back every time (16 segments of 8,192 tokens, 32q/4kv: 193 GB of DRAM traffic for a
 // backward pass whose tensors total 5 GB, L2 hit rate 21 %, the kernel runs at HBM speed). Walked group by group
 // -- all key tiles of one (segment, kv head), first key tile (largest cost) first -- the CTAs of a group sweep the q
 // tiles together and every accumulator row, Q tile and dO tile is fetched once per group. Groups go by segment
-// length descending: all CTAs then start the longest group at the same moment, which is what keeps them on the same
-// q tile (started after a tail of shorter groups they enter it scattered and stay scattered: 131,072 tokens at
-// 16q/1kv next to 131,072 tokens of shorter segments ran 4 % slower that way, a long-tailed batch 8 %), and the walk
-// ends with the cheapest items of the shortest segments. Same items, same costs: a permutation of the published list.
+// length descending (ties: segment, then kv head, ascending): all CTAs then start the longest group at the same
+// moment, which is what keeps them on the same q tile (started after a tail of shorter groups they enter it scattered
+// and stay scattered: 131,072 tokens at 16q/1kv next to 131,072 tokens of shorter segments ran 4 % slower that way, a
+// long-tailed batch 8 %), and the walk ends with the cheapest items of the shortest segments. Same items, same
+// costs: a permutation of the published list.
 std::vector<nsp_tile_t> build_bwd_exec_order(const std::vector<SegInfo>& seg, int bm, int bn) {
   struct Group { int32_t len, s, g; };
   std::vector<Group> groups;
@@ -110,6 +112,18 @@ std::vector<nsp_tile_t> build_bwd_exec_order(const std::vector<SegInfo>& seg, in
   return out;
 }
 
+// The plan's failure state: set once a kernel of the plan has recorded a failure. The record sits in mapped pinned
+// host memory, so looking at it costs a host load, not a synchronisation; a failure is seen by the first call made
+// after the failing kernel wrote it.
+int plan_failed(const nsp_plan* plan) {
+  if (!plan->sticky && plan->h_status) {
+    const int code = *reinterpret_cast<volatile int32_t*>(plan->h_status);
+    if (code != 0) const_cast<nsp_plan*>(plan)->sticky = code;
+  }
+  return plan->sticky;
+}
+StatusWord status_word(const nsp_plan* plan) { return StatusWord{plan->d_status, plan->h_status_dev}; }
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -123,6 +137,7 @@ void free_plan(nsp_plan* p) {
   cudaFree(p->d_front);
   cudaFree(p->d_counters);
   cudaFree(p->d_status);
+  if (p->h_status) cudaFreeHost(p->h_status);
   for (cudaEvent_t e : p->ev)
     if (e) cudaEventDestroy(e);
   delete p;
@@ -149,6 +164,7 @@ const char* nsp_status_string(int code) {
     case NSP_ERR_CUDA: return "CUDA call failed";
     case NSP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
     case NSP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case NSP_ERR_DEVICE_ASSERT: return "device-side index check failed (checked build)";
     case NSP_ERR_INFEASIBLE: return "no plan within the token budget";
     default: return "unknown status";
   }
@@ -182,7 +198,6 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
   p->n_seg = n_seg;
   p->bm = bm;
   p->bn = bn;
-  p->build_stream = static_cast<cudaStream_t>(stream);
   std::vector<int64_t> row_base, fwd_base, bwd_base;
   try {
     p->seg.resize(n_seg);
@@ -263,7 +278,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     delete p;
     return NSP_ERR_UNSUPPORTED;
   }
-  cudaStream_t st = p->build_stream;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
   int64_t* d_bases = nullptr;
   uint64_t* d_keys = nullptr;
   void* d_tmp = nullptr;
@@ -278,8 +293,20 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
   A(reinterpret_cast<void**>(&p->d_bwd), sizeof(nsp_tile_t) * nb);
   A(reinterpret_cast<void**>(&p->d_bwd_exec), sizeof(nsp_tile_t) * nb);
   A(reinterpret_cast<void**>(&p->d_front), sizeof(int32_t) * (nb / kFrontBlock + 1));
-  A(reinterpret_cast<void**>(&p->d_counters), 2 * sizeof(int32_t));
+  A(reinterpret_cast<void**>(&p->d_counters), 4 * sizeof(int32_t));
   A(reinterpret_cast<void**>(&p->d_status), 4 * sizeof(int32_t));
+  if (okc) {
+    void* hp = nullptr;
+    void* dp = nullptr;
+    if (cudaHostAlloc(&hp, 4 * sizeof(int32_t), cudaHostAllocMapped) != cudaSuccess) {
+      okc = false;
+    } else {
+      p->h_status = static_cast<int32_t*>(hp);
+      std::memset(hp, 0, 4 * sizeof(int32_t));
+      if (cudaHostGetDevicePointer(&dp, hp, 0) != cudaSuccess) okc = false;
+      p->h_status_dev = static_cast<int32_t*>(dp);
+    }
+  }
   A(reinterpret_cast<void**>(&d_bases), 2 * sizeof(int64_t) * (n_seg + 1));
   A(reinterpret_cast<void**>(&d_keys), 2 * sizeof(uint64_t) * (nf + nb));
   A(&d_tmp, tmp_bytes);
@@ -292,7 +319,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     auto C = [&](cudaError_t x) {
       if (e == cudaSuccess) e = x;
     };
-    C(cudaMemsetAsync(p->d_counters, 0, 2 * sizeof(int32_t), st));
+    C(cudaMemsetAsync(p->d_counters, 0, 4 * sizeof(int32_t), st));
     C(cudaMemsetAsync(p->d_status, 0, 4 * sizeof(int32_t), st));
     if (n_seg > 0) {
       C(cudaMemcpyAsync(p->d_seg, p->seg.data(), sizeof(SegInfo) * n_seg, cudaMemcpyHostToDevice, st));
@@ -338,7 +365,6 @@ int nsp_plan_get(const nsp_plan_t* plan, int pass, nsp_tile_t* host_out, int64_t
   *n_items = n;
   if (!host_out || cap == 0 || n == 0) return NSP_OK;
   const int64_t m = cap < n ? cap : n;
-  if (cudaStreamSynchronize(plan->build_stream) != cudaSuccess) return NSP_ERR_CUDA;
   const nsp_tile_t* src = pass == 0 ? plan->d_fwd : (pass == 1 ? plan->d_bwd : plan->d_bwd_exec);
   if (cudaMemcpy(host_out, src, sizeof(nsp_tile_t) * m, cudaMemcpyDeviceToHost) !=
       cudaSuccess)
@@ -351,7 +377,7 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   (void)ws;
   (void)ws_bytes;
   if (!plan) return NSP_ERR_INVALID_ARG;
-  if (plan->sticky) return plan->sticky;
+  if (const int failed = plan_failed(plan)) return failed;
   if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return NSP_ERR_INVALID_ARG;
   if (plan->n_fwd == 0) return NSP_OK;
   if (!q || !k || !v || !o || !lse) return NSP_ERR_INVALID_ARG;
@@ -372,7 +398,7 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.items = plan->d_fwd;
   a.n_items = static_cast<int32_t>(plan->n_fwd);
   a.counter = plan->d_counters;
-  a.status = plan->d_status;
+  a.status = status_word(plan);
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
@@ -399,7 +425,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
              const void* o, const void* d_o, const float* lse, void* dq, void* dk, void* dv, int dq_dtype,
              int dkv_dtype, float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
   if (!plan) return NSP_ERR_INVALID_ARG;
-  if (plan->sticky) return plan->sticky;
+  if (const int failed = plan_failed(plan)) return failed;
   if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return NSP_ERR_INVALID_ARG;
   if ((dq_dtype != NSP_BF16 && dq_dtype != NSP_F32) || (dkv_dtype != NSP_BF16 && dkv_dtype != NSP_F32))
     return NSP_ERR_INVALID_ARG;
@@ -447,7 +473,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
     fa.items = plan->d_fwd;
     fa.n_items = static_cast<int32_t>(plan->n_fwd);
     fa.counter = plan->d_counters;
-    fa.status = plan->d_status;
+    fa.status = status_word(plan);
     fa.o = nullptr;
     fa.lse = lse_ws;
     fa.scale_log2 = softmax_scale * 1.4426950408889634f;
@@ -470,7 +496,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   a.items = plan->d_bwd_exec;
   a.n_items = static_cast<int32_t>(plan->n_bwd);
   a.counter = plan->d_counters + 1;
-  a.status = plan->d_status;
+  a.status = status_word(plan);
   a.lse = recompute ? lse_ws : lse;
   a.delta = delta;
   a.dq_acc = dq_acc;
@@ -480,10 +506,6 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   a.dkv_f32 = dkv_dtype == NSP_F32;
   a.scale = softmax_scale;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
-  {
-    const char* dbg = std::getenv("NSP_DEBUG_FLAGS");
-    a.debug_flags = dbg ? std::atoi(dbg) : 0;
-  }
   prof_mark(plan, NSP_KERNEL_BWD_MAIN, 0, st);
   if (launch_bwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_MAIN, 1, st);
@@ -553,7 +575,7 @@ int nsp_recompute_mark(const int32_t* cu_seqlens, const int32_t* hq, const int32
 namespace {
 // One warp waits on a barrier nothing ever arrives at; the bounded wait runs out after limit_clk SM cycles and the
 // warp records it in the status word exactly as the attention kernels would.
-__global__ void selftest_wait_kernel(int32_t* status, long long limit_clk) {
+__global__ void selftest_wait_kernel(StatusWord status, long long limit_clk) {
   __shared__ uint64_t bar;
   if (threadIdx.x == 0) {
     mbar_init(&bar, 1);
@@ -567,8 +589,8 @@ __global__ void selftest_wait_kernel(int32_t* status, long long limit_clk) {
 
 int nsp_selftest_wait_timeout(const nsp_plan_t* plan, int64_t limit_clk, void* stream) {
   if (!plan || limit_clk < 1 || limit_clk > (1ll << 31)) return NSP_ERR_INVALID_ARG;
-  if (plan->sticky) return plan->sticky;
-  selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(plan->d_status, limit_clk);
+  if (const int failed = plan_failed(plan)) return failed;
+  selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status_word(plan), limit_clk);
   count_launches(1);
   return cudaGetLastError() == cudaSuccess ? NSP_OK : NSP_ERR_CUDA;
 }
@@ -577,7 +599,7 @@ int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]) {
   if (!plan || !out) return NSP_ERR_INVALID_ARG;
   if (cudaDeviceSynchronize() != cudaSuccess) return NSP_ERR_CUDA;
   if (cudaMemcpy(out, plan->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return NSP_ERR_CUDA;
-  if (out[0] != 0) const_cast<nsp_plan_t*>(plan)->sticky = out[0];
+  if (out[0] != 0 && !plan->sticky) const_cast<nsp_plan_t*>(plan)->sticky = out[0];
   return NSP_OK;
 }
 

@@ -17,7 +17,7 @@
 // TMEM: R0 [0,128), R1 [128,256), dK [256,384), dV [384,512).
 // Roles:  warps 0-7  softmax / dS (key row = TMEM lane, two column halves)
 //         warps 8-15 dQ: TMEM -> fp32 accumulator in global memory (lane quadrant x 64-column half)
-//         warp 16    TMA producer (K, V once per item; Q, dO two-stage ring)
+//         warp 16    TMA producer (K, V once per item; Q two-stage ring, dO single buffer)
 //         warp 17    MMA issuer A (single thread): dV(t), S^T(t+1)
 //         warp 18    LSE / delta loader (two-stage ring in shared memory)
 //         warp 19    MMA issuer B (single thread): dK(t), dQ^T(t), dP^T(t+1)
@@ -55,21 +55,7 @@ constexpr int kRegsSoftmax = 136, kRegsReduce = 80, kRegsAux = 48;
 constexpr int kFrontMinSteps = 2048;          // items shorter than this start at once
 constexpr int kFrontMinGroup = 8;             // so do items of groups with fewer q heads per kv head
 constexpr long long kFrontWaitClk = 1500000;  // ~0.9 ms: upper bound of the start alignment (also: 1/16 of the item)
-
-// Optional step timeline (compiled in only with -DNSP_TRACE, for tuning): clock64 stamps of the first CTA's roles.
-#ifdef NSP_TRACE
-__device__ long long g_trace[64 * 24];
-#ifndef NSP_TRACE_BASE
-#define NSP_TRACE_BASE 200
-#endif
-#define NSP_TRACE_STAMP(slot)                                                                  \
-  do {                                                                                         \
-    const uint32_t tix_ = gs + vt - NSP_TRACE_BASE;                                            \
-    if (blockIdx.x == 0 && tix_ < 64u) g_trace[tix_ * 24 + (slot)] = clock64();                \
-  } while (0)
-#else
-#define NSP_TRACE_STAMP(slot)
-#endif
+constexpr int kQStages = 2;                   // Q ring (three stages measured 3 % slower on the nested shard)
 
 // A decoded work item: written by thread 0, read by every role after the CTA-wide barrier of next_item().
 struct ItemCtx {
@@ -86,15 +72,15 @@ struct ItemCtx {
 struct BwdSmem {
   uint8_t k[2][kHalfTileBytes];
   uint8_t v[2][kHalfTileBytes];
-  uint8_t q[3][2][kHalfTileBytes];    // [stage][64-column half]: three-stage ring, loaded a whole step ahead
+  uint8_t q[kQStages][2][kHalfTileBytes];  // [stage][64-column half]: ring, loaded a whole step ahead
   uint8_t d_o[2][kHalfTileBytes];     // [half]: single buffer (its consumers leave a long window for the refill)
   uint8_t ds[2][kHalfTileBytes];      // dS^T, [key row][query col], two 64-column halves
   float lse[2][128];                  // [stage] LSE * log2(e) of the q tile (+inf for rows past the segment)
   float delta[2][128];                // [stage]
   ItemCtx ctx[2];
   uint64_t bar_kv;
-  uint64_t bar_q_full[3];
-  uint64_t bar_q_empty[3][2];  // [stage][issuer A / B]: that issuer's MMAs reading the Q stage have completed
+  uint64_t bar_q_full[kQStages];
+  uint64_t bar_q_empty[kQStages][2];  // [stage][issuer A / B]: that issuer's MMAs reading the Q stage have completed
   uint64_t bar_do_full;
   uint64_t bar_do_empty[2];    // [issuer A / B]: that issuer's MMAs reading the dO buffer have completed
   uint64_t bar_a_done;         // dV of the step (issuer A) has completed
@@ -156,12 +142,12 @@ struct StepWalk {
   }
 };
 
-// Position in the three-stage Q ring; it runs on across items. ph is the parity of the number of earlier uses of
+// Position in the Q ring; it runs on across items. ph is the parity of the number of earlier uses of
 // the current stage.
 struct QRing {
   uint32_t st = 0, ph = 0;
   __device__ __forceinline__ void next() {
-    if (++st == 3) st = 0, ph ^= 1;
+    if (++st == kQStages) st = 0, ph ^= 1;
   }
 };
 
@@ -169,14 +155,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   BwdSmem& s = *reinterpret_cast<BwdSmem*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
-  if ((smem_u32(smem_raw) & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
-    if (tid == 0) report_timeout(a.status, -1, kWhereBwdSmemAlign, 0);
-    return;
-  }
+  // swizzled tiles need a 1024-byte aligned base
+  const bool misaligned = (smem_u32(smem_raw) & 1023u) != 0;
 
   if (tid == 0) {
     mbar_init(&s.bar_kv, 1);
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < kQStages; ++i) {
       mbar_init(&s.bar_q_full[i], 1);
       mbar_init(&s.bar_q_empty[i][0], 1);
       mbar_init(&s.bar_q_empty[i][1], 1);
@@ -201,7 +185,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     s.abort = 0;
     fence_mbar_init();
   }
-  if (warp == 0) {
+  if (warp == 0 && !misaligned) {
     tmem_alloc(&s.tmem_base, kBwdTmemCols);
     tmem_relinquish();
   }
@@ -212,10 +196,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   // The CTA owns all 512 TMEM columns, so the allocation starts at column 0 and every TMEM address is a
   // compile-time constant.
   constexpr uint32_t tR0 = 0, tR1 = 128, tDK = 256, tDV = 384;
-  if (s.tmem_base != 0) {
-    if (tid == 0) report_timeout(a.status, -1, kWhereBwdTmemBase, static_cast<int32_t>(s.tmem_base));
+  if (misaligned || s.tmem_base != 0) {
+    if (tid == 0)
+      report_timeout(a.status, -1, misaligned ? kWhereBwdSmemAlign : kWhereBwdTmemBase, static_cast<int32_t>(s.tmem_base));
     __syncthreads();
-    if (warp == 0) tmem_dealloc(s.tmem_base, kBwdTmemCols);
+    if (warp == 0 && !misaligned) tmem_dealloc(s.tmem_base, kBwdTmemCols);
     return;
   }
   volatile int32_t* abort_flag = &s.abort;
@@ -238,8 +223,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         x.g = item.head, x.n = item.tile;
         x.G = sg.hq / sg.hkv;
         x.first = (item.tile == 0);
-        x.two_pass = (x.first && (a.debug_flags & 1) == 0) ? 1 : 0;
-        x.mode_first = (a.debug_flags & 2) == 0 ? 1 : 0;
+        x.two_pass = x.first;  // hi / lo split of P and dS for the first q tile
+        x.mode_first = 1;      // exact delta for the first q tile
         x.per_head = (sg.len + kBM - 1) / kBM - item.tile + x.two_pass;  // q tiles n .. Mt-1 (bm == bn)
         x.steps = x.G * x.per_head;
         // Start alignment. kFrontBlock consecutive items are neighbouring key tiles of one (segment, kv head) and
@@ -308,7 +293,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               *abort_flag = 1;
               break;
             }
-            NSP_TRACE_STAMP(14);
             mbar_expect_tx(&s.bar_q_full[qr.st], kTileBytes);
             tma_load_3d(s.q[qr.st][0], mq, &s.bar_q_full[qr.st], 0, h, c.tok0 + m * kBM);
             tma_load_3d(s.q[qr.st][1], mq, &s.bar_q_full[qr.st], 64, h, c.tok0 + m * kBM);
@@ -350,9 +334,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           int where = 0;
           bool okm = mbar_wait(&s.bar_kv, gi & 1);
           if (!okm) where = kWhereBwdLoadKV;
-          const uint32_t q0_lo = smem_u32(s.q[0][0]) >> 4, do_lo = smem_u32(s.d_o[0]) >> 4;
+          const uint32_t q0_lo = smem_desc_addr(s.q[0][0]), do_lo = smem_desc_addr(s.d_o[0]);
           if (is_a) {
-            const uint32_t k_km = (smem_u32(s.k[0]) >> 4) | lbo_km;
+            const uint32_t k_km = smem_desc_addr(s.k[0]) | lbo_km;
             // S^T of the next step not yet issued -> R0 (A = K, B = Q of the ring stage, both K-major)
             auto issue_s = [&]() -> bool {
               if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph)) { where = kWhereBwdLoadQ; return false; }
@@ -375,7 +359,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               if (*abort_flag) break;
               if (!mbar_wait(&s.bar_do_full, cs & 1)) { okm = false; where = kWhereBwdLoadQ; break; }
               if (!mbar_wait(&s.bar_p_ready, cs & 1)) { okm = false; where = kWhereBwdPReady; break; }
-              NSP_TRACE_STAMP(0);
               tc_fence_after_sync();
               const uint32_t acc = vt > 0;
               // dV += P^T dO; packed P^T columns of K-step kk (16 query columns) sit at R0 + (kk/2)*32 + (kk%2)*8
@@ -385,13 +368,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
                            acc | (kk > 0));
               umma_commit(&s.bar_a_done);       // S^T and dV of the step
               umma_commit(&s.bar_do_empty[0]);  // this thread is done with the dO buffer
-              NSP_TRACE_STAMP(15);
               if (vt + 1 < steps && !issue_s()) { okm = false; break; }
-              NSP_TRACE_STAMP(1);
             }
           } else {
-            const uint32_t v_km = (smem_u32(s.v[0]) >> 4) | lbo_km, k_mn = (smem_u32(s.k[0]) >> 4) | lbo_mn;
-            const uint32_t ds_km = (smem_u32(s.ds[0]) >> 4) | lbo_km, ds_mn = (smem_u32(s.ds[0]) >> 4) | lbo_mn;
+            const uint32_t v_km = smem_desc_addr(s.v[0]) | lbo_km, k_mn = smem_desc_addr(s.k[0]) | lbo_mn;
+            const uint32_t ds_km = smem_desc_addr(s.ds[0]) | lbo_km, ds_mn = smem_desc_addr(s.ds[0]) | lbo_mn;
             // dP^T of step vt -> R1, once the dQ warps have drained dQ^T of the previous step from it
             auto issue_dp = [&](int vt) -> bool {
               const uint32_t cs = gs + vt;
@@ -414,7 +395,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               if (*abort_flag) break;
               if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph)) { okm = false; where = kWhereBwdLoadQ; break; }
               if (!mbar_wait(&s.bar_ds_ready, cs & 1)) { okm = false; where = kWhereBwdDsReady; break; }
-              NSP_TRACE_STAMP(2);
               tc_fence_after_sync();
               const uint32_t acc = vt > 0;
               const uint32_t q_mn = (q0_lo + qr.st * kStageStep) | lbo_mn;
@@ -432,9 +412,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               umma_commit(&s.bar_b_done);              // dP^T, dQ^T and dK of the step
               umma_commit(&s.bar_q_empty[qr.st][1]);  // this thread is done with the Q stage
               qr.next();
-              NSP_TRACE_STAMP(3);
               if (vt + 1 < steps && !issue_dp(vt + 1)) { okm = false; break; }
-              NSP_TRACE_STAMP(4);
             }
           }
           if (!okm) {
@@ -504,7 +482,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           break;
         }
         tc_fence_after_sync();
-        if (warp == 8 && lane == 0) NSP_TRACE_STAMP(10);
         int h, m, mode;
         w.get(c, h, m, mode);
         w.next(c);
@@ -512,9 +489,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         // one accumulator row (128 bytes, one request). Eight warps issue them: one SM sustains about 25 bytes
         // per clock of reductions, and four warps reach only half of that. Rows past the segment end are
         // skipped (their dS^T columns are zero, and they may lie outside the buffer).
-        const int n_valid = min(kBM, c.len - m * kBM) - colhalf * 64;
-        float* p0 = a.dq_acc + c.q_off + ((static_cast<int64_t>(m) * kBM + colhalf * 64) * c.hq + h) * kHeadDim + d;
-        const bool do_red = (a.debug_flags & 4) == 0;
+        const int rows_left = c.len - m * kBM;  // valid query rows of this q tile (>= 128 for an interior tile)
+        float* const tile0 = a.dq_acc + c.q_off + (static_cast<int64_t>(m) * kBM * c.hq + h) * kHeadDim + d;
+        const int n_valid = min(kBM, rows_left) - colhalf * 64;
+        float* p0 = tile0 + colhalf * 64 * q_stride;
         if (n_valid >= 64) {  // interior tile: no row checks
           uint32_t v0[32], v1[32];
           tmem_ld32(tR1 + lane_off + colhalf * 64, v0);
@@ -522,8 +500,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           tmem_wait_ld();
           tc_fence_before_sync();
           mbar_arrive(&s.bar_dq_empty);  // R1 is drained: the next dP^T may overwrite it
-          if (warp == 8 && lane == 0) NSP_TRACE_STAMP(11);
-          if (do_red) {
+          // The reductions sit in a conditional region on purpose (the condition always holds): as straight-line
+          // code the compiler computes all 64 row addresses ahead of the TMEM loads, runs out of the 80 registers
+          // this role has and spills inside the loop (measured: the whole kernel 25 % slower).
+          if (c.hq > 0) {
             float* p1 = p0 + 32 * q_stride;
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
@@ -531,9 +511,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               red_add_f32(p1, __uint_as_float(v1[e]));
               p0 += q_stride;
               p1 += q_stride;
-#ifdef NSP_RED_PACE_NS
-              if ((e & NSP_RED_PACE_MASK) == NSP_RED_PACE_MASK) __nanosleep(NSP_RED_PACE_NS);
-#endif
             }
           }
         } else {  // ragged tail: 16 columns at a time, each row checked
@@ -548,12 +525,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             }
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              if (do_red && ch * 16 + e < n_valid) red_add_f32(p0, __uint_as_float(v[e]));
+              if (c.hq > 0 && ch * 16 + e < n_valid) red_add_f32(p0, __uint_as_float(v[e]));
               p0 += q_stride;
             }
           }
         }
-        if (warp == 8 && lane == 0) NSP_TRACE_STAMP(12);
       }
       item_done();
     }
@@ -583,7 +559,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         oks = __all_sync(0xffffffffu, oks);
         if (!oks) { where = kWhereBwdS; break; }
         tc_fence_after_sync();
-        if (tid == 0) NSP_TRACE_STAMP(5);
         const float* lse_s = s.lse[st] + half * 64;
         float* delta_s = s.delta[st] + half * 64;
         // ---- common step (interior tile; the diagonal tile runs a second copy of the same code with a mask on P,
@@ -602,7 +577,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           tmem_ld32(tS, sv[0]);
           tmem_ld32(tS + 32, sv[1]);
           tmem_wait_ld();
-          if (tid == 0) NSP_TRACE_STAMP(6);
           uint32_t pp[2][16];  // P^T as bf16 pairs: what goes to R0, and what the dS^T product uses below
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
@@ -634,13 +608,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               }
             }
             if (ch & 1) tmem_st16(tS + (ch >> 1) * 32, pp[ch >> 1]);  // columns [32g, 32g + 32) -> packed [32g, +16)
-            if (tid == 0) NSP_TRACE_STAMP(16 + (ch >> 1));
           }
           tmem_wait_st();
-          if (tid == 0) NSP_TRACE_STAMP(18);
           tc_fence_before_sync();
           mbar_arrive(&s.bar_p_ready);
-          if (tid == 0) NSP_TRACE_STAMP(7);
           // Phase 2: dS^T = P^T o (dP^T - delta) -> swizzled shared memory; P enters with its bf16 value, the one
           // the dV product uses. The dS buffer is free: dP^T of this step was issued behind dK / dQ^T of the
           // previous step, so bar_dp_full implies they have completed.
@@ -650,7 +621,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           oks = __all_sync(0xffffffffu, oks);
           if (!oks) { where = kWhereBwdDp; return false; }
           tc_fence_after_sync();
-          if (tid == 0) NSP_TRACE_STAMP(8);
           uint32_t dpv[2][16];
           tmem_ld16(tDP, dpv[0]);
 #pragma unroll
@@ -661,7 +631,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
 #pragma unroll
               for (int i = 0; i < 4; ++i) aux[(ch + 1) & 1][i] = lds128(delta_s + (ch + 1) * 16 + 4 * i);
             }
-            if (tid == 0) NSP_TRACE_STAMP(19 + ch);
             uint32_t dsp[8];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -694,7 +663,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           if (!oks) { where = kWhereBwdDp; break; }
           tc_fence_after_sync();
           const bool diag = (m == c.n);
-          if (tid == 0) NSP_TRACE_STAMP(6);
           if (mode & 1) {
             // delta_i = sum_j P_ij dP_ij over the keys of this tile (all keys of rows 0..127), fp32
             float* part = reinterpret_cast<float*>(s.ds[half]);  // [4 quadrants][64 columns]; free until dS is written
@@ -746,7 +714,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             oks = __all_sync(0xffffffffu, oks);
             if (!oks) { where = kWhereBwdDelta; break; }
           }
-          if (tid == 0) NSP_TRACE_STAMP(16);
 #pragma unroll 1
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t sv[16], dpv[16], pp[8], dsp[8];
@@ -786,7 +753,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             *reinterpret_cast<uint4*>(ds_row + ((2 * ch + 1) ^ (r & 7)) * 16) = make_uint4(dsp[4], dsp[5], dsp[6], dsp[7]);
           }
           tmem_wait_st();
-          if (tid == 0) NSP_TRACE_STAMP(17);
           tc_fence_before_sync();
           mbar_arrive(&s.bar_p_ready);
         }
@@ -794,7 +760,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         tc_fence_before_sync();
         mbar_arrive(&s.bar_ds_ready);
         mbar_arrive(&s.bar_ld_empty[st]);
-        if (tid == 0) NSP_TRACE_STAMP(9);
       }
       // ---- epilogue: wait for the last MMAs of the item, then write dK (scaled) and dV of this key tile
       if (oks) {
@@ -936,12 +901,6 @@ __global__ void bwd_postprocess_kernel(const float* __restrict__ acc, void* __re
 }
 
 }  // namespace
-
-#ifdef NSP_TRACE
-extern "C" int nsp_debug_trace_read(long long* host, int n) {
-  return cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
-}
-#endif
 
 cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
                                   const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta,

@@ -1,6 +1,6 @@
 // Forward: packed variable-length causal GQA attention on tcgen05 tensor cores.
 //
-// One persistent CTA per SM (384 threads) pops work items (segment, q head, q tile) from the longest-first
+// One persistent CTA per SM (640 threads) pops work items (segment, q head, q tile) from the longest-first
 // list TWO at a time. Neighbouring items of the list are the same (segment, q tile) for consecutive q heads, so
 // when they share a KV head (GQA) the CTA runs them as a pair "A/B" over the SAME K/V tiles: every K/V tile is
 // fetched once for 256 query rows, and the tensor pipe alternates between the two while their softmax
@@ -10,8 +10,9 @@
 //     O_x += P_x V_j        tcgen05.mma TS (A = P_x from TMEM, B = V MN-major from smem)          -> TMEM O_x
 // Issue order of the single MMA thread: PV_A(j), S_A(j+1), PV_B(j), S_B(j+1): S of the next key tile is already
 // running while the other half's softmax is still working. TMEM: S_A, S_B, O_A, O_B = 4 x 128 columns.
-// Roles: warps 0-3 softmax of A, warps 4-7 softmax of B, warp 8 TMA producer (Q pair, two-stage K and V rings),
-// warp 9 MMA issuer; register budgets are set per warpgroup with setmaxnreg.
+// Roles: warps 0-7 softmax of A, warps 8-15 softmax of B (two threads per query row, 64 score columns each), warp 16
+// TMA producer (Q pair, two-stage K and V rings), warp 17 MMA issuer; register budgets are set per warpgroup with
+// setmaxnreg.
 // O stays in TMEM for the whole item and is rescaled in place only when the running maximum grows by more than
 // 2^8 (the stale reference maximum is exact in the final normalisation because the same reference is used for
 // the row sum). Only the diagonal tile is masked; tiles above the diagonal are never visited.
@@ -27,17 +28,6 @@ constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;  // one [128 rows x 64 cols] b
 constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;
 constexpr uint32_t kFwdTmemCols = 512;  // S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512)
 constexpr int kFwdRegsSoftmax = 104, kFwdRegsAux = 64;  // 4*104 + 64 = 480 = 5 * 96, the launch-time allocation
-
-// Optional timeline (compiled in only with -DNSP_TRACE, for tuning): clock64 stamps of the first CTA's roles.
-#ifdef NSP_TRACE
-__device__ long long g_ftrace[64 * 24];
-#define NSP_FTRACE(slot)                                                                                          \
-  do {                                                                                                            \
-    if (blockIdx.x == 0 && gp == 1 && j >= 100 && j < 164) g_ftrace[(j - 100) * 24 + (slot)] = clock64();         \
-  } while (0)
-#else
-#define NSP_FTRACE(slot)
-#endif
 
 // One pop of the work list, decoded by thread 0 into shared memory (two slots: the next pop is fetched while the
 // current one runs).
@@ -245,9 +235,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             // offset (in 16-byte units) to the low word, which keeps the single issuing thread fast.
             const uint32_t hi = static_cast<uint32_t>(make_smem_desc_sw128(0, 16, 1024) >> 32);
             constexpr uint32_t lbo_km = (16u >> 4) << 16, lbo_mn = (kHalfTileBytes >> 4) << 16;
-            const uint32_t q_lo = (smem_u32(s.q[0][0]) >> 4) | lbo_km;  // item B: + kTileBytes / 16
-            const uint32_t k_lo = (smem_u32(s.k[0][0]) >> 4) | lbo_km;  // stage 1: + kTileBytes / 16
-            const uint32_t v_lo = (smem_u32(s.v[0][0]) >> 4) | lbo_mn;
+            const uint32_t q_lo = smem_desc_addr(s.q[0][0]) | lbo_km;  // item B: + kTileBytes / 16
+            const uint32_t k_lo = smem_desc_addr(s.k[0][0]) | lbo_km;  // stage 1: + kTileBytes / 16
+            const uint32_t v_lo = smem_desc_addr(s.v[0][0]) | lbo_mn;
             constexpr uint32_t kTileStep = kTileBytes >> 4;
             // S_x of key tile in stage kst -> TMEM columns [128*x, 128*x + 128)
             auto issue_s = [&](int x, uint32_t kst) {
@@ -287,7 +277,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               const bool more = j + 1 < n_kv;
               if (!mbar_wait(&s.bar_p_ready[0], pn[0] & 1)) { ok = false; where = kWhereFwdS; break; }
               ++pn[0];
-              NSP_FTRACE(0);
               if (!mbar_wait(&s.bar_v_full[vst], (vn >> 1) & 1)) { ok = false; where = kWhereFwdLoad; break; }
               tc_fence_after_sync();
               issue_pv(0, vst, j);
@@ -297,11 +286,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 tc_fence_after_sync();
                 issue_s(0, kst);
               }
-              NSP_FTRACE(1);
               if (joint) {
                 if (!mbar_wait(&s.bar_p_ready[1], pn[1] & 1)) { ok = false; where = kWhereFwdS; break; }
                 ++pn[1];
-                NSP_FTRACE(2);
                 tc_fence_after_sync();
                 issue_pv(1, vst, j);
               }
@@ -312,7 +299,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 umma_commit(&s.bar_k_empty[kst]);
                 ++kn;
               }
-              NSP_FTRACE(3);
             }
             if (!ok) {
               report_timeout(a.status, it0, where, 0);
@@ -362,13 +348,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             ++sn;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { where = kWhereFwdS; break; }
-            if (rl == 0 && ch == 0) NSP_FTRACE(4 + 8 * x);
             tc_fence_after_sync();
             uint32_t sr[2][32];
             tmem_ld32(tS + lane_off + ch * 64, sr[0]);
             tmem_ld32(tS + lane_off + ch * 64 + 32, sr[1]);
             tmem_wait_ld();
-            if (rl == 0 && ch == 0) NSP_FTRACE(5 + 8 * x);
             const bool last = (j == n_kv - 1);
             if (last) {  // diagonal tile: keys past the query are masked
 #pragma unroll
@@ -401,7 +385,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               m_ref = fmaxf(mx, partner_slot[0]) * a.scale_log2;
             } else if (pending) {
               ok = mbar_wait(pair_bar, xn & 1);
-              if (rl == 0 && ch == 0) NSP_FTRACE(7 + 8 * x);
               ++xn;
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) { where = kWhereFwdPair; break; }
@@ -413,7 +396,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               }
               pending = false;
             }
-            if (rl == 0 && ch == 0) NSP_FTRACE(6 + 8 * x);
             l *= alpha;
             float sum0 = 0.f, sum1 = 0.f;
             float mx_tile = -INFINITY;  // this tile's half-row maximum (raw scores), for the next tile
@@ -435,7 +417,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             // packed columns [64*ch, 64*ch + 32) = score columns [64*ch, 64*ch + 64): inside this thread's own
             // columns, so no other thread's unread scores are overwritten
             tmem_st32(tS + lane_off + ch * 64, pk);
-            if (rl == 0 && ch == 0) NSP_FTRACE(8 + 8 * x);
             // rescale this thread's 64 columns of O in place when some row of the warp moved its reference
             // maximum; the previous PV product of this half must have completed first (the next one is not
             // issued before p_ready).
@@ -457,7 +438,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&s.bar_p_ready[x]);
-            if (rl == 0 && ch == 0) NSP_FTRACE(9 + 8 * x);
             if (j > 0 && !last) {
               // post this tile's half-row maximum for the next tile. Slot by tile parity: the partner reads slot
               // j & 1 at the start of tile j + 1, and this thread writes it again only at the end of tile j + 2,
@@ -572,12 +552,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
 }
 
 }  // namespace
-
-#ifdef NSP_TRACE
-extern "C" int nsp_debug_ftrace_read(long long* host, int n) {
-  return cudaMemcpyFromSymbol(host, g_ftrace, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
-}
-#endif
 
 cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st) {
   if (args.n_items == 0) return cudaSuccess;

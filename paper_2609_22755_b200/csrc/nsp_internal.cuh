@@ -40,7 +40,14 @@ struct BwdMaps {
   CUtensorMap q[NSP_MAX_RUNS], d_o[NSP_MAX_RUNS], k[NSP_MAX_RUNS], v[NSP_MAX_RUNS];
 };
 
-// Device status word: {code, item, where, aux}; first writer wins (atomicCAS on code).
+// Device status record {code, item, where, aux}; the first writer wins (atomicCAS on the code in device memory) and
+// also copies its record into mapped pinned host memory, code last, so that the host sees a failure at its next API
+// call without synchronising.
+struct StatusWord {
+  int32_t* dev;   // device memory, four words
+  int32_t* host;  // device pointer to the same four words in mapped pinned host memory
+};
+
 enum DeviceWhere : int32_t {
   kWhereFwdLoad = 1,
   kWhereFwdS = 2,
@@ -67,12 +74,27 @@ enum DeviceWhere : int32_t {
   kWhereSelfTest = 90,
 };
 
-__device__ __forceinline__ void report_timeout(int32_t* status, int32_t item, int32_t where, int32_t aux) {
-  if (atomicCAS(status, 0, NSP_ERR_DEVICE_TIMEOUT) == 0) {
-    status[1] = item;
-    status[2] = where;
-    status[3] = aux;
+// Out of line on purpose: the callers sit in instruction-cache-sensitive loops and only get here when a wait ran out.
+static __device__ __noinline__ void report_status_raw(int32_t* dev, int32_t* host, int32_t code, int32_t item, int32_t where,
+                                               int32_t aux) {
+  if (atomicCAS(dev, 0, code) == 0) {
+    dev[1] = item;
+    dev[2] = where;
+    dev[3] = aux;
+    volatile int32_t* h = host;
+    h[1] = item;
+    h[2] = where;
+    h[3] = aux;
+    __threadfence_system();
+    h[0] = code;
+    __threadfence_system();
   }
+}
+__device__ __forceinline__ void report_status(StatusWord st, int32_t code, int32_t item, int32_t where, int32_t aux) {
+  report_status_raw(st.dev, st.host, code, item, where, aux);
+}
+__device__ __forceinline__ void report_timeout(StatusWord st, int32_t item, int32_t where, int32_t aux) {
+  report_status_raw(st.dev, st.host, NSP_ERR_DEVICE_TIMEOUT, item, where, aux);
 }
 
 struct FwdArgs {
@@ -80,7 +102,7 @@ struct FwdArgs {
   const nsp_tile_t* items;
   int32_t n_items;
   int32_t* counter;  // work-list cursor, zeroed before the launch
-  int32_t* status;
+  StatusWord status;
   __nv_bfloat16* o;
   float* lse;
   float scale_log2;  // softmax_scale * log2(e)
@@ -95,8 +117,8 @@ struct BwdArgs {
   const SegInfo* seg;
   const nsp_tile_t* items;
   int32_t n_items;
-  int32_t* counter;
-  int32_t* status;
+  int32_t* counter;  // work-list cursor, zeroed before the launch
+  StatusWord status;
   const float* lse;
   const float* delta;
   float* dq_acc;  // fp32 [q_elems], zeroed before the launch
@@ -105,8 +127,7 @@ struct BwdArgs {
   int32_t dkv_f32;
   float scale;
   float scale_log2;
-  int32_t debug_flags;  // experiments only: bit 0 = no hi/lo split, bit 1 = no exact delta
-  int32_t* front;       // [ceil(n_items / kFrontBlock)] arrival counters, zeroed before the launch (see next_item)
+  int32_t* front;    // [n_items / kFrontBlock + 1] arrival counters, zeroed before the launch (see next_item)
 };
 
 // Host-side launchers implemented next to their kernels.

@@ -1,9 +1,9 @@
-// Host-side routing of a batch onto the SP tree (paper Sec. 4.2: cost model and Algorithm 1, "Prefix-Completion
+// Host-side routing of a batch onto the SP tree (paper Sec. 4.1.2: cost model; Sec. 4.1.3: Algorithm 1, "Prefix-Completion
 // SP-Tree Routing"). No device code: this file is part of the library so that a caller gets the planner, its cost
 // table and the attention kernels behind one C ABI.
 //
 // Tree: the full binary tree over P = 2^(n_levels-1) GPUs; node (l, i) covers GPUs [i * 2^l, (i + 1) * 2^l) and
-// runs its samples at SP degree 2^l (paper Sec. 4.1, Def. 1). The cost model is additive: cost[j * n_levels + l] is
+// runs its samples at SP degree 2^l (paper Sec. 4.1.1, Def. 1). The cost model is additive: cost[j * n_levels + l] is
 // the load placed on every GPU of a level-l node by sample j, so the per-GPU load C_p of a plan is a plain sum.
 // Token loads (the paper's Tok_p) are kept in units of 1/P token, which keeps them integers.
 #include <algorithm>

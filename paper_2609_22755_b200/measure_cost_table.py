@@ -4,7 +4,7 @@
 batches through the library for every SP level of a model (level l: hq / 2^l query heads and max(1, hkv / 2^l) KV
 heads per GPU) and every length class b (segments of about 2^(b+5.5) tokens), and writes
 ``tcomp_ns[l][b]`` = nanoseconds per causal (query, key) pair and local query head, forward + backward: the profiled
-compute throughput the paper's cost model takes as an input (Sec. 4.2, SP-backend level). Length classes whose batch
+compute throughput the paper's cost model takes as an input (Sec. 4.1.2, SP-backend level). Length classes whose batch
 would exceed ``--max-pflop`` are not run; they take the value of the longest class that was (the time per pair no
 longer changes there). Needs a CUDA device.
 """

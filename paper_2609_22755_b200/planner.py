@@ -1,8 +1,8 @@
 """From a routed batch to the per-GPU shards the attention kernels take (host only, no arithmetic of the method).
 
 After the all-to-all of a degree-d node every GPU of the node holds the node's samples at full length with 1/d of
-the query heads (paper Sec. 2.2); a GPU's shard is the packed list of the samples of all nodes on its leaf-to-root
-chain (paper Sec. 4.1). Segments are ordered root first, inside a node by nonincreasing length.
+the query heads (paper Sec. 2.1); a GPU's shard is the packed list of the samples of all nodes on its leaf-to-root
+chain (paper Sec. 4.1.1). Segments are ordered root first, inside a node by nonincreasing length.
 """
 from __future__ import annotations
 

@@ -1,4 +1,4 @@
-"""Ulysses prologue / epilogue of one SP-tree node (paper Sec. 2.2; the communication phases of Sec. 4.2).
+"""Ulysses prologue / epilogue of one SP-tree node (paper Sec. 2.1; the communication phases of Sec. 4.1.2).
 
 Before attention, every GPU of a degree-d node holds a 1/d token slice of each of the node's samples with all heads;
 attention needs complete sequences with 1/d of the heads. The exchange is an all-to-all among the d GPUs. Here it is

@@ -3,11 +3,11 @@
 This module holds none of the method's arithmetic. It is the one module that both the CUDA tests/bench and
 the CPU oracle's tests consume, so that both sides see the same bytes.
 
-A workload is one GPU's share of a nested sequence-parallel plan (paper Sec. 4.1, Def. 1 and the per-GPU
+A workload is one GPU's share of a nested sequence-parallel plan (paper Sec. 4.1.1, Def. 1 and the per-GPU
 leaf-to-root chain): a packed list of segments, each at its own Ulysses degree d, which after the all-to-all
-appears on this GPU at full length with H/d query heads (paper Sec. 2.2). The five named configurations and
+appears on this GPU at full length with H/d query heads (paper Sec. 2.1). The five named configurations and
 their scaled-down twins follow the benchmark definition; lengths are long-tailed like the paper's corpora
-(Sec. 3, Fig. "long-tail": 94.0 % of samples below 8K tokens), drawn from a lognormal.
+(Sec. 3.1, Fig. "long-tail": 94.0 % of samples below 8K tokens), drawn from a lognormal.
 
 Recipe for lognormal lengths: x = median * exp(sigma * z), z ~ N(0,1) from numpy PCG64(seed);
 L = 16 * max(1, floor(x / 16 + 0.5)); clip to [lo, hi]; L = min(L, remaining budget); stop when the budget is
@@ -143,7 +143,7 @@ def config(idx: int, seed: int | None = None, twin: bool = False) -> Workload:
 
 
 def full_tree_shard(seed: int = 5, twin: bool = False) -> Workload:
-    """One GPU's chain in a full binary SP tree over eight GPUs (paper Sec. 4.1, Def. 1) for a 32q/4kv model: the
+    """One GPU's chain in a full binary SP tree over eight GPUs (paper Sec. 4.1.1, Def. 1) for a 32q/4kv model: the
     root's segment at degree 8 (4q/1kv), two at degree 4 (8q/1kv), four at degree 2 (16q/2kv) and a long-tailed
     degree-1 leaf batch (32q/4kv). Four runs with four different head counts in one shard. Not one of the five
     benchmark configurations (index 6); the twin divides the lengths by 32."""

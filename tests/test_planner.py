@@ -1,4 +1,4 @@
-"""Routing (paper Sec. 4.2: cost model and Algorithm 1): the oracle against exhaustive search, a textbook list
+"""Routing (paper Sec. 4.1.2: cost model; Sec. 4.1.3: Algorithm 1): the oracle against exhaustive search, a textbook list
 scheduler and invariants; the library's host functions against the oracle. No device is touched."""
 import heapq
 import itertools

@@ -1,4 +1,4 @@
-"""Save / recompute marking (paper Sec. 4.2, "Tree-Level Recomputation"): the oracle's walk against a hand-worked
+"""Save / recompute marking (paper Sec. 4.2.2 "Tree-Level Recomputation"): the oracle's walk against a hand-worked
 fixture, against a brute-force definition on small random shards, and the library's host function against the
 oracle. No device is touched."""
 import itertools

@@ -1,4 +1,4 @@
-"""Ulysses prologue / epilogue (paper Sec. 2.2, Sec. 4.2): the exchange schedule on CPU ranks (gloo, world sizes 2 and
+"""Ulysses prologue / epilogue (paper Sec. 2.1 "Sequence Parallelism", Sec. 4.1.2): the exchange schedule on CPU ranks (gloo, world sizes 2 and
 4, layout steps by a plain torch stand-in), and the library's CUDA layout kernels on one GPU against the same
 stand-in, including an emulation of all ranks of a node in one process."""
 import os
