@@ -319,7 +319,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       const bool is_a = warp == 17;
       QRing qr;
       while (next_item()) {
-        if (lane == 0) {
+        {
+          const bool leader = elect_one();
           constexpr uint32_t idesc_kk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
           constexpr uint32_t idesc_kn = make_idesc_bf16(128, 128, 0, 1);  // A K-major (or TMEM), B MN-major
           constexpr uint32_t idesc_nn = make_idesc_bf16(128, 128, 1, 1);  // A MN-major, B MN-major
@@ -345,10 +346,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
-                umma_ss_lh(tR0, k_km + off, hi, b_lo + off, hi, idesc_kk, kk > 0);
+                if (leader) umma_ss_lh(tR0, k_km + off, hi, b_lo + off, hi, idesc_kk, kk > 0);
               }
-              umma_commit(&s.bar_s_full);
-              umma_commit(&s.bar_q_empty[qr.st][0]);  // this thread is done with the Q stage
+              if (leader) umma_commit(&s.bar_s_full);
+              if (leader) umma_commit(&s.bar_q_empty[qr.st][0]);  // this thread is done with the Q stage
               qr.next();
               return true;
             };
@@ -364,10 +365,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               // dV += P^T dO; packed P^T columns of K-step kk (16 query columns) sit at R0 + (kk/2)*32 + (kk%2)*8
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk)
-                umma_ts_lh(tDV, tR0 + (kk >> 1) * 32 + (kk & 1) * 8, (do_lo | lbo_mn) + kk * 128, hi, idesc_kn,
+                if (leader) umma_ts_lh(tDV, tR0 + (kk >> 1) * 32 + (kk & 1) * 8, (do_lo | lbo_mn) + kk * 128, hi, idesc_kn,
                            acc | (kk > 0));
-              umma_commit(&s.bar_a_done);       // S^T and dV of the step
-              umma_commit(&s.bar_do_empty[0]);  // this thread is done with the dO buffer
+              if (leader) umma_commit(&s.bar_a_done);       // S^T and dV of the step
+              if (leader) umma_commit(&s.bar_do_empty[0]);  // this thread is done with the dO buffer
               if (vt + 1 < steps && !issue_s()) { okm = false; break; }
             }
           } else {
@@ -382,10 +383,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
-                umma_ss_lh(tR1, v_km + off, hi, (do_lo | lbo_km) + off, hi, idesc_kk, kk > 0);
+                if (leader) umma_ss_lh(tR1, v_km + off, hi, (do_lo | lbo_km) + off, hi, idesc_kk, kk > 0);
               }
-              umma_commit(&s.bar_dp_full);
-              umma_commit(&s.bar_do_empty[1]);  // this thread is done with the dO buffer
+              if (leader) umma_commit(&s.bar_dp_full);
+              if (leader) umma_commit(&s.bar_do_empty[1]);  // this thread is done with the dO buffer
               return true;
             };
             okm = okm && issue_dp(0);
@@ -401,22 +402,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               // dQ^T = K^T dS^T -> R1 (dP^T of this step has been consumed: ds_ready). It goes first: the dQ warps
               // drain R1 while dK runs, so that dP^T of the next step can follow dK without a gap.
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk) umma_ss_lh(tR1, k_mn + kk * 128, hi, ds_mn + kk * 128, hi, idesc_nn, kk > 0);
-              umma_commit(&s.bar_dq_full);
+              for (int kk = 0; kk < 8; ++kk) if (leader) umma_ss_lh(tR1, k_mn + kk * 128, hi, ds_mn + kk * 128, hi, idesc_nn, kk > 0);
+              if (leader) umma_commit(&s.bar_dq_full);
               // dK += dS^T Q
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
-                umma_ss_lh(tDK, ds_km + off, hi, q_mn + kk * 128, hi, idesc_kn, acc | (kk > 0));
+                if (leader) umma_ss_lh(tDK, ds_km + off, hi, q_mn + kk * 128, hi, idesc_kn, acc | (kk > 0));
               }
-              umma_commit(&s.bar_b_done);              // dP^T, dQ^T and dK of the step
-              umma_commit(&s.bar_q_empty[qr.st][1]);  // this thread is done with the Q stage
+              if (leader) umma_commit(&s.bar_b_done);              // dP^T, dQ^T and dK of the step
+              if (leader) umma_commit(&s.bar_q_empty[qr.st][1]);  // this thread is done with the Q stage
               qr.next();
               if (vt + 1 < steps && !issue_dp(vt + 1)) { okm = false; break; }
             }
           }
           if (!okm) {
-            report_timeout(a.status, item_it, where, is_a ? 0 : 1);
+            if (leader) report_timeout(a.status, item_it, where, is_a ? 0 : 1);
             *abort_flag = 1;
           }
         }

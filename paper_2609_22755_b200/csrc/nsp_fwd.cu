@@ -225,7 +225,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       uint32_t qn = 0, kn = 0, vn = 0, pn[2] = {0, 0};
       while (next_pop()) {
         for (int r = 0; r < n_rounds; ++r) {
-          if (lane == 0 && !*abort_flag) {
+          if (!*abort_flag) {
+            const bool leader = elect_one();
             const nsp_tile_t ia = r == 0 ? rd.a : rd.b;
             const int n_kv = ia.cost;
             const int joint = rd.joint;
@@ -245,18 +246,18 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
-                umma_ss_lh(tmem + 128 * x, a_lo + off, hi, b_lo + off, hi, idesc_qk, kk > 0);
+                if (leader) umma_ss_lh(tmem + 128 * x, a_lo + off, hi, b_lo + off, hi, idesc_qk, kk > 0);
               }
-              umma_commit(&s.bar_s_full[x]);
+              if (leader) umma_commit(&s.bar_s_full[x]);
             };
             // O_x += P_x V (P_x: bf16 pairs in columns [0,32) and [64,96) of S_x)
             auto issue_pv = [&](int x, uint32_t vst, int j) {
               const uint32_t b_lo = v_lo + vst * kTileStep;
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk)
-                umma_ts_lh(tmem + 256 + 128 * x, tmem + 128 * x + (kk >> 2) * 64 + (kk & 3) * 8, b_lo + kk * 128, hi, idesc_pv,
+                if (leader) umma_ts_lh(tmem + 256 + 128 * x, tmem + 128 * x + (kk >> 2) * 64 + (kk & 3) * 8, b_lo + kk * 128, hi, idesc_pv,
                            (j > 0 || kk > 0));
-              umma_commit(&s.bar_pv_done[x]);
+              if (leader) umma_commit(&s.bar_pv_done[x]);
             };
             bool ok = mbar_wait(&s.bar_q, qn & 1);
             ++qn;
@@ -270,7 +271,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 tc_fence_after_sync();
                 issue_s(0, kst);
                 if (joint) issue_s(1, kst);
-                umma_commit(&s.bar_k_empty[kst]);
+                if (leader) umma_commit(&s.bar_k_empty[kst]);
                 ++kn;
               }
               const uint32_t vst = vn & 1;
@@ -292,16 +293,16 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 tc_fence_after_sync();
                 issue_pv(1, vst, j);
               }
-              umma_commit(&s.bar_v_empty[vst]);
+              if (leader) umma_commit(&s.bar_v_empty[vst]);
               ++vn;
               if (more) {
                 if (joint) issue_s(1, kst);
-                umma_commit(&s.bar_k_empty[kst]);
+                if (leader) umma_commit(&s.bar_k_empty[kst]);
                 ++kn;
               }
             }
             if (!ok) {
-              report_timeout(a.status, it0, where, 0);
+              if (leader) report_timeout(a.status, it0, where, 0);
               *abort_flag = 1;
             }
           }
