@@ -33,9 +33,20 @@ from paper_2609_22755_b200 import workloads as W  # noqa: E402
 
 METRIC = "causal attention TFLOP/s fwd+bwd on 1 B200 and % of dense BF16 roofline"
 UNIT = "TFLOP/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one backward-main launch on the bench workload, from the
-# two-metric ncu capture summarised in profiles/bwd_kernel_nested_profile_case_64k.md.
-BWD_MAIN_DRAM_TRAFFIC_BYTES = int(42.52e9)  # measured on the bench workload itself (cfg4): 26.93 GB read + 15.59 GB written
+
+
+def captured_traffic(kernel: str, workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of `kernel` on `workload`, from the ncu capture
+    summaries kept as text under profiles/ (lines `traffic <kernel> <workload> <bytes> ...`); None when no capture
+    covers that pair."""
+    f = ROOT / "profiles" / "dram_traffic.txt"
+    if not f.exists():
+        return None
+    for line in f.read_text().splitlines():
+        parts = line.split()
+        if len(parts) >= 4 and parts[0] == "traffic" and parts[1] == kernel and parts[2] == workload:
+            return int(float(parts[3]))
+    return None
 
 
 def measured_peaks():
@@ -72,6 +83,90 @@ def run_oracle_sample(w: W.Workload):
     return flops / dt / 1e12, dt, oracle.num_threads(), desc
 
 
+def peaks_in_run(torch):
+    """The two roofline denominators measured again in this process, the way the stored measured peaks were taken:
+    a bf16 matmul of 8192^3 (best of 10 = burst) and a copy of 2^30 bf16 elements (read + write bytes, best of 10)."""
+    dev = torch.device("cuda")
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    a = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+    b = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+    for _ in range(3):
+        torch.matmul(a, b)
+    best = float("inf")
+    for _ in range(10):
+        e0, e1 = ev(), ev()
+        e0.record()
+        torch.matmul(a, b)
+        e1.record()
+        e1.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    tflops = 2 * 8192 ** 3 / (best * 1e-3) / 1e12
+    del a, b
+    x = torch.empty(1 << 30, device=dev, dtype=torch.bfloat16)
+    y = torch.empty_like(x)
+    for _ in range(2):
+        y.copy_(x)
+    best = float("inf")
+    for _ in range(10):
+        e0, e1 = ev(), ev()
+        e0.record()
+        y.copy_(x)
+        e1.record()
+        e1.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    gbs = 2 * x.numel() * 2 / (best * 1e-3) / 1e9
+    del x, y
+    torch.cuda.empty_cache()
+    return {"bf16_tflops": tflops, "hbm_gbs": gbs, "how": "torch.matmul bf16 8192^3 best of 10; copy of 2^30 bf16 best of 10"}
+
+
+def short_segment_roofline(torch, B, peaks, lengths=(128, 512), iters=5):
+    """The HBM-bound class: uniform batches of 131,072 tokens at 32q/4kv in segments of L tokens; achieved algorithmic
+    bytes per second of the forward launch and of the backward launches against the measured copy bandwidth."""
+    out = {}
+    dev = torch.device("cuda")
+    for L in lengths:
+        n = 131072 // L
+        w = W.custom([L] * n, 32, 4, seed=7, name=f"uniform_{n}x{L}_32q4kv")
+        qe, kve, le = w.q_elems(), w.kv_elems(), w.lse_elems()
+        bf = torch.bfloat16
+        q, do = (torch.randn(qe, device=dev, dtype=torch.float32).to(bf) for _ in range(2))
+        k, v = (torch.randn(kve, device=dev, dtype=torch.float32).to(bf) for _ in range(2))
+        o, dq = torch.empty_like(q), torch.empty_like(q)
+        lse = torch.empty(le, device=dev, dtype=torch.float32)
+        dk, dv = (torch.empty(kve, device=dev, dtype=torch.float32) for _ in range(2))
+        plan = B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, w.head_dim)
+        ws = torch.empty(max(plan.bwd_ws_bytes, 256), dtype=torch.uint8, device=dev)
+        fwd = lambda: B.nsp_attn_fwd(plan, q, k, v, o, lse, w.softmax_scale)
+        bwd = lambda: B.nsp_attn_bwd(plan, q, k, v, o, do, lse, dq, dk, dv, w.softmax_scale, ws)
+
+        def timed(fn):
+            for _ in range(3):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                fn()
+            e1.record()
+            e1.synchronize()
+            return e0.elapsed_time(e1) / iters
+
+        t_f, t_b = timed(fwd), timed(bwd)
+        bytes_f = 2 * (qe + 2 * kve) + 2 * qe + 4 * le                     # read Q,K,V; write O, LSE
+        bytes_b = 2 * (3 * qe + 2 * kve) + 4 * le + 8 * le + 2 * qe + 8 * kve   # read Q,K,V,O,dO,LSE; delta w+r; dQ bf16, dK/dV fp32
+        ff, fb = w.flops()
+        out[f"L{L}"] = {
+            "workload": w.name, "fwd_ms": t_f, "bwd_ms": t_b, "fwd_gbs": bytes_f / t_f / 1e6, "bwd_gbs": bytes_b / t_b / 1e6,
+            "fwd_frac": bytes_f / t_f / 1e6 / peaks["hbm_gbs"], "bwd_frac": bytes_b / t_b / 1e6 / peaks["hbm_gbs"],
+            "fwd_tflops": ff / t_f / 1e9, "bwd_tflops": fb / t_b / 1e9, "algorithmic_bytes": [bytes_f, bytes_b],
+        }
+        plan.destroy()
+        del q, do, k, v, o, dq, lse, dk, dv, ws
+        torch.cuda.empty_cache()
+    return {"bound": "hbm", "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_kind": f"hbm_gbs of {peaks['source']}",
+            "note": "bwd = memset + preprocess + main + postprocess", **out}
+
+
 class ClockSampler:
     """nvidia-smi clocks line sampled every 200 ms while the timed region runs."""
 
@@ -79,11 +174,13 @@ class ClockSampler:
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_id: str):
+        """gpu_id: what nvidia-smi -i takes; the device's UUID, because nvidia-smi numbers the GPUs of the machine,
+        not the ones CUDA_VISIBLE_DEVICES leaves to this process."""
         self.proc = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                ["nvidia-smi", "-i", str(gpu_id), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                  "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -122,7 +219,7 @@ def reference_arm(args, rank, world):
     """The oracle as it stands, timed on the host cores; each step is one bounded sample of the workload."""
     if rank != 0:
         return
-    w = W.profile_case() if args.config == 0 else W.config(args.config)
+    w = rank_workload(args.config, args.uniform, 0)
     vals = []
     for _ in range(args.warmup):
         run_oracle_sample(w)
@@ -186,6 +283,8 @@ def main():
                          "studies; not a bench value)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the in-run re-measurement of the peaks and the short-segment (HBM-bound) roofline lines")
     ap.add_argument("--profile-mode", action="store_true",
                     help="for runs under a profiler: allows fewer than 3 warm-up steps; the printed line is not a bench value")
     args = ap.parse_args()
@@ -198,6 +297,19 @@ def main():
         return
     if not args.profile_mode:
         args.warmup = max(args.warmup, 3)
+
+    # The CPU baseline is timed first, in a process of its own that never touches CUDA (it is the reference arm of
+    # this script run for one step): timed inside this process after the GPU work, next to 3.5 GB of pinned memory
+    # and the CUDA runtime's threads, the same oracle sample ran half as fast.
+    cpu = None
+    if world == 1 and rank == 0 and not args.no_cpu_baseline:
+        cmd = [sys.executable, str(Path(__file__).resolve()), "--impl", "reference", "--steps", "1", "--warmup", "0",
+               "--config", str(args.config)] + (["--uniform", str(args.uniform)] if args.uniform else [])
+        r = subprocess.run(cmd, capture_output=True, text=True)
+        try:
+            cpu = json.loads(r.stdout.strip().splitlines()[-1])["cpu_baseline"]
+        except Exception:
+            cpu = {"value": None, "unit": UNIT, "cores": None, "kind": "oracle", "sample": "failed: " + r.stderr[-200:]}
 
     import torch
     import torch.distributed as dist
@@ -233,7 +345,11 @@ def main():
     barrier()
     assert eng.status()[0] == 0, f"device status {eng.status()}"
 
-    sampler = ClockSampler(local_rank)
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
     launches0 = B.launch_count()
     k_fwd, k_bwd, k_pre, k_post = [], [], [], []
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -271,15 +387,25 @@ def main():
 
     if rank == 0:
         peaks = measured_peaks()
+        extras = {}
+        if world == 1 and not args.no_extras:
+            del eng, host  # give the device memory back before the extra measurements
+            torch.cuda.empty_cache()
+            extras["peaks_in_run"] = peaks_in_run(torch)
+            extras["roofline_short"] = short_segment_roofline(torch, B, peaks)
         bwd_ms = statistics.mean(k_bwd)
         achieved = f_bwd / (bwd_ms * 1e-3) / 1e12
         roofline = {
             "kernel": "bwd_kernel (backward main)", "bound": "tensor", "achieved": achieved, "peak": peaks["sustained"],
-            "unit": "TFLOP/s", "frac": achieved / peaks["sustained"], "traffic": BWD_MAIN_DRAM_TRAFFIC_BYTES,
+            "unit": "TFLOP/s", "frac": achieved / peaks["sustained"], "traffic": captured_traffic("bwd_kernel", w.name),
             "peak_kind": f"bf16_tflops_sustained of {peaks['source']} (kernel runs hundreds of ms inside a step)",
             "frac_of_burst_peak": achieved / peaks["burst"], "burst_peak": peaks["burst"],
             "launch_ms": bwd_ms, "flops_per_launch": f_bwd,
         }
+        if clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+            # the same launch scaled to the maximum SM clock (time x median MHz / max MHz): what the kernel would reach
+            # if the 1,000 W cap did not pull the clock down; a reading aid, not a measured number
+            roofline["achieved_at_max_clock"] = achieved * clocks["sm_max_mhz"] / clocks["sm_mhz"]
         fwd_ms = statistics.mean(k_fwd)
         roofline_fwd = {
             "kernel": "fwd_kernel", "bound": "tensor", "achieved": f_fwd / (fwd_ms * 1e-3) / 1e12, "peak": peaks["sustained"],
@@ -287,10 +413,6 @@ def main():
             "frac_of_burst_peak": f_fwd / (fwd_ms * 1e-3) / 1e12 / peaks["burst"], "launch_ms": fwd_ms,
             "flops_per_launch": f_fwd,
         }
-        cpu = None
-        if world == 1 and not args.no_cpu_baseline:
-            tf, dt, cores, desc = run_oracle_sample(w)
-            cpu = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
         line = {
             **({"profile_mode": True} if args.profile_mode else {}),
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -303,6 +425,9 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "roofline_fwd": roofline_fwd, "cpu_baseline": cpu,
             "fraction_of_burst_peak": value / world / peaks["burst"],
             "fraction_of_sustained_peak": value / world / peaks["sustained"],
+            "peaks": {"bf16_tflops_burst": peaks["burst"], "bf16_tflops_sustained": peaks["sustained"],
+                      "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
+            **extras,
             "kernels_ms": {"fwd": statistics.mean(k_fwd), "bwd_preprocess": statistics.mean(k_pre),
                            "bwd_main": bwd_ms, "bwd_postprocess": statistics.mean(k_post)},
             "tflops": {"fwd": f_fwd / (statistics.mean(k_fwd) * 1e-3) / 1e12,

@@ -135,15 +135,20 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
  * device memory to its own planner or caching pool at start-up has no way to obtain a transient q-sized fp32
  * buffer mid-iteration, because cudaMalloc would synchronise the device, may fail once the pool owns the memory,
  * and is banned inside some schedulers. For them the scratch (fp32 dQ accumulator + delta) is a fixed array of
- * NSP_STATIC_WS_BYTES inside the library image; every GPU that loads the library holds that much memory until exit.
+ * NSP_STATIC_WS_BYTES inside the library image. The driver reserves that memory on a GPU when it loads the module that
+ * holds the array: with the default lazy module loading that is the FIRST call of this function on the device (which
+ * looks up the array's device address with cudaGetSymbolAddress, that device being current), with eager loading
+ * (CUDA_MODULE_LOADING=EAGER) it is library load; the GPU then holds it until the process exits. So make that first
+ * call (any small batch will do) at start-up, before the caller's pool takes the remaining memory and before any
+ * stream capture begins: made later it may fail with NSP_ERR_CUDA for lack of memory, and it may synchronise.
+ * From the second call on a device, the call makes no cudaMalloc / cudaFree, calls no allocating routine and changes
+ * nothing about the device's free memory.
  * Arguments, outputs and results are those of nsp_attn_bwd (same kernels); inputs and outputs are still the caller's.
  * Limit: plans whose bwd_ws_bytes (see nsp_plan_sizes; roughly 4 * q_elems + 4 * lse_elems bytes) exceed
  * NSP_STATIC_WS_BYTES are rejected with NSP_ERR_WORKSPACE and nothing is enqueued.
- * This call makes no cudaMalloc / cudaFree and calls no allocating routine. The first call on each device looks up
- * the array's device address (cudaGetSymbolAddress, with that device current); make that first call before any
- * stream capture begins. The array is shared by all calls and keeps the previous call's contents: the
- * accumulator part is cleared on `stream` at the start of each call, and two calls whose device work overlaps
- * (other streams or host threads) race on it -- serialise them.
+ * The array is shared by all calls and keeps the previous call's contents: the accumulator part is cleared on
+ * `stream` at the start of each call, and two calls whose device work overlaps (other streams or host threads) race
+ * on it -- serialise them.
  * Errors: INVALID_ARG, WORKSPACE (batch too large), CUDA, DEVICE_TIMEOUT, as nsp_attn_bwd.
  */
 #define NSP_STATIC_WS_BYTES (32u * 1024u * 1024u)

@@ -448,9 +448,25 @@ int orc_attn_cols(const void* q, const void* k, const void* v, const void* d_o, 
  *   pass 1 (backward): one item per (segment s, kv head g, key tile n); cost = G * (Mt - floor(n*bn / bm)),
  *                      the number of (q head, q tile) visits of the key tile.
  * Order: cost descending, then segment, tile, head ascending -- a total order, so the list is unique.
+ *   pass 2 (backward, as executed): the items of pass 1 in the order the backward pass walks them: the groups
+ *                      (segment, kv head) by segment length descending, then segment ascending, then kv head
+ *                      ascending; inside a group the key tiles ascending. Also a total order.
  * Each item is four int32 {seg, head, tile, cost}. Returns the item count in *n_items; writes at most cap.
  */
 typedef struct { int32_t seg, head, tile, cost; } item_t;
+
+/* order of pass 2; the segment lengths are reached through this file-scope pointer while qsort runs */
+static const int32_t* g_cmp_cu = 0;
+static int item_cmp_exec(const void* a, const void* b) {
+  const item_t* x = (const item_t*)a;
+  const item_t* y = (const item_t*)b;
+  const int64_t lx = (int64_t)g_cmp_cu[x->seg + 1] - g_cmp_cu[x->seg], ly = (int64_t)g_cmp_cu[y->seg + 1] - g_cmp_cu[y->seg];
+  if (lx != ly) return lx > ly ? -1 : 1;
+  if (x->seg != y->seg) return x->seg < y->seg ? -1 : 1;
+  if (x->head != y->head) return x->head < y->head ? -1 : 1;
+  if (x->tile != y->tile) return x->tile < y->tile ? -1 : 1;
+  return 0;
+}
 
 static int item_cmp(const void* a, const void* b) {
   const item_t* x = (const item_t*)a;
@@ -464,7 +480,7 @@ static int item_cmp(const void* a, const void* b) {
 
 int orc_plan_tiles(const int32_t* cu, const int32_t* hq, const int32_t* hkv, int n_seg, int bm, int bn, int pass,
                    int32_t* out, int64_t cap, int64_t* n_items) {
-  if (n_seg < 0 || bm <= 0 || bn <= 0 || (pass != 0 && pass != 1) || !n_items) return ORC_BAD;
+  if (n_seg < 0 || bm <= 0 || bn <= 0 || pass < 0 || pass > 2 || !n_items) return ORC_BAD;
   int64_t total = 0;
   for (int s = 0; s < n_seg; ++s) {
     const int64_t L = (int64_t)cu[s + 1] - cu[s];
@@ -491,6 +507,11 @@ int orc_plan_tiles(const int32_t* cu, const int32_t* hq, const int32_t* hkv, int
         for (int64_t n = 0; n < Nt; ++n) it[w++] = (item_t){s, g, (int32_t)n, (int32_t)(G * (Mt - (n * bn) / bm))};
     }
   }
-  qsort(it, (size_t)total, sizeof(item_t), item_cmp);
+  if (pass == 2) {
+    g_cmp_cu = cu; /* not re-entrant: the Python front end calls this from one thread */
+    qsort(it, (size_t)total, sizeof(item_t), item_cmp_exec);
+  } else {
+    qsort(it, (size_t)total, sizeof(item_t), item_cmp);
+  }
   return ORC_OK;
 }

@@ -37,6 +37,8 @@ KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST = 0, 1, 2, 3
 
 import os
 
+# NSP_LIBRARY names another build of the same library (for instance the checked build, libnsp_checked.so, whose
+# kernels verify every index they compute); the default is the library built next to this file.
 LIB_PATH = Path(os.environ.get("NSP_LIBRARY", Path(__file__).resolve().parent / "libnsp.so"))
 _lib = None
 
@@ -123,7 +125,8 @@ def _i32(a):
 
 
 def _ptr(t):
-    """Device (or host) address of a torch tensor / numpy array / int / None."""
+    """Address of a torch tensor / numpy array (host metadata only) / int / None. Tensor arguments of the compute
+    calls are validated by _check_tensors before they get here."""
     if t is None:
         return None
     if isinstance(t, int):
@@ -131,6 +134,50 @@ def _ptr(t):
     if isinstance(t, np.ndarray):
         return t.ctypes.data_as(ctypes.c_void_p)
     return ctypes.c_void_p(t.data_ptr())
+
+
+def _check_tensors(what, plan, specs):
+    """Refuse buffers the kernels would read or write out of bounds: every tensor must be a contiguous CUDA tensor
+    of the stated dtype with at least the plan's element count. specs: (name, tensor, allowed dtypes, min elements).
+    Sizes of zero need no buffer at all."""
+    import torch
+
+    for name, t, dtypes, need in specs:
+        if need == 0:
+            continue
+        if not isinstance(t, torch.Tensor) or not t.is_cuda or not t.is_contiguous():
+            raise NspError(NSP_ERR_INVALID_ARG, f"{what}: {name} must be a contiguous CUDA tensor")
+        if t.dtype not in dtypes:
+            raise NspError(NSP_ERR_INVALID_ARG, f"{what}: {name} has dtype {t.dtype}")
+        if t.numel() < need:
+            raise NspError(NSP_ERR_INVALID_ARG, f"{what}: {name} holds {t.numel()} elements, the plan needs {need}")
+        if t.device.index != torch.cuda.current_device():
+            raise NspError(NSP_ERR_INVALID_ARG, f"{what}: {name} is on {t.device}, not on the current device")
+
+
+def _fwd_specs(plan, q, k, v, o, lse):
+    import torch
+
+    bf, f32 = (torch.bfloat16,), (torch.float32,)
+    return [("q", q, bf, plan.q_elems), ("k", k, bf, plan.kv_elems), ("v", v, bf, plan.kv_elems),
+            ("o", o, bf, plan.q_elems), ("lse", lse, f32, plan.lse_elems)]
+
+
+def _bwd_specs(plan, q, k, v, o, d_o, lse, dq, dk, dv, dq_dtype, dkv_dtype):
+    import torch
+
+    bf, f32 = (torch.bfloat16,), (torch.float32,)
+    return _fwd_specs(plan, q, k, v, o, lse) + [
+        ("d_o", d_o, bf, plan.q_elems), ("dq", dq, f32 if dq_dtype == NSP_F32 else bf, plan.q_elems),
+        ("dk", dk, f32 if dkv_dtype == NSP_F32 else bf, plan.kv_elems),
+        ("dv", dv, f32 if dkv_dtype == NSP_F32 else bf, plan.kv_elems)]
+
+
+def _check_ws(what, ws):
+    import torch
+
+    if ws is not None and (not isinstance(ws, torch.Tensor) or not ws.is_cuda or not ws.is_contiguous()):
+        raise NspError(NSP_ERR_WORKSPACE, f"{what}: the workspace must be a contiguous CUDA tensor")
 
 
 def _stream_ptr(stream):
@@ -200,6 +247,8 @@ def nsp_plan_get(plan: Plan, pass_: int) -> np.ndarray:
 
 
 def nsp_attn_fwd(plan: Plan, q, k, v, o, lse, softmax_scale, ws=None, stream=None):
+    _check_tensors("nsp_attn_fwd", plan, _fwd_specs(plan, q, k, v, o, lse))
+    _check_ws("nsp_attn_fwd", ws)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     rc = lib().nsp_attn_fwd(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), float(softmax_scale), _ptr(ws),
                             ws_bytes, _stream_ptr(stream))
@@ -215,6 +264,10 @@ def nsp_attn_bwd(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, softmax_scale, ws
         dq_dtype = NSP_F32 if dq.dtype == torch.float32 else NSP_BF16
     if dkv_dtype is None:
         dkv_dtype = NSP_F32 if dk.dtype == torch.float32 else NSP_BF16
+    if dq_dtype not in (NSP_BF16, NSP_F32) or dkv_dtype not in (NSP_BF16, NSP_F32):
+        raise NspError(NSP_ERR_INVALID_ARG, "nsp_attn_bwd: gradient dtype")
+    _check_tensors("nsp_attn_bwd", plan, _bwd_specs(plan, q, k, v, o, d_o, lse, dq, dk, dv, dq_dtype, dkv_dtype))
+    _check_ws("nsp_attn_bwd", ws)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     rc = lib().nsp_attn_bwd(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk),
                             _ptr(dv), dq_dtype, dkv_dtype, float(softmax_scale), _ptr(ws), ws_bytes,
@@ -334,6 +387,9 @@ def nsp_attn_bwd_recompute(plan: Plan, recompute, q, k, v, o, d_o, lse, dq, dk, 
         dq_dtype = NSP_F32 if dq.dtype == torch.float32 else NSP_BF16
     if dkv_dtype is None:
         dkv_dtype = NSP_F32 if dk.dtype == torch.float32 else NSP_BF16
+    _check_tensors("nsp_attn_bwd_recompute", plan,
+                   _bwd_specs(plan, q, k, v, o, d_o, lse, dq, dk, dv, dq_dtype, dkv_dtype))
+    _check_ws("nsp_attn_bwd_recompute", ws)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     rc = lib().nsp_attn_bwd_recompute(plan.handle, recompute.ctypes.data_as(ctypes.c_void_p), _ptr(q), _ptr(k), _ptr(v),
                                       _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv), dq_dtype, dkv_dtype,
@@ -382,6 +438,8 @@ def nsp_attn_bwd_static(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, softmax_sc
         dq_dtype = NSP_F32 if dq.dtype == torch.float32 else NSP_BF16
     if dkv_dtype is None:
         dkv_dtype = NSP_F32 if dk.dtype == torch.float32 else NSP_BF16
+    _check_tensors("nsp_attn_bwd_static", plan,
+                   _bwd_specs(plan, q, k, v, o, d_o, lse, dq, dk, dv, dq_dtype, dkv_dtype))
     rc = lib().nsp_attn_bwd_static(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq),
                                    _ptr(dk), _ptr(dv), dq_dtype, dkv_dtype, float(softmax_scale), _stream_ptr(stream))
     if rc != NSP_OK:

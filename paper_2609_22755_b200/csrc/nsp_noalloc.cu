@@ -8,8 +8,10 @@
 // forbidden outright inside some schedulers' critical sections). Such a caller still owns its inputs and
 // outputs, which its planner sized up front, but has nowhere to put a transient q-sized fp32 buffer.
 //
-// Cost: every GPU on which this library's module is loaded carries NSP_STATIC_WS_BYTES of global memory until
-// the process exits. All calls share the one array. It keeps whatever the previous call left in it; the part
+// Cost: every GPU on which the module of this file is loaded carries NSP_STATIC_WS_BYTES of global memory until
+// the process exits. With lazy module loading (the CUDA default) the module is loaded, and the memory reserved, by
+// the first cudaGetSymbolAddress on that device, i.e. inside the first call of the entry point: that call belongs at
+// start-up, before the caller's pool has taken the rest of the memory. All calls share the one array. It keeps whatever the previous call left in it; the part
 // that has to start at zero (the dQ accumulator) is cleared on the stream at the start of every call. Two calls
 // whose device work overlaps in time (different streams, or different host threads) race on the array.
 #include <mutex>

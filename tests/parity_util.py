@@ -48,14 +48,39 @@ class GpuRun:
         self.plan = B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, w.head_dim)
         assert self.plan.q_elems == w.q_elems() and self.plan.kv_elems == w.kv_elems()
         assert self.plan.lse_elems == w.lse_elems()
-        self.o = torch.full((w.q_elems(),), float("nan"), dtype=torch.bfloat16, device=self.dev)
-        self.lse = torch.full((w.lse_elems(),), float("nan"), dtype=torch.float32, device=self.dev)
+        # Every buffer the library writes sits between two 4 KiB guard bands filled with a byte pattern; results()
+        # checks that the bands are untouched (a stand-in for a memory checker: an out-of-range store of a kernel
+        # shows up as a failed test instead of silent corruption). Outputs start as NaN so that an element nobody
+        # wrote is seen as well.
+        self._guards = []
         tq = torch.float32 if dq_dtype == "f32" else torch.bfloat16
         tkv = torch.float32 if dkv_dtype == "f32" else torch.bfloat16
-        self.dq = torch.full((w.q_elems(),), float("nan"), dtype=tq, device=self.dev)
-        self.dk = torch.full((w.kv_elems(),), float("nan"), dtype=tkv, device=self.dev)
-        self.dv = torch.full((w.kv_elems(),), float("nan"), dtype=tkv, device=self.dev)
-        self.ws = torch.empty(max(self.plan.bwd_ws_bytes, 256), dtype=torch.uint8, device=self.dev)
+        self.o = self._guarded(w.q_elems(), torch.bfloat16)
+        self.lse = self._guarded(w.lse_elems(), torch.float32)
+        self.dq = self._guarded(w.q_elems(), tq)
+        self.dk = self._guarded(w.kv_elems(), tkv)
+        self.dv = self._guarded(w.kv_elems(), tkv)
+        self.ws = self._guarded(max(self.plan.bwd_ws_bytes, 256), torch.uint8, fill=None)
+
+    GUARD_BYTES = 4096
+    GUARD_PATTERN = 0xA5
+
+    def _guarded(self, n, dtype, fill=float("nan")):
+        torch = self.torch
+        size = torch.empty((), dtype=dtype).element_size()
+        raw = torch.full((2 * self.GUARD_BYTES + n * size,), self.GUARD_PATTERN, dtype=torch.uint8, device=self.dev)
+        body = raw[self.GUARD_BYTES:self.GUARD_BYTES + n * size].view(dtype)
+        if fill is not None and n:
+            body.fill_(fill)
+        self._guards.append(raw)
+        return body
+
+    def check_guards(self):
+        torch = self.torch
+        for i, raw in enumerate(self._guards):
+            lo, hi = raw[:self.GUARD_BYTES], raw[raw.numel() - self.GUARD_BYTES:]
+            assert bool((lo == self.GUARD_PATTERN).all()) and bool((hi == self.GUARD_PATTERN).all()), \
+                f"guard band of output buffer {i} was overwritten"
 
     def forward(self):
         self.B.nsp_attn_fwd(self.plan, self.q, self.k, self.v, self.o, self.lse, self.w.softmax_scale)
@@ -70,6 +95,7 @@ class GpuRun:
     def results(self):
         t = self.torch
         t.cuda.synchronize()
+        self.check_guards()
         f = lambda x: x.float().cpu().numpy().astype(np.float64)
         return {"o": f(self.o), "lse": f(self.lse), "dq": f(self.dq), "dk": f(self.dk), "dv": f(self.dv)}
 

@@ -32,9 +32,20 @@ def test_header_symbols_are_exported(B):
 
 def test_status_strings(B):
     assert B.status_string(B.NSP_OK) == "ok"
-    for code in range(1, 8):
+    for code in range(1, 9):
         assert B.status_string(code) not in ("ok", "unknown status")
     assert B.status_string(99) == "unknown status"
+
+
+def test_error_codes_match_the_header(B):
+    """The binding's constants are the header's enum, value by value (DEVICE_ASSERT keeps code 7, the planner's
+    INFEASIBLE has its own)."""
+    header = (ROOT / "include" / "nsp.h").read_text()
+    enum = dict((m.group(1), int(m.group(2))) for m in re.finditer(r"\b(NSP_(?:OK|ERR_[A-Z_]+))\s*=\s*(\d+)", header))
+    assert enum["NSP_ERR_DEVICE_TIMEOUT"] == 5 and enum["NSP_ERR_DEVICE_ASSERT"] == 7 and enum["NSP_ERR_INFEASIBLE"] == 8
+    for name, value in enum.items():
+        assert getattr(B, name) == value, name
+    assert len(set(enum.values())) == len(enum)
 
 
 def _plan_rc(B, cu, hq, hkv, head_dim=128, opts=None, null=None):

@@ -41,16 +41,12 @@ def test_tile_plan_bit_exact_full_size(env, idx):
     B, W, oracle = env["B"], env["W"], env["oracle"]
     w = W.config(idx)
     plan = B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, w.head_dim)
-    for p in (0, 1):
+    # pass 2 is the order the backward kernel walks (group-major); the oracle defines it independently
+    for p in (0, 1, 2):
         got = B.nsp_plan_get(plan, p)
         want = oracle.plan_tiles(w.cu_seqlens, w.hq, w.hkv, 128, 128, p)
         assert got.dtype == np.int32 and got.shape == want.shape
         assert np.array_equal(got, want)
-    # the order the backward kernel walks its items in is a permutation of the published backward list
-    exe = B.nsp_plan_get(plan, 2)
-    pub = B.nsp_plan_get(plan, 1)
-    key = lambda t: np.lexsort((t[:, 3], t[:, 2], t[:, 1], t[:, 0]))
-    assert exe.shape == pub.shape and np.array_equal(exe[key(exe)], pub[key(pub)])
     plan.destroy()
 
 
@@ -228,11 +224,17 @@ def test_bounded_wait_runs_out_and_is_reported(env):
     w = W.config(1)
     run = P.GpuRun(w)
     B.nsp_selftest_wait_timeout(run.plan, 1_000_000)
-    code, item, where, aux = B.nsp_device_status(run.plan)
-    assert (code, item, where, aux) == (B.NSP_ERR_DEVICE_TIMEOUT, -1, 90, 1_000_000 >> 10)
+    # the failing kernel writes its record to mapped host memory: once it has run, the very next call on the plan
+    # refuses, without anybody having polled nsp_device_status
+    env["torch"].cuda.synchronize()
     with pytest.raises(B.NspError) as e:
         run.forward()
     assert e.value.code == B.NSP_ERR_DEVICE_TIMEOUT
+    with pytest.raises(B.NspError) as e:
+        run.backward()
+    assert e.value.code == B.NSP_ERR_DEVICE_TIMEOUT
+    code, item, where, aux = B.nsp_device_status(run.plan)
+    assert (code, item, where, aux) == (B.NSP_ERR_DEVICE_TIMEOUT, -1, 90, 1_000_000 >> 10)
     _full_case(env, w)  # a fresh plan on the same context runs and matches the oracle
 
 
@@ -302,14 +304,23 @@ def test_packing_order_invariance_and_reproducibility(env):
     run.forward()
     run.backward()
     a = run.results()
-    # same inputs again: O, LSE, dK, dV bitwise equal (fixed accumulation order); dQ within tolerance
-    # (its tiles are added to the fp32 accumulator with floating-point reductions in arrival order)
+    # same inputs again: O, LSE, dK, dV bitwise equal (fixed accumulation order). dQ tiles are added to the fp32
+    # accumulator with floating-point reductions in arrival order: equal up to the rounding of an fp32 sum, which
+    # shows in the fp32 output (1e-5 of the largest element), not at the parity tolerance
+    run32 = P.GpuRun(w, tensors=run.host, dq_dtype="f32")
+    dq32 = []
+    for _ in range(2):
+        run32.forward()
+        run32.backward()
+        dq32.append(run32.results()["dq"])
+    assert np.max(np.abs(dq32[0] - dq32[1])) <= 1e-5 * np.max(np.abs(dq32[0]))
     run.forward()
     run.backward()
     b = run.results()
     for n in ("o", "lse", "dk", "dv"):
         assert np.array_equal(a[n], b[n]), n
-    assert P.errors(a["dq"], b["dq"])[0] <= 2e-2
+    # bf16 dQ of two runs: at most one rounding step apart where an fp32 sum sits on a rounding boundary
+    assert np.max(np.abs(a["dq"] - b["dq"]) / np.maximum(np.abs(a["dq"]), 1e-3)) <= 2.0 ** -7
     # permute the two runs (segments 2,3 first): every segment's results are unchanged
     qo, kvo, lo = w.q_offsets(), w.kv_offsets(), w.lse_offsets()
     perm = [2, 3, 0, 1]
@@ -325,7 +336,8 @@ def test_packing_order_invariance_and_reproducibility(env):
     for new, p in enumerate(perm):
         for n, off, poff in (("o", qo, pqo), ("lse", lo, plo), ("dk", kvo, pkvo), ("dv", kvo, pkvo)):
             assert np.array_equal(a[n][off[p]:off[p + 1]], c[n][poff[new]:poff[new + 1]]), (n, p)
-        assert P.errors(c["dq"][pqo[new]:pqo[new + 1]], a["dq"][qo[p]:qo[p + 1]])[0] <= 2e-2
+        x, y = c["dq"][pqo[new]:pqo[new + 1]], a["dq"][qo[p]:qo[p + 1]]
+        assert np.max(np.abs(x - y) / np.maximum(np.abs(y), 1e-3)) <= 2.0 ** -7
 
 
 def _sample_rows(w, rng, per_seg):
@@ -395,7 +407,7 @@ def test_full_size_configs_sampled(env, idx, per_seg, last_cols):
     assert float((got - want).abs().max()) <= 2e-3 * float(dv0.abs().sum(dim=0).max())
 
 
-@pytest.mark.parametrize("idx", [4, 5])
+@pytest.mark.parametrize("idx", [2, 3, 4, 5, 6])
 def test_full_size_sparse_dO_probe(env, idx):
     """dO non-zero on a sparse set of query rows: every element of dK and dV then depends on those rows only,
     so the oracle can produce ALL of dK/dV of the full-size configuration; dQ must vanish off the rows."""

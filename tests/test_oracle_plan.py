@@ -80,3 +80,36 @@ def test_hand_enumerated_fixture():
     cu, hq, hkv = [0, 300, 300, 428], [2, 2, 4], [1, 1, 4]
     assert [tuple(x) for x in oracle.plan_tiles(cu, hq, hkv, 128, 128, 0).tolist()] == want["fwd"]
     assert [tuple(x) for x in oracle.plan_tiles(cu, hq, hkv, 128, 128, 1).tolist()] == want["bwd"]
+    assert [tuple(x) for x in oracle.plan_tiles(cu, hq, hkv, 128, 128, 2).tolist()] == want["bwd_exec"]
+    cu2, hq2, hkv2 = [0, 128, 428, 728], [2, 2, 4], [2, 1, 2]
+    assert [tuple(x) for x in oracle.plan_tiles(cu2, hq2, hkv2, 128, 128, 1).tolist()] == want["bwd2"]
+    assert [tuple(x) for x in oracle.plan_tiles(cu2, hq2, hkv2, 128, 128, 2).tolist()] == want["bwd2_exec"]
+
+
+def _brute_exec(cu, hq, hkv, bm, bn):
+    """The executed backward order written out as nested loops (no sort): lengths from the longest down, for equal
+    lengths the segments in index order, kv heads, key tiles; the cost of an item counted from the causal mask."""
+    L = [int(cu[s + 1] - cu[s]) for s in range(len(hq))]
+    out = []
+    for length in sorted(set(L), reverse=True):
+        for s in range(len(hq)):
+            if L[s] != length or length == 0:
+                continue
+            G = hq[s] // hkv[s]
+            Mt, Nt = -(-length // bm), -(-length // bn)
+            for g in range(hkv[s]):
+                for n in range(Nt):
+                    visits = sum(1 for m in range(Mt) if n * bn <= min(length, (m + 1) * bm) - 1)
+                    out.append((s, g, n, G * visits))
+    return out
+
+
+@pytest.mark.parametrize("lengths,hq,hkv", CASES + [([300, 128, 300, 0, 300, 128], [4, 2, 2, 2, 8, 4], [2, 1, 2, 2, 2, 4])])
+@pytest.mark.parametrize("bm,bn", [(128, 128), (256, 128), (128, 64)])
+def test_executed_backward_order_matches_nested_loops(lengths, hq, hkv, bm, bn):
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    e = oracle.plan_tiles(cu, hq, hkv, bm, bn, 2)
+    assert [tuple(x) for x in e.tolist()] == _brute_exec(cu, hq, hkv, bm, bn)
+    # the same items as the published list
+    b = oracle.plan_tiles(cu, hq, hkv, bm, bn, 1)
+    assert sorted(map(tuple, e.tolist())) == sorted(map(tuple, b.tolist()))

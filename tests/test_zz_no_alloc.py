@@ -29,6 +29,7 @@ def test_static_workspace_backward_matches_regular_entry_point_twice():
     assert run.status()[0] == 0
     ref = run.results()
 
+    free_after = []
     for call in range(2):
         # poison the outputs so a call that silently did nothing cannot pass
         for t in (run.dq, run.dk, run.dv):
@@ -37,19 +38,25 @@ def test_static_workspace_backward_matches_regular_entry_point_twice():
                               w.softmax_scale)
         assert run.status()[0] == 0
         got = run.results()
+        free_after.append(torch.cuda.mem_get_info()[0])
         # same kernels, same order of the dK/dV accumulation -> bitwise equal; dQ tiles are added in arrival
         # order, so it is compared within the parity tolerance
         assert np.array_equal(got["dk"], ref["dk"]), f"call {call}"
         assert np.array_equal(got["dv"], ref["dv"]), f"call {call}"
         P.check(f"static call {call}: dq", got["dq"], ref["dq"])
+    # the first call on a device may make the driver load the module that holds the array (that is when the memory is
+    # reserved); a later call must not change the amount of free device memory
+    assert free_after[1] == free_after[0]
 
     # a batch whose scratch would not fit the fixed array is rejected, and nothing is written
     big = W.custom([16384], [8], [2], seed=1)
     plan = B.nsp_plan_tiles(big.cu_seqlens, big.hq, big.hkv, 128)
     assert plan.bwd_ws_bytes > B.NSP_STATIC_WS_BYTES
-    dummy = torch.zeros(16, dtype=torch.bfloat16, device="cuda")
+    mk = lambda n, dt: torch.zeros(n, dtype=dt, device="cuda")
+    bq, bkv = mk(plan.q_elems, torch.bfloat16), mk(plan.kv_elems, torch.bfloat16)
+    blse, bdkv = mk(plan.lse_elems, torch.float32), mk(plan.kv_elems, torch.float32)
     with pytest.raises(B.NspError) as e:
-        B.nsp_attn_bwd_static(plan, dummy, dummy, dummy, dummy, dummy, dummy, dummy, dummy, dummy, 0.1,
+        B.nsp_attn_bwd_static(plan, bq, bkv, bkv, bq, bq, blse, bq, bdkv, bdkv, 0.1,
                               dq_dtype=B.NSP_BF16, dkv_dtype=B.NSP_F32)
     assert e.value.code == B.NSP_ERR_WORKSPACE
     plan.destroy()
