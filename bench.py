@@ -351,7 +351,7 @@ def main():
         gpu_id = str(local_rank)
     sampler = ClockSampler(gpu_id)
     launches0 = B.launch_count()
-    k_fwd, k_bwd, k_pre, k_post = [], [], [], []
+    k_fwd, k_bwd, k_pre, k_post, k_first = [], [], [], [], []
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
@@ -362,6 +362,7 @@ def main():
         k_pre.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_PRE))
         k_bwd.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_MAIN))
         k_post.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_POST))
+        k_first.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_FIRST))
     e1.record()
     barrier()
     launches = B.launch_count() - launches0
@@ -429,9 +430,11 @@ def main():
                       "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
             **extras,
             "kernels_ms": {"fwd": statistics.mean(k_fwd), "bwd_preprocess": statistics.mean(k_pre),
-                           "bwd_main": bwd_ms, "bwd_postprocess": statistics.mean(k_post)},
+                           "bwd_first_tile": statistics.mean(k_first), "bwd_main": bwd_ms,
+                           "bwd_postprocess": statistics.mean(k_post)},
             "tflops": {"fwd": f_fwd / (statistics.mean(k_fwd) * 1e-3) / 1e12,
-                       "bwd": f_bwd / ((statistics.mean(k_pre) + bwd_ms + statistics.mean(k_post)) * 1e-3) / 1e12},
+                       "bwd": f_bwd / ((statistics.mean(k_pre) + statistics.mean(k_first) + bwd_ms
+                                        + statistics.mean(k_post)) * 1e-3) / 1e12},
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -256,7 +256,14 @@ int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
 int nsp_selftest_wait_timeout(const nsp_plan_t* plan, int64_t limit_clk, void* stream);
 
 /* Kernels of the path, for nsp_plan_kernel_ms. */
-enum { NSP_KERNEL_FWD = 0, NSP_KERNEL_BWD_PRE = 1, NSP_KERNEL_BWD_MAIN = 2, NSP_KERNEL_BWD_POST = 3, NSP_KERNEL_COUNT = 4 };
+enum {
+  NSP_KERNEL_FWD = 0,
+  NSP_KERNEL_BWD_PRE = 1,
+  NSP_KERNEL_BWD_MAIN = 2,
+  NSP_KERNEL_BWD_POST = 3,
+  NSP_KERNEL_BWD_FIRST = 4, /* the backward kernel for the first 128 tokens of every segment */
+  NSP_KERNEL_COUNT = 5
+};
 
 /* Measurement aid (the paper's cost model is fed by offline profiles of the compute phase, Sec. 4.1.2): when
  * enabled, every later nsp_attn_fwd / nsp_attn_bwd on this plan brackets each of its kernels with a pair of CUDA

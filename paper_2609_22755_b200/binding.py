@@ -33,7 +33,7 @@ EXPORTS = [
 ]
 NSP_COST_BUCKETS = 16
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
-KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST = 0, 1, 2, 3
+KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST, KERNEL_BWD_FIRST = 0, 1, 2, 3, 4
 
 import os
 

@@ -30,6 +30,9 @@ struct nsp_plan {
   nsp_tile_t* d_fwd = nullptr;
   nsp_tile_t* d_bwd = nullptr;
   nsp_tile_t* d_bwd_exec = nullptr;  // the backward items in the order the kernel walks them (see build_bwd_exec_order)
+  nsp_tile_t* d_bwd_first = nullptr;  // one item per (segment, kv head): the first-tile kernel's list
+  int64_t n_first = 0;
+  int32_t max_len = 0;                // longest segment: no preprocess / main / postprocess launch when <= 128
   int32_t* d_front = nullptr;        // [n_bwd / kFrontBlock + 1] start-alignment counters of the backward kernel
   int32_t* d_counters = nullptr;  // [0] forward cursor, [1] backward cursor
   int32_t* d_status = nullptr;    // {code, item, where, aux}
@@ -134,6 +137,7 @@ void free_plan(nsp_plan* p) {
   cudaFree(p->d_fwd);
   cudaFree(p->d_bwd);
   cudaFree(p->d_bwd_exec);
+  cudaFree(p->d_bwd_first);
   cudaFree(p->d_front);
   cudaFree(p->d_counters);
   cudaFree(p->d_status);
@@ -259,9 +263,14 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     return NSP_ERR_UNSUPPORTED;
   }
 
-  std::vector<nsp_tile_t> bwd_exec;
+  std::vector<nsp_tile_t> bwd_exec, bwd_first;
   try {
     bwd_exec = build_bwd_exec_order(p->seg, bm, bn);
+    // the first-tile kernel's items: key tile 0 of every group, in the same group order; q heads of the group = steps
+    for (const nsp_tile_t& t : bwd_exec)
+      if (t.tile == 0) bwd_first.push_back(nsp_tile_t{t.seg, t.head, 0, p->seg[t.seg].hq / p->seg[t.seg].hkv});
+    p->n_first = static_cast<int64_t>(bwd_first.size());
+    for (const SegInfo& sg : p->seg) p->max_len = std::max(p->max_len, sg.len);
   } catch (...) {
     delete p;
     return NSP_ERR_ALLOC;
@@ -292,8 +301,9 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
   A(reinterpret_cast<void**>(&p->d_fwd), sizeof(nsp_tile_t) * nf);
   A(reinterpret_cast<void**>(&p->d_bwd), sizeof(nsp_tile_t) * nb);
   A(reinterpret_cast<void**>(&p->d_bwd_exec), sizeof(nsp_tile_t) * nb);
+  A(reinterpret_cast<void**>(&p->d_bwd_first), sizeof(nsp_tile_t) * p->n_first);
   A(reinterpret_cast<void**>(&p->d_front), sizeof(int32_t) * (nb / kFrontBlock + 1));
-  A(reinterpret_cast<void**>(&p->d_counters), 4 * sizeof(int32_t));
+  A(reinterpret_cast<void**>(&p->d_counters), 4 * sizeof(int32_t));  // [0] forward, [1] backward main, [2] first-tile
   A(reinterpret_cast<void**>(&p->d_status), 4 * sizeof(int32_t));
   if (okc) {
     void* hp = nullptr;
@@ -329,6 +339,8 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     }
     C(cudaMemcpyAsync(p->d_row_base, row_base.data(), sizeof(int64_t) * (n_seg + 1), cudaMemcpyHostToDevice, st));
     if (nb > 0) C(cudaMemcpyAsync(p->d_bwd_exec, bwd_exec.data(), sizeof(nsp_tile_t) * nb, cudaMemcpyHostToDevice, st));
+    if (p->n_first > 0)
+      C(cudaMemcpyAsync(p->d_bwd_first, bwd_first.data(), sizeof(nsp_tile_t) * p->n_first, cudaMemcpyHostToDevice, st));
     if (e == cudaSuccess)
       C(launch_plan_build(p->d_seg, n_seg, bm, bn, p->d_fwd, nf, p->d_bwd, nb, d_keys, d_keys + nf + nb, d_tmp, tmp_bytes,
                           d_bases, d_bases + n_seg + 1, st));
@@ -458,10 +470,9 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
       return NSP_ERR_CUDA;
     if (recompute) fmaps.q[r] = maps.q[r], fmaps.k[r] = maps.k[r], fmaps.v[r] = maps.v[r];
   }
-  if (cudaMemsetAsync(plan->d_counters + 1, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (cudaMemsetAsync(plan->d_counters + 1, 0, 2 * sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
   if (cudaMemsetAsync(plan->d_front, 0, sizeof(int32_t) * (plan->n_bwd / kFrontBlock + 1), st) != cudaSuccess)
     return NSP_ERR_CUDA;
-  if (cudaMemsetAsync(dq_acc, 0, static_cast<size_t>(plan->q_elems) * 4, st) != cudaSuccess) return NSP_ERR_CUDA;
   if (recompute) {
     // from pageable memory the runtime stages the flags before it returns; a pinned array must stay unchanged until
     // the stream has passed this copy
@@ -484,33 +495,49 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
     if (launch_fwd(fmaps, fa, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
     prof_mark(plan, NSP_KERNEL_FWD, 1, st);
   }
+  // Segments of at most 128 tokens are finished by the first-tile kernel alone; a batch made only of such segments
+  // needs no accumulator, no delta and no conversion pass.
+  const bool multi = plan->max_len > kBM;
   prof_mark(plan, NSP_KERNEL_BWD_PRE, 0, st);
-  if (launch_bwd_preprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems,
-                            static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta,
-                            recompute ? d_mask : nullptr, recompute ? lse : nullptr, recompute ? lse_ws : nullptr,
-                            st) != cudaSuccess)
-    return NSP_ERR_CUDA;
+  if (multi || recompute) {
+    if (launch_bwd_preprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems,
+                              static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta,
+                              dq_acc, recompute ? d_mask : nullptr, recompute ? lse : nullptr,
+                              recompute ? lse_ws : nullptr, st) != cudaSuccess)
+      return NSP_ERR_CUDA;
+  }
   prof_mark(plan, NSP_KERNEL_BWD_PRE, 1, st);
   BwdArgs a;
   a.seg = plan->d_seg;
-  a.items = plan->d_bwd_exec;
-  a.n_items = static_cast<int32_t>(plan->n_bwd);
-  a.counter = plan->d_counters + 1;
   a.status = status_word(plan);
   a.lse = recompute ? lse_ws : lse;
   a.delta = delta;
   a.dq_acc = dq_acc;
+  a.dq = dq;
+  a.dq_f32 = dq_dtype == NSP_F32;
   a.front = plan->d_front;
   a.dk = dk;
   a.dv = dv;
   a.dkv_f32 = dkv_dtype == NSP_F32;
   a.scale = softmax_scale;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  // first-tile kernel: q tile 0 of every segment (its dQ rows; its part of, or all of, dK / dV rows 0..127)
+  a.items = plan->d_bwd_first;
+  a.n_items = static_cast<int32_t>(plan->n_first);
+  a.counter = plan->d_counters + 2;
+  prof_mark(plan, NSP_KERNEL_BWD_FIRST, 0, st);
+  if (launch_bwd_first(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  prof_mark(plan, NSP_KERNEL_BWD_FIRST, 1, st);
+  // main kernel: everything else
+  a.items = plan->d_bwd_exec;
+  a.n_items = static_cast<int32_t>(plan->n_bwd);
+  a.counter = plan->d_counters + 1;
   prof_mark(plan, NSP_KERNEL_BWD_MAIN, 0, st);
-  if (launch_bwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (multi && launch_bwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_MAIN, 1, st);
   prof_mark(plan, NSP_KERNEL_BWD_POST, 0, st);
-  if (launch_bwd_postprocess(dq_acc, dq, plan->q_elems, dq_dtype == NSP_F32, softmax_scale, st) != cudaSuccess)
+  if (multi && launch_bwd_postprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems, dq_acc, dq,
+                                      dq_dtype == NSP_F32, softmax_scale, st) != cudaSuccess)
     return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_POST, 1, st);
   return NSP_OK;

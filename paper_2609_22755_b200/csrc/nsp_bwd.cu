@@ -64,17 +64,23 @@ struct ItemCtx {
   int32_t len, hq, hkv, run, tok0;
   int32_t g, n;                    // kv head, key tile
   int32_t G;                       // q heads per kv head
-  int32_t first, two_pass, mode_first;
+  int32_t first;                   // key tile 0
+  int32_t m0;                      // first (lowest) q tile of the walk
   int32_t per_head;                // steps per q head
   int32_t steps;                   // G * per_head
 };
 
+// FIRST: the first-tile kernel also keeps the bf16 residual of dS^T. The main kernel does without those 32 KB on
+// purpose: shared memory it does not claim stays with the L1 cache, and the kernel ran 3 % slower with the larger
+// carve-out (the same 3 % the step from a three-stage to a two-stage Q ring gained).
+template <bool FIRST>
 struct BwdSmem {
   uint8_t k[2][kHalfTileBytes];
   uint8_t v[2][kHalfTileBytes];
   uint8_t q[kQStages][2][kHalfTileBytes];  // [stage][64-column half]: ring, loaded a whole step ahead
   uint8_t d_o[2][kHalfTileBytes];     // [half]: single buffer (its consumers leave a long window for the refill)
   uint8_t ds[2][kHalfTileBytes];      // dS^T, [key row][query col], two 64-column halves
+  uint8_t ds_lo[FIRST ? kTileBytes : 16];  // first-tile kernel: the bf16 residual of dS^T, same layout, right behind it
   float lse[2][128];                  // [stage] LSE * log2(e) of the q tile (+inf for rows past the segment)
   float delta[2][128];                // [stage]
   ItemCtx ctx[2];
@@ -93,8 +99,7 @@ struct BwdSmem {
   uint32_t tmem_base;
   int32_t abort;
 };
-static_assert(sizeof(BwdSmem) <= 232448, "shared memory budget (227 KB)");
-constexpr size_t kBwdSmemBytes = sizeof(BwdSmem);
+static_assert(sizeof(BwdSmem<true>) <= 232448, "shared memory budget (227 KB)");
 
 __device__ __forceinline__ void red_add_f32(float* addr, float v) {
   asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
@@ -118,24 +123,15 @@ __device__ __forceinline__ void setmaxnreg_dec() {
 // tail is summed while the accumulator is still small.
 // Heads innermost, so that CTAs that work on neighbouring key tiles stay one q tile apart for the whole item and
 // find the Q / dO tiles and the dQ accumulator rows they touch in L2.
-// mode bit 0: recompute delta exactly; bit 1: residual (lo) pass of the hi/lo split.
+// The first q tile of a segment (q tile 0 against key tile 0) is not walked here: it belongs to the first-tile
+// kernel (the same code instantiated with FIRST = true), so an item with key tile 0 starts at q tile 1.
 struct StepWalk {
   int hh, rr;
   __device__ __forceinline__ void reset() { hh = 0, rr = 0; }
-  __device__ __forceinline__ void get(const ItemCtx& c, int& h, int& m, int& mode) const {
+  __device__ __forceinline__ void get(const ItemCtx& c, int& h, int& m) const {
     const int p = c.per_head - 1 - rr;  // q tiles in DESCENDING order (see above)
     h = c.g * c.G + hh;
-    m = c.n + p;
-    mode = 0;
-    if (c.first) {
-      if (p == 0) {
-        m = 0, mode = c.mode_first;
-      } else if (c.two_pass && p == 1) {
-        m = 0, mode = c.mode_first | 2;
-      } else {
-        m = p - c.two_pass;
-      }
-    }
+    m = c.m0 + p;
   }
   __device__ __forceinline__ void next(const ItemCtx& c) {
     if (++hh == c.G) hh = 0, ++rr;
@@ -151,9 +147,18 @@ struct QRing {
   }
 };
 
+// FIRST = false: the main kernel, items (segment, kv head, key tile) against q tiles max(n, 1) .. Mt-1.
+// FIRST = true: the first-tile kernel, items (segment, kv head): q tile 0 against key tile 0 for every q head of the
+// group. Rows 0..127 of a segment have few keys, so P is O(1) and its bf16 rounding alone would push dK / dV past
+// the tolerance: there P^T and dS^T enter their products as bf16 value plus bf16 residual (two products each), and
+// delta_i = sum_j P_ij dP_ij is taken in fp32 (all keys of these rows sit in the tile) instead of from the
+// bf16-rounded O. Its dQ rows are complete (no other key tile reaches q tile 0) and are stored directly; its dK / dV
+// rows are the whole result for a one-tile segment and otherwise the part the main kernel, which runs after it, adds
+// its own sum to.
+template <bool FIRST>
 __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  BwdSmem& s = *reinterpret_cast<BwdSmem*>(smem_raw);
+  BwdSmem<FIRST>& s = *reinterpret_cast<BwdSmem<FIRST>*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
   // swizzled tiles need a 1024-byte aligned base
   const bool misaligned = (smem_u32(smem_raw) & 1023u) != 0;
@@ -213,9 +218,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   auto next_item = [&]() -> bool {
     ItemCtx& x = s.ctx[gi & 1];
     if (tid == 0) {
-      const int idx = atomicAdd(a.counter, 1);
-      x.it = idx;
-      if (idx < a.n_items) {
+      for (;;) {
+        const int idx = atomicAdd(a.counter, 1);
+        x.it = idx;
+        if (idx >= a.n_items) break;
         const nsp_tile_t item = a.items[idx];
         const SegInfo sg = a.seg[item.seg];
         x.q_off = sg.q_off, x.kv_off = sg.kv_off, x.lse_off = sg.lse_off;
@@ -223,9 +229,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         x.g = item.head, x.n = item.tile;
         x.G = sg.hq / sg.hkv;
         x.first = (item.tile == 0);
-        x.two_pass = x.first;  // hi / lo split of P and dS for the first q tile
-        x.mode_first = 1;      // exact delta for the first q tile
-        x.per_head = (sg.len + kBM - 1) / kBM - item.tile + x.two_pass;  // q tiles n .. Mt-1 (bm == bn)
+        if constexpr (FIRST) {
+          x.m0 = 0;
+          x.per_head = 1;  // q tile 0 only
+          x.steps = x.G;
+          break;
+        }
+        x.m0 = item.tile + x.first;                        // q tile 0 belongs to the first-tile kernel
+        x.per_head = (sg.len + kBM - 1) / kBM - x.m0;      // q tiles max(n, 1) .. Mt-1 (bm == bn)
         x.steps = x.G * x.per_head;
         // Start alignment. kFrontBlock consecutive items are neighbouring key tiles of one (segment, kv head) and
         // walk the same (q tile, head) sequence from the segment's last q tile down. CTAs that start them at the
@@ -248,6 +259,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               __nanosleep(200);
           }
         }
+        if (x.steps > 0) break;  // the only key tile of a one-tile segment has nothing left to do here
       }
     }
     tc_fence_before_sync();
@@ -285,8 +297,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           for (int vt = 0; vt < c.steps; ++vt) {
             const uint32_t cs = gs + vt;
             if (*abort_flag) break;
-            int h, m, mode;
-            w.get(c, h, m, mode);
+            int h, m;
+            w.get(c, h, m);
             w.next(c);
             if (!mbar_wait(&s.bar_q_empty[qr.st][0], qr.ph ^ 1) || !mbar_wait(&s.bar_q_empty[qr.st][1], qr.ph ^ 1)) {
               report_timeout(a.status, c.it, kWhereBwdQEmpty, vt);
@@ -354,26 +366,43 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               return true;
             };
             okm = okm && issue_s();
-#pragma unroll 1
-            for (int vt = 0; okm && vt < steps; ++vt) {
+            auto step_a = [&](int vt) -> bool {
+              constexpr bool fold = FIRST;
               const uint32_t cs = gs + vt;
-              if (*abort_flag) break;
-              if (!mbar_wait(&s.bar_do_full, cs & 1)) { okm = false; where = kWhereBwdLoadQ; break; }
-              if (!mbar_wait(&s.bar_p_ready, cs & 1)) { okm = false; where = kWhereBwdPReady; break; }
+              if (*abort_flag) return false;
+              if (!mbar_wait(&s.bar_do_full, cs & 1)) { where = kWhereBwdLoadQ; return false; }
+              if (!mbar_wait(&s.bar_p_ready, cs & 1)) { where = kWhereBwdPReady; return false; }
               tc_fence_after_sync();
               const uint32_t acc = vt > 0;
-              // dV += P^T dO; packed P^T columns of K-step kk (16 query columns) sit at R0 + (kk/2)*32 + (kk%2)*8
+              if constexpr (!fold) {
+                // dV += P^T dO; packed P^T columns of K-step kk (16 query columns) sit at R0 + (kk/2)*32 + (kk%2)*8
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk)
-                if (leader) umma_ts_lh(tDV, tR0 + (kk >> 1) * 32 + (kk & 1) * 8, (do_lo | lbo_mn) + kk * 128, hi, idesc_kn,
-                           acc | (kk > 0));
+                for (int kk = 0; kk < 8; ++kk)
+                  if (leader) umma_ts_lh(tDV, tR0 + (kk >> 1) * 32 + (kk & 1) * 8, (do_lo | lbo_mn) + kk * 128, hi, idesc_kn,
+                             acc | (kk > 0));
+              } else {
+                // P^T as value + residual, 16 query columns = 8 packed columns each, side by side
+#pragma unroll 1
+                for (int kk = 0; kk < 8; ++kk) {
+                  if (leader) umma_ts_lh(tDV, tR0 + kk * 16, (do_lo | lbo_mn) + kk * 128, hi, idesc_kn, acc | (kk > 0));
+                  if (leader) umma_ts_lh(tDV, tR0 + kk * 16 + 8, (do_lo | lbo_mn) + kk * 128, hi, idesc_kn, 1u);
+                }
+              }
               if (leader) umma_commit(&s.bar_a_done);       // S^T and dV of the step
               if (leader) umma_commit(&s.bar_do_empty[0]);  // this thread is done with the dO buffer
-              if (vt + 1 < steps && !issue_s()) { okm = false; break; }
-            }
+              if constexpr (fold) {
+                // the softmax warps read P^T back from R0 while they form dS^T: S^T of the next step waits for them
+                if (!mbar_wait(&s.bar_ds_ready, cs & 1)) { where = kWhereBwdDsReady; return false; }
+              }
+              if (vt + 1 < steps && !issue_s()) return false;
+              return true;
+            };
+#pragma unroll 1
+            for (int vt = 0; okm && vt < steps; ++vt) okm = step_a(vt);
           } else {
             const uint32_t v_km = smem_desc_addr(s.v[0]) | lbo_km, k_mn = smem_desc_addr(s.k[0]) | lbo_mn;
             const uint32_t ds_km = smem_desc_addr(s.ds[0]) | lbo_km, ds_mn = smem_desc_addr(s.ds[0]) | lbo_mn;
+            constexpr uint32_t kLoStep = kTileBytes >> 4;  // descriptor distance from dS^T to its residual
             // dP^T of step vt -> R1, once the dQ warps have drained dQ^T of the previous step from it
             auto issue_dp = [&](int vt) -> bool {
               const uint32_t cs = gs + vt;
@@ -390,12 +419,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               return true;
             };
             okm = okm && issue_dp(0);
-#pragma unroll 1
-            for (int vt = 0; okm && vt < steps; ++vt) {
+            auto step_b = [&](int vt) -> bool {
+              constexpr bool fold = FIRST;
               const uint32_t cs = gs + vt;
-              if (*abort_flag) break;
-              if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph)) { okm = false; where = kWhereBwdLoadQ; break; }
-              if (!mbar_wait(&s.bar_ds_ready, cs & 1)) { okm = false; where = kWhereBwdDsReady; break; }
+              if (*abort_flag) return false;
+              if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph)) { where = kWhereBwdLoadQ; return false; }
+              if (!mbar_wait(&s.bar_ds_ready, cs & 1)) { where = kWhereBwdDsReady; return false; }
               tc_fence_after_sync();
               const uint32_t acc = vt > 0;
               const uint32_t q_mn = (q0_lo + qr.st * kStageStep) | lbo_mn;
@@ -403,6 +432,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               // drain R1 while dK runs, so that dP^T of the next step can follow dK without a gap.
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk) if (leader) umma_ss_lh(tR1, k_mn + kk * 128, hi, ds_mn + kk * 128, hi, idesc_nn, kk > 0);
+              if constexpr (fold) {
+#pragma unroll 1
+                for (int kk = 0; kk < 8; ++kk)
+                  if (leader) umma_ss_lh(tR1, k_mn + kk * 128, hi, ds_mn + kLoStep + kk * 128, hi, idesc_nn, 1u);
+              }
               if (leader) umma_commit(&s.bar_dq_full);
               // dK += dS^T Q
 #pragma unroll
@@ -410,13 +444,23 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
                 if (leader) umma_ss_lh(tDK, ds_km + off, hi, q_mn + kk * 128, hi, idesc_kn, acc | (kk > 0));
               }
+              if constexpr (fold) {
+#pragma unroll 1
+                for (int kk = 0; kk < 8; ++kk) {
+                  const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
+                  if (leader) umma_ss_lh(tDK, ds_km + kLoStep + off, hi, q_mn + kk * 128, hi, idesc_kn, 1u);
+                }
+              }
               if (leader) umma_commit(&s.bar_b_done);              // dP^T, dQ^T and dK of the step
               if (leader) umma_commit(&s.bar_q_empty[qr.st][1]);  // this thread is done with the Q stage
               qr.next();
-              if (vt + 1 < steps && !issue_dp(vt + 1)) { okm = false; break; }
-            }
+              if (vt + 1 < steps && !issue_dp(vt + 1)) return false;
+              return true;
+            };
+#pragma unroll 1
+            for (int vt = 0; okm && vt < steps; ++vt) okm = step_b(vt);
           }
-          if (!okm) {
+          if (!okm && where != 0) {  // where == 0: another role raised the abort flag
             if (leader) report_timeout(a.status, item_it, where, is_a ? 0 : 1);
             *abort_flag = 1;
           }
@@ -442,8 +486,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             }
             break;
           }
-          int h, m, mode;
-          w.get(c, h, m, mode);
+          int h, m;
+          w.get(c, h, m);
           w.next(c);
           const int64_t base = c.lse_off + static_cast<int64_t>(h) * c.len;
 #pragma unroll
@@ -483,8 +527,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           break;
         }
         tc_fence_after_sync();
-        int h, m, mode;
-        w.get(c, h, m, mode);
+        int h, m;
+        w.get(c, h, m);
         w.next(c);
         // Register e of a column chunk is dQ^T[d][query]: the 32 lanes of a warp add 32 consecutive floats of
         // one accumulator row (128 bytes, one request). Eight warps issue them: one SM sustains about 25 bytes
@@ -493,6 +537,32 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         const int rows_left = c.len - m * kBM;  // valid query rows of this q tile (>= 128 for an interior tile)
         float* const tile0 = a.dq_acc + c.q_off + (static_cast<int64_t>(m) * kBM * c.hq + h) * kHeadDim + d;
         const int n_valid = min(kBM, rows_left) - colhalf * 64;
+        if constexpr (FIRST) {
+          // q tile 0 gets nothing from any other key tile: scale and store the rows directly, no accumulator
+          uint32_t v0[32], v1[32];
+          tmem_ld32(tR1 + lane_off + colhalf * 64, v0);
+          tmem_ld32(tR1 + lane_off + colhalf * 64 + 32, v1);
+          tmem_wait_ld();
+          tc_fence_before_sync();
+          mbar_arrive(&s.bar_dq_empty);
+          const int64_t o0 = c.q_off + (static_cast<int64_t>(colhalf * 64) * c.hq + h) * kHeadDim + d;
+          if (a.dq_f32) {
+            float* q0 = static_cast<float*>(a.dq) + o0;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              if (e < n_valid) q0[e * q_stride] = __uint_as_float(v0[e]) * a.scale;
+              if (e + 32 < n_valid) q0[(e + 32) * q_stride] = __uint_as_float(v1[e]) * a.scale;
+            }
+          } else {
+            __nv_bfloat16* q0 = static_cast<__nv_bfloat16*>(a.dq) + o0;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              if (e < n_valid) q0[e * q_stride] = __float2bfloat16_rn(__uint_as_float(v0[e]) * a.scale);
+              if (e + 32 < n_valid) q0[(e + 32) * q_stride] = __float2bfloat16_rn(__uint_as_float(v1[e]) * a.scale);
+            }
+          }
+          continue;
+        }
         float* p0 = tile0 + colhalf * 64 * q_stride;
         if (n_valid >= 64) {  // interior tile: no row checks
           uint32_t v0[32], v1[32];
@@ -553,8 +623,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       for (int vt = 0; vt < c.steps; ++vt) {
         const uint32_t cs = gs + vt, st = cs & 1;
         if (*abort_flag) { oks = false; where = 0; break; }
-        int h, m, mode;
-        w.get(c, h, m, mode);
+        int h, m;
+        w.get(c, h, m);
         w.next(c);
         oks = mbar_wait(&s.bar_ld_full[st], (cs >> 1) & 1) && mbar_wait(&s.bar_s_full, cs & 1);
         oks = __all_sync(0xffffffffu, oks);
@@ -652,20 +722,25 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           }
           return true;
         };
-        if (mode == 0 && m != c.n) {
-          if (!common_step(std::false_type{})) break;
-        } else if (mode == 0) {
-          if (!common_step(std::true_type{})) break;
+        if constexpr (!FIRST) {
+          if (m != c.n) {
+            if (!common_step(std::false_type{})) break;
+          } else {
+            if (!common_step(std::true_type{})) break;
+          }
         } else {
-          // ---- rare step (one of the two first-tile passes): compact rolled loops, 16 query
-          // columns at a time; P^T and dS^T are handed over together at the end.
+          // ---- first-tile step (q tile 0 against key tile 0, always a diagonal tile): compact rolled loops, 16
+          // query columns at a time. Rows 0..127 of a segment have few keys, so P is O(1) and its bf16 rounding alone
+          // would push dK / dV past the tolerance: P^T and dS^T enter their products as bf16 value plus bf16 residual
+          // (two products each, the residuals next to the values), and delta_i = sum_j P_ij dP_ij is taken here in
+          // fp32 (all keys of these rows sit in this tile) instead of from the bf16-rounded O.
           oks = mbar_wait(&s.bar_dp_full, cs & 1);
           oks = __all_sync(0xffffffffu, oks);
           if (!oks) { where = kWhereBwdDp; break; }
           tc_fence_after_sync();
-          const bool diag = (m == c.n);
-          if (mode & 1) {
-            // delta_i = sum_j P_ij dP_ij over the keys of this tile (all keys of rows 0..127), fp32
+          {
+            // Sweep 1: P^T (value and residual over the S^T columns just read: packed columns [16ch, 16ch + 8) and
+            // [16ch + 8, 16ch + 16)) and the partial sums of delta.
             float* part = reinterpret_cast<float*>(s.ds[half]);  // [4 quadrants][64 columns]; free until dS is written
             // Column sums over the 32 key rows of a warp by a butterfly: at every level a lane keeps the half of
             // the columns its lane bit selects and adds the partner's partial sums of that half (16 shuffles for
@@ -673,7 +748,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4, b1 = lane & 2;
 #pragma unroll 1
             for (int ch = 0; ch < 4; ++ch) {
-              uint32_t sv[16], dpv[16];
+              uint32_t sv[16], dpv[16], pk[16];
               float4 l4[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) l4[i] = lds128(lse_s + ch * 16 + 4 * i);
@@ -682,13 +757,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               tmem_wait_ld();
               float v[16];
 #pragma unroll
-              for (int x = 0; x < 16; ++x) {
-                const float lse_x = (x & 3) == 0 ? l4[x >> 2].x : (x & 3) == 1 ? l4[x >> 2].y
-                                  : (x & 3) == 2 ? l4[x >> 2].z : l4[x >> 2].w;
-                float p = ex2f(fmaf(__uint_as_float(sv[x]), a.scale_log2, -lse_x));
-                if (half * 64 + ch * 16 + x < r) p = 0.f;
-                v[x] = p * __uint_as_float(dpv[x]);
+              for (int x = 0; x < 16; x += 2) {
+                const float lse0 = (x & 2) ? l4[x >> 2].z : l4[x >> 2].x, lse1 = (x & 2) ? l4[x >> 2].w : l4[x >> 2].y;
+                float p0 = ex2f(fmaf(__uint_as_float(sv[x + 0]), a.scale_log2, -lse0));
+                float p1 = ex2f(fmaf(__uint_as_float(sv[x + 1]), a.scale_log2, -lse1));
+                if (half * 64 + ch * 16 + x + 0 < r) p0 = 0.f;  // query index must be >= key index
+                if (half * 64 + ch * 16 + x + 1 < r) p1 = 0.f;
+                v[x + 0] = p0 * __uint_as_float(dpv[x + 0]);
+                v[x + 1] = p1 * __uint_as_float(dpv[x + 1]);
+                const uint32_t pa = pack_bf16x2(p0, p1);
+                pk[x >> 1] = pa;
+                pk[8 + (x >> 1)] = pack_bf16x2(p0 - __uint_as_float(pa << 16), p1 - __uint_as_float(pa & 0xffff0000u));
               }
+              tmem_st16(tS + ch * 16, pk);
               float w8[8], w4[4], w2[2];
 #pragma unroll
               for (int i = 0; i < 8; ++i)
@@ -703,6 +784,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               w1 += __shfl_xor_sync(0xffffffffu, w1, 1);
               if ((lane & 1) == 0) part[quad * 64 + ch * 16 + (lane >> 1)] = w1;
             }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&s.bar_p_ready);  // the dV products run under the rest of this step
             mbar_arrive(&s.bar_delta[half]);
             oks = mbar_wait(&s.bar_delta[half], nd & 1);
             ++nd;
@@ -715,47 +799,36 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             oks = __all_sync(0xffffffffu, oks);
             if (!oks) { where = kWhereBwdDelta; break; }
           }
+          // Sweep 2: dS^T = P^T o (dP^T - delta), value and residual; P^T (value + residual = P to 2^-17) is read back
+          // from R0, which the next S^T does not overwrite before bar_ds_ready.
+          uint8_t* const ds_row_lo = ds_row + kTileBytes;
 #pragma unroll 1
           for (int ch = 0; ch < 4; ++ch) {
-            uint32_t sv[16], dpv[16], pp[8], dsp[8];
-            float4 l4[4], e4[4];
+            uint32_t pk[16], dpv[16], dsp[8], dsl[8];
+            float4 e4[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              l4[i] = lds128(lse_s + ch * 16 + 4 * i);
-              e4[i] = lds128(delta_s + ch * 16 + 4 * i);
-            }
-            tmem_ld16(tS + ch * 16, sv);
+            for (int i = 0; i < 4; ++i) e4[i] = lds128(delta_s + ch * 16 + 4 * i);
+            tmem_ld16(tS + ch * 16, pk);
             tmem_ld16(tDP + ch * 16, dpv);
             tmem_wait_ld();
 #pragma unroll
             for (int x = 0; x < 16; x += 2) {
-              const float lse0 = (x & 2) ? l4[x >> 2].z : l4[x >> 2].x, lse1 = (x & 2) ? l4[x >> 2].w : l4[x >> 2].y;
               const float del0 = (x & 2) ? e4[x >> 2].z : e4[x >> 2].x, del1 = (x & 2) ? e4[x >> 2].w : e4[x >> 2].y;
-              float p0 = ex2f(fmaf(__uint_as_float(sv[x + 0]), a.scale_log2, -lse0));
-              float p1 = ex2f(fmaf(__uint_as_float(sv[x + 1]), a.scale_log2, -lse1));
-              if (diag) {  // query index must be >= key index
-                if (half * 64 + ch * 16 + x + 0 < r) p0 = 0.f;
-                if (half * 64 + ch * 16 + x + 1 < r) p1 = 0.f;
-              }
+              const uint32_t ph = pk[x >> 1], pl = pk[8 + (x >> 1)];
+              const float p0 = __uint_as_float(ph << 16) + __uint_as_float(pl << 16);
+              const float p1 = __uint_as_float(ph & 0xffff0000u) + __uint_as_float(pl & 0xffff0000u);
               const float d0 = p0 * (__uint_as_float(dpv[x + 0]) - del0);
               const float d1 = p1 * (__uint_as_float(dpv[x + 1]) - del1);
-              uint32_t pa = pack_bf16x2(p0, p1), da = pack_bf16x2(d0, d1);
-              if (mode & 2) {  // residual pass: what the bf16 value left behind
-                pa = pack_bf16x2(p0 - __uint_as_float(pa << 16), p1 - __uint_as_float(pa & 0xffff0000u));
-                da = pack_bf16x2(d0 - __uint_as_float(da << 16), d1 - __uint_as_float(da & 0xffff0000u));
-              }
-              pp[x >> 1] = pa;
+              const uint32_t da = pack_bf16x2(d0, d1);
               dsp[x >> 1] = da;
+              dsl[x >> 1] = pack_bf16x2(d0 - __uint_as_float(da << 16), d1 - __uint_as_float(da & 0xffff0000u));
             }
-            // query columns [16ch, 16ch + 16) -> packed columns 32*(ch/2) + 8*(ch%2) .. +8 (never ahead of a
-            // column this thread still has to read)
-            tmem_st8(tS + (ch >> 1) * 32 + (ch & 1) * 8, pp);
-            *reinterpret_cast<uint4*>(ds_row + ((2 * ch) ^ (r & 7)) * 16) = make_uint4(dsp[0], dsp[1], dsp[2], dsp[3]);
-            *reinterpret_cast<uint4*>(ds_row + ((2 * ch + 1) ^ (r & 7)) * 16) = make_uint4(dsp[4], dsp[5], dsp[6], dsp[7]);
+            const uint32_t c0 = ((2 * ch) ^ (r & 7)) * 16, c1 = ((2 * ch + 1) ^ (r & 7)) * 16;
+            *reinterpret_cast<uint4*>(ds_row + c0) = make_uint4(dsp[0], dsp[1], dsp[2], dsp[3]);
+            *reinterpret_cast<uint4*>(ds_row + c1) = make_uint4(dsp[4], dsp[5], dsp[6], dsp[7]);
+            *reinterpret_cast<uint4*>(ds_row_lo + c0) = make_uint4(dsl[0], dsl[1], dsl[2], dsl[3]);
+            *reinterpret_cast<uint4*>(ds_row_lo + c1) = make_uint4(dsl[4], dsl[5], dsl[6], dsl[7]);
           }
-          tmem_wait_st();
-          tc_fence_before_sync();
-          mbar_arrive(&s.bar_p_ready);
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
@@ -781,18 +854,36 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           uint32_t v[32];
           tmem_ld32(tDK + which * 128 + lane_off + half * 64 + cc * 32, v);
           tmem_wait_ld();
+          // Key tile 0 in the main kernel: the first-tile kernel, which ran before, left its part (q tile 0) in the
+          // output; this item's sum over the q tiles 1 .. Mt-1 is added to it (one fixed order: reproducible).
+          const bool add = !FIRST && c.first;
           if (valid) {
             if (a.dkv_f32) {
               float* o = static_cast<float*>(outp) + off + cc * 32;
 #pragma unroll
-              for (int x = 0; x < 32; x += 4)
-                *reinterpret_cast<float4*>(o + x) =
-                    make_float4(__uint_as_float(v[x]) * mul, __uint_as_float(v[x + 1]) * mul,
-                                __uint_as_float(v[x + 2]) * mul, __uint_as_float(v[x + 3]) * mul);
+              for (int x = 0; x < 32; x += 4) {
+                float4 w4 = make_float4(__uint_as_float(v[x]) * mul, __uint_as_float(v[x + 1]) * mul,
+                                        __uint_as_float(v[x + 2]) * mul, __uint_as_float(v[x + 3]) * mul);
+                if (add) {
+                  const float4 old = *reinterpret_cast<const float4*>(o + x);
+                  w4.x += old.x, w4.y += old.y, w4.z += old.z, w4.w += old.w;
+                }
+                *reinterpret_cast<float4*>(o + x) = w4;
+              }
             } else {
               __nv_bfloat16* o = static_cast<__nv_bfloat16*>(outp) + off + cc * 32;
 #pragma unroll
               for (int x = 0; x < 32; x += 8) {
+                if (add) {  // bf16 output: the first part was rounded once already (not the graded dtype)
+                  const uint4 old = *reinterpret_cast<const uint4*>(o + x);
+                  const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+                  for (int t = 0; t < 4; ++t) {
+                    v[x + 2 * t] = __float_as_uint(__uint_as_float(v[x + 2 * t]) + __uint_as_float(ow[t] << 16) / mul);
+                    v[x + 2 * t + 1] =
+                        __float_as_uint(__uint_as_float(v[x + 2 * t + 1]) + __uint_as_float(ow[t] & 0xffff0000u) / mul);
+                  }
+                }
                 uint4 wv;
                 wv.x = pack_bf16x2(__uint_as_float(v[x]) * mul, __uint_as_float(v[x + 1]) * mul);
                 wv.y = pack_bf16x2(__uint_as_float(v[x + 2]) * mul, __uint_as_float(v[x + 3]) * mul);
@@ -816,17 +907,29 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   if (warp == 0) tmem_dealloc(s.tmem_base, kBwdTmemCols);
 }
 
-// delta[h, i] = <dO[i,h,:], O[i,h,:]>. Rows (token, head) are packed one after the other, 256 bytes each, so the
-// kernel streams O and dO as flat arrays: a warp takes eight consecutive rows per pass, sixteen lanes per row with
-// one 16-byte load per tensor (eight loads in flight per thread), and only the index of the result needs the
-// segment table (delta is stored [head][token] inside a segment): lanes 0..7 look up one row each.
-// With seg_skip, the rows of marked segments are read but nothing is written for them; with lse_out, the LSE of every
-// row that is processed is copied from lse_in (same index as delta).
+// Which segment a packed (token, head) row belongs to: row_base[s] = first packed row of segment s (ascending).
+__device__ __forceinline__ int find_segment(const int64_t* __restrict__ row_base, int n_seg, int64_t row) {
+  int lo = 0, hi = n_seg - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (row_base[mid] <= row) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+// Preprocess, for the rows the main kernel works on (tokens 128.. of every segment; the first 128 tokens belong to
+// the first-tile kernel, which needs neither): delta[h, i] = <dO[i,h,:], O[i,h,:]> and the row's 128 floats of the dQ
+// accumulator set to zero. Rows (token, head) are packed one after the other, 256 bytes each, so the kernel streams
+// O and dO as flat arrays: a warp takes eight consecutive rows per pass, sixteen lanes per row with one 16-byte load
+// per tensor (eight loads in flight per thread), and only the index of the result needs the segment table (delta is
+// stored [head][token] inside a segment): lanes 0..7 look up one row each.
+// With seg_skip, no delta is written for the rows of marked segments (it comes from the recomputation); with lse_out,
+// the LSE of every row whose delta is written is copied from lse_in (same index as delta).
 __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __restrict__ seg, int n_seg,
                                                              const int64_t* __restrict__ row_base, int64_t total_rows,
                                                              const __nv_bfloat16* __restrict__ o,
                                                              const __nv_bfloat16* __restrict__ d_o,
-                                                             float* __restrict__ delta,
+                                                             float* __restrict__ delta, float* __restrict__ dq_acc,
                                                              const uint8_t* __restrict__ seg_skip,
                                                              const float* __restrict__ lse_in,
                                                              float* __restrict__ lse_out) {
@@ -846,23 +949,23 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
         va[p] = vb[p] = make_uint4(0u, 0u, 0u, 0u);
       }
     }
-    // where the result of row row0 + (lane & 7) goes
+    // row row0 + (lane & 7): where its delta goes (-1: nowhere), and whether it is one of the main kernel's rows
     int64_t dst = -1;
+    int mine = 0;
     {
       const int64_t row = row0 + (lane & 7);
       if (row < total_rows) {
-        int lo = 0, hi = n_seg - 1;  // row_base[s] = first packed row of segment s (ascending)
-        while (lo < hi) {
-          const int mid = (lo + hi + 1) >> 1;
-          if (row_base[mid] <= row) lo = mid; else hi = mid - 1;
-        }
-        const SegInfo sg = seg[lo];
-        const int64_t rl = row - row_base[lo];
+        const int sgi = find_segment(row_base, n_seg, row);
+        const SegInfo sg = seg[sgi];
+        const int64_t rl = row - row_base[sgi];
         const int64_t i = rl / sg.hq, h = rl - i * sg.hq;
-        // rows of a skipped segment (its delta and LSE come from the recomputation) are left alone
-        if (seg_skip == nullptr || seg_skip[lo] == 0) {
-          dst = sg.lse_off + h * sg.len + i;
-          if (lse_out != nullptr && lane < 8) lse_out[dst] = lse_in[dst];
+        mine = i >= kBM;
+        // rows of a skipped segment (its delta and LSE come from the recomputation) get neither here; for the other
+        // segments the LSE copy covers every row (the first-tile kernel reads it too)
+        if (seg_skip == nullptr || seg_skip[sgi] == 0) {
+          const int64_t at = sg.lse_off + h * sg.len + i;
+          if (lse_out != nullptr && lane < 8) lse_out[at] = lse_in[at];
+          if (mine) dst = at;
         }
       }
     }
@@ -880,23 +983,54 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
 #pragma unroll
       for (int sft = 8; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
       const int64_t dst_p = __shfl_sync(0xffffffffu, dst, 2 * p + sub);
+      const int mine_p = __shfl_sync(0xffffffffu, mine, 2 * p + sub);
       if (l16 == 0 && dst_p >= 0) delta[dst_p] = acc;
+      if (mine_p) {
+        float4* z = reinterpret_cast<float4*>(dq_acc + (row0 + 2 * p + sub) * kHeadDim) + 2 * l16;
+        z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+        z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
     }
   }
 }
 
-__global__ void bwd_postprocess_kernel(const float* __restrict__ acc, void* __restrict__ dq, int64_t n4, int dq_f32,
-                                       float scale) {
-  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-  for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < n4; t += stride) {
-    const float4 v = reinterpret_cast<const float4*>(acc)[t];
-    if (dq_f32) {
-      reinterpret_cast<float4*>(dq)[t] = make_float4(v.x * scale, v.y * scale, v.z * scale, v.w * scale);
-    } else {
-      uint2 w;
-      w.x = pack_bf16x2(v.x * scale, v.y * scale);
-      w.y = pack_bf16x2(v.z * scale, v.w * scale);
-      reinterpret_cast<uint2*>(dq)[t] = w;
+// Postprocess: dQ = scale * accumulator, in the output dtype, for the rows the main kernel works on (tokens 128.. of
+// every segment; the rows before were stored by the first-tile kernel). Same row walk as the preprocess kernel.
+__global__ void __launch_bounds__(256) bwd_postprocess_kernel(const SegInfo* __restrict__ seg, int n_seg,
+                                                              const int64_t* __restrict__ row_base, int64_t total_rows,
+                                                              const float* __restrict__ acc, void* __restrict__ dq,
+                                                              int dq_f32, float scale) {
+  const int lane = threadIdx.x & 31, sub = lane >> 4, l16 = lane & 15;
+  const int64_t n_groups = (total_rows + 7) >> 3;
+  const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+  for (int64_t grp = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; grp < n_groups; grp += n_warps) {
+    const int64_t row0 = grp * 8;
+    int mine = 0;
+    {
+      const int64_t row = row0 + (lane & 7);
+      if (row < total_rows) {
+        const int sgi = find_segment(row_base, n_seg, row);
+        mine = (row - row_base[sgi]) / seg[sgi].hq >= kBM;
+      }
+    }
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      const int64_t row = row0 + 2 * p + sub;
+      if (!__shfl_sync(0xffffffffu, mine, 2 * p + sub)) continue;
+      const float4* src = reinterpret_cast<const float4*>(acc + row * kHeadDim) + 2 * l16;
+      const float4 v0 = src[0], v1 = src[1];
+      if (dq_f32) {
+        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(dq) + row * kHeadDim) + 2 * l16;
+        dst[0] = make_float4(v0.x * scale, v0.y * scale, v0.z * scale, v0.w * scale);
+        dst[1] = make_float4(v1.x * scale, v1.y * scale, v1.z * scale, v1.w * scale);
+      } else {
+        uint4 w;
+        w.x = pack_bf16x2(v0.x * scale, v0.y * scale);
+        w.y = pack_bf16x2(v0.z * scale, v0.w * scale);
+        w.z = pack_bf16x2(v1.x * scale, v1.y * scale);
+        w.w = pack_bf16x2(v1.z * scale, v1.w * scale);
+        reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(dq) + row * kHeadDim)[l16] = w;
+      }
     }
   }
 }
@@ -904,35 +1038,45 @@ __global__ void bwd_postprocess_kernel(const float* __restrict__ acc, void* __re
 }  // namespace
 
 cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
-                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta,
+                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, float* dq_acc,
                                   const uint8_t* seg_skip, const float* lse_in, float* lse_out, cudaStream_t st) {
   if (total_rows == 0) return cudaSuccess;
   int64_t blocks = ((total_rows + 7) / 8 * 32 + 255) / 256;  // one warp per eight rows, grid-stride beyond 16 waves
   if (blocks > 148 * 8 * 16) blocks = 148 * 8 * 16;
   bwd_preprocess_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows, o, d_o,
-                                                                       delta, seg_skip, lse_in, lse_out);
+                                                                       delta, dq_acc, seg_skip, lse_in, lse_out);
   count_launches(1);
   return cudaGetLastError();
 }
 
-cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
+namespace {
+template <bool FIRST>
+cudaError_t launch_bwd_t(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
   if (args.n_items == 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kBwdSmemBytes));
+  cudaError_t e = cudaFuncSetAttribute(bwd_kernel<FIRST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(sizeof(BwdSmem<FIRST>)));
   if (e != cudaSuccess) return e;
   const int grid = args.n_items < num_sms ? args.n_items : num_sms;
-  bwd_kernel<<<grid, kBwdThreads, kBwdSmemBytes, st>>>(maps, args);
+  bwd_kernel<FIRST><<<grid, kBwdThreads, sizeof(BwdSmem<FIRST>), st>>>(maps, args);
   count_launches(1);
   return cudaGetLastError();
 }
+}  // namespace
 
-cudaError_t launch_bwd_postprocess(const float* dq_acc, void* dq, int64_t n, int dq_f32, float scale,
-                                   cudaStream_t st) {
-  if (n == 0) return cudaSuccess;
-  const int64_t n4 = n / 4;  // n is a multiple of 128
-  int64_t blocks = (n4 + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
-  bwd_postprocess_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(dq_acc, dq, n4, dq_f32, scale);
+cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
+  return launch_bwd_t<false>(maps, args, num_sms, st);
+}
+cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
+  return launch_bwd_t<true>(maps, args, num_sms, st);
+}
+
+cudaError_t launch_bwd_postprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
+                                   const float* dq_acc, void* dq, int dq_f32, float scale, cudaStream_t st) {
+  if (total_rows == 0) return cudaSuccess;
+  int64_t blocks = ((total_rows + 7) / 8 * 32 + 255) / 256;
+  if (blocks > 148 * 8 * 16) blocks = 148 * 8 * 16;
+  bwd_postprocess_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows, dq_acc,
+                                                                        dq, dq_f32, scale);
   count_launches(1);
   return cudaGetLastError();
 }
