@@ -239,6 +239,20 @@ int nsp_route_sp_tree(const int32_t* lengths, const int64_t* cost, int32_t n_sam
  * Errors: INVALID_ARG, UNSUPPORTED (row size not a multiple of 16 bytes), CUDA.
  */
 #define NSP_A2A_MAX_PEERS 64
+/*
+ * nsp_a2a_gather_heads_to: the send side of the prologue fused with the exchange. The same head gather as
+ * nsp_a2a_gather_heads, but block p is not staged: its rows are stored straight into dst_base[p], the packed
+ * attention buffer [t_full, heads_per_block, head_dim] the receiving GPU's nsp_attn_fwd reads (a peer's memory mapped
+ * into this process, or a local buffer). src holds the token slices of n_samples samples one after the other;
+ * sample_off (DEVICE, int64 [n_samples + 1], sample_off[0] = 0, last = tokens) gives their rows in src, and
+ * dst_row (DEVICE, int64 [n_blocks * n_samples]) the row in dst_base[p] where this GPU's slice of sample j starts
+ * (entry p * n_samples + j). dst_base and first_head are host arrays [n_blocks]. The stores are plain 16-byte stores
+ * issued by the library's own kernel; the receiver may read its buffer once it has synchronised with this stream
+ * (an event or a barrier between the GPUs is the caller's). Errors as nsp_a2a_gather_heads.
+ */
+int nsp_a2a_gather_heads_to(const void* src, void* const* dst_base, const int64_t* dst_row, const int64_t* sample_off,
+                            int32_t n_samples, int64_t tokens, int32_t heads, int32_t heads_per_block, int32_t n_blocks,
+                            int32_t head_dim, int32_t dtype, const int32_t* first_head, void* stream);
 int nsp_a2a_gather_heads(const void* src, void* dst, int64_t tokens, int32_t heads, int32_t heads_per_block,
                          int32_t n_blocks, int32_t head_dim, int32_t dtype, const int32_t* first_head, void* stream);
 int nsp_a2a_scatter_heads(const void* src, void* dst, int64_t tokens, int32_t heads, int32_t heads_per_block,

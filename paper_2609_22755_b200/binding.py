@@ -29,7 +29,7 @@ EXPORTS = [
     "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string", "nsp_plan_set_profiling", "nsp_plan_kernel_ms",
     "nsp_attn_bwd_static", "nsp_recompute_mark", "nsp_plan_recompute_ws_bytes", "nsp_attn_bwd_recompute",
     "nsp_cost_table", "nsp_route_sp_tree", "nsp_a2a_gather_heads", "nsp_a2a_scatter_heads",
-    "nsp_selftest_wait_timeout",
+    "nsp_selftest_wait_timeout", "nsp_a2a_gather_heads_to",
 ]
 NSP_COST_BUCKETS = 16
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
@@ -94,6 +94,9 @@ def lib() -> ctypes.CDLL:
             f.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                           ctypes.c_int32, vp, vp]
             f.restype = ctypes.c_int
+        L.nsp_a2a_gather_heads_to.argtypes = [vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
+                                              ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
+        L.nsp_a2a_gather_heads_to.restype = ctypes.c_int
         L.nsp_selftest_wait_timeout.argtypes = [vp, ctypes.c_int64, vp]
         L.nsp_selftest_wait_timeout.restype = ctypes.c_int
         L.nsp_device_status.argtypes = [vp, i32p]
@@ -359,6 +362,32 @@ def _a2a(fn_name, src, dst, tokens, heads, heads_per_block, head_dim, first_head
 def nsp_a2a_gather_heads(src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream=None):
     """[tokens, heads, D] -> [len(first_head)][tokens, heads_per_block, D] (device tensors, flat or shaped)."""
     _a2a("nsp_a2a_gather_heads", src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream)
+
+
+def nsp_a2a_gather_heads_to(src, dst_tensors, dst_row, sample_off, tokens, heads, heads_per_block, head_dim, first_head,
+                            stream=None):
+    """The head gather fused with the exchange: block p is stored into dst_tensors[p] (the receiving GPU's packed
+    attention buffer, or a local stand-in) at the rows dst_row[p, j] (device int64 [n_blocks, n_samples]) for the
+    samples whose rows in src are given by sample_off (device int64 [n_samples + 1])."""
+    import numpy as np
+    import torch
+
+    dtype = NSP_F32 if src.dtype == torch.float32 else NSP_BF16
+    n = len(dst_tensors)
+    fh = np.ascontiguousarray(first_head, dtype=np.int32)
+    if len(fh) != n or any(t.dtype != src.dtype or not t.is_cuda for t in dst_tensors):
+        raise ValueError("one destination tensor of the source's dtype per block")
+    if dst_row.dtype != torch.int64 or sample_off.dtype != torch.int64 or not dst_row.is_cuda or not sample_off.is_cuda:
+        raise ValueError("dst_row and sample_off are int64 device tensors")
+    n_samples = sample_off.numel() - 1
+    if dst_row.numel() != n * n_samples:
+        raise ValueError("dst_row holds one row per (block, sample)")
+    bases = (ctypes.c_void_p * n)(*[t.data_ptr() for t in dst_tensors])
+    rc = lib().nsp_a2a_gather_heads_to(_ptr(src), bases, _ptr(dst_row.contiguous()), _ptr(sample_off.contiguous()),
+                                       n_samples, int(tokens), int(heads), int(heads_per_block), n, int(head_dim), dtype,
+                                       fh.ctypes.data_as(ctypes.c_void_p), _stream_ptr(stream))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_a2a_gather_heads_to")
 
 
 def nsp_a2a_scatter_heads(src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream=None):

@@ -47,6 +47,42 @@ __global__ void __launch_bounds__(256) gather_heads_kernel(const uint4* __restri
   }
 }
 
+// The fused send side of the prologue: the same head gather, but every block is stored where its receiver reads it.
+// Block p goes to base[p] (the packed attention buffer [t_full, Hd, D] of peer p: that GPU's own memory mapped into
+// this process, or a local buffer), the tokens of sample j starting at row dst_row[p * n_samples + j] there (where
+// this GPU's token slice of the sample sits inside the complete sequence). Plain 16-byte stores from this kernel: no
+// library kernel is handed a peer pointer, and nothing here is a TMA or multicast access.
+struct PeerBases {
+  uint4* base[NSP_A2A_MAX_PEERS];
+};
+__global__ void __launch_bounds__(256) gather_heads_to_kernel(const uint4* __restrict__ src, int64_t T, int H, int Hd,
+                                                              int n, int vec_per_row, int n_samples,
+                                                              const int64_t* __restrict__ sample_off,
+                                                              const int64_t* __restrict__ dst_row,
+                                                              const __grid_constant__ HeadMap map,
+                                                              const __grid_constant__ PeerBases peers) {
+  const int row = Hd * vec_per_row;  // vectors of one token inside a block
+  const int64_t threads = static_cast<int64_t>(gridDim.x) * blockDim.x;  // a multiple of `row`
+  const int64_t t0 = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int in_row = static_cast<int>(t0 % row);
+  const int hh = in_row / vec_per_row, v = in_row - hh * vec_per_row;
+  const int64_t tok_step = threads / row;
+  int64_t tok = t0 / row;
+  int p = 0;
+  for (;;) {
+    while (tok >= T && p < n) tok -= T, ++p;
+    if (p >= n) break;
+    int lo = 0, hi = n_samples - 1;  // the sample the token belongs to: sample_off ascending, sample_off[0] = 0
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (sample_off[mid] <= tok) lo = mid; else hi = mid - 1;
+    }
+    const int64_t r = dst_row[static_cast<int64_t>(p) * n_samples + lo] + (tok - sample_off[lo]);
+    peers.base[p][r * row + in_row] = __ldg(src + (tok * H + map.first_head[p] + hh) * vec_per_row + v);
+    tok += tok_step;
+  }
+}
+
 // one thread per 16 bytes of the [T, H, D] side; the blocks that carry the thread's head are found once, the common
 // case of exactly one is a plain copy (two tokens per pass, so that two loads are in flight), several are added in
 // block order in fp32
@@ -190,6 +226,31 @@ extern "C" int nsp_a2a_scatter_heads(const void* src, void* dst, int64_t tokens,
   else
     scatter_heads_kernel<false><<<grid_for(total, heads * vec), 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
                                                                  tokens, heads, heads_per_block, n_blocks, vec, map);
+  nsp::count_launches(1);
+  return cudaGetLastError() == cudaSuccess ? NSP_OK : NSP_ERR_CUDA;
+}
+
+extern "C" int nsp_a2a_gather_heads_to(const void* src, void* const* dst_base, const int64_t* dst_row,
+                                       const int64_t* sample_off, int32_t n_samples, int64_t tokens, int32_t heads,
+                                       int32_t heads_per_block, int32_t n_blocks, int32_t head_dim, int32_t dtype,
+                                       const int32_t* first_head, void* stream) {
+  if (!dst_base || n_samples < 0 || n_blocks <= 0 || n_blocks > NSP_A2A_MAX_PEERS) return NSP_ERR_INVALID_ARG;
+  HeadMap map = {};
+  // the shared checks want one destination pointer: every block's base has to pass them
+  PeerBases peers = {};
+  for (int p = 0; p < n_blocks; ++p) {
+    const int rc = check(src, dst_base[p], tokens, heads, heads_per_block, n_blocks, head_dim, dtype, first_head, &map);
+    if (rc != NSP_OK) return rc;
+    peers.base[p] = static_cast<uint4*>(dst_base[p]);
+  }
+  if (tokens == 0) return NSP_OK;
+  if (n_samples == 0 || !dst_row || !sample_off) return NSP_ERR_INVALID_ARG;
+  const int vec = head_dim * (dtype == NSP_F32 ? 4 : 2) / 16;
+  const int64_t total = tokens * heads_per_block * vec * n_blocks;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  gather_heads_to_kernel<<<grid_for(total, heads_per_block * vec), 256, 0, st>>>(
+      static_cast<const uint4*>(src), tokens, heads, heads_per_block, n_blocks, vec, n_samples, sample_off, dst_row, map,
+      peers);
   nsp::count_launches(1);
   return cudaGetLastError() == cudaSuccess ? NSP_OK : NSP_ERR_CUDA;
 }

@@ -33,6 +33,13 @@ class CudaLayoutOps:
 
         B.nsp_a2a_scatter_heads(src, dst, tokens, heads, heads_per_block, head_dim, first_head, stream)
 
+    def gather_to(self, src, dst_tensors, dst_row, sample_off, tokens, heads, heads_per_block, head_dim, first_head,
+                  stream=None):
+        from . import binding as B
+
+        B.nsp_a2a_gather_heads_to(src, dst_tensors, dst_row, sample_off, tokens, heads, heads_per_block, head_dim,
+                                  first_head, stream)
+
 
 @dataclass
 class NodeLayout:
@@ -129,6 +136,27 @@ class UlyssesExchange:
 
         self._exchange(send_of, recv_of)
         return out
+
+    def store_to_attention_layouts(self, x_loc, kind, peer_buffers, stream=None):
+        """The prologue without a staging buffer and without a separate exchange: this GPU's token slices go, head block
+        by head block, straight into the packed attention buffers of the node's GPUs. peer_buffers[p] is GPU p's
+        [t_full, H / d, D] buffer as a tensor this process can write (its own for p == rank; a peer's memory mapped
+        into this process otherwise, e.g. through CUDA IPC or a symmetric-memory allocation). One kernel of the library
+        issues plain stores; the caller orders it against the readers (every GPU of the node runs this call, then the
+        group synchronises, then attention runs)."""
+        import torch
+
+        lay = self.lay
+        H, h_loc, first = lay.heads(kind)
+        D = lay.head_dim
+        x_loc = x_loc.reshape(lay.t_loc, H, D)
+        if len(peer_buffers) != lay.degree:
+            raise ValueError("one attention buffer per GPU of the node")
+        # this GPU holds the token range [rank L_j / d, (rank + 1) L_j / d) of sample j, for every receiver alike
+        rows = [[int(lay.full_off[j]) + lay.rank * lay.tok_loc[j] for j in range(len(lay.lengths))]] * lay.degree
+        dst_row = torch.tensor(rows, dtype=torch.int64, device=x_loc.device)
+        sample_off = torch.as_tensor(lay.loc_off, dtype=torch.int64).to(x_loc.device)
+        self.ops.gather_to(x_loc, list(peer_buffers), dst_row, sample_off, lay.t_loc, H, h_loc, D, first, stream)
 
     def from_attention_layout(self, y_full, kind, out=None, stream=None):
         """The reverse: y_full [t_full, H / d, D] -> [t_loc, H, D]. Blocks that carry the same head (partial dK / dV of

@@ -32,6 +32,15 @@ class TorchLayoutOps:
                 dst[:, h] = acc.to(dst.dtype)
 
 
+    def gather_to(self, src, dst_tensors, dst_row, sample_off, tokens, heads, hpb, D, first, stream=None):
+        src = src.reshape(tokens, heads, D)
+        off = [int(x) for x in sample_off.tolist()]
+        for p, f in enumerate(first):
+            for j in range(len(off) - 1):
+                r = int(dst_row[p][j])
+                dst_tensors[p].reshape(-1, hpb, D)[r:r + off[j + 1] - off[j]] = src[off[j]:off[j + 1], f:f + hpb]
+
+
 def _global(lengths, H, D, seed, dtype=torch.float32):
     g = torch.Generator().manual_seed(seed)
     return [torch.randn(L, H, D, generator=g).to(dtype) for L in lengths]
@@ -87,11 +96,31 @@ def _free_port():
         return s.getsockname()[1]
 
 
-@pytest.mark.parametrize("world,hq,hkv", [(2, 8, 4), (2, 4, 1), (4, 8, 2), (4, 8, 8)])
+@pytest.mark.parametrize("world,hq,hkv", [(2, 8, 4), (2, 4, 1), (4, 8, 2), (4, 8, 8), (8, 32, 4), (8, 8, 2)])
 def test_exchange_schedule_on_cpu_ranks(world, hq, hkv):
     import torch.multiprocessing as mp
 
     mp.spawn(_worker, args=(world, _free_port(), hq, hkv), nprocs=world, join=True)
+
+
+@pytest.mark.parametrize("d,hq,hkv", [(2, 8, 4), (4, 8, 2), (8, 32, 4)])
+def test_fused_prologue_rows_on_cpu(d, hq, hkv):
+    """Where the fused send side puts every block: all ranks of a node in one process, the stores done by the plain
+    torch stand-in; every rank's attention buffer must come out as the global slicing."""
+    from paper_2609_22755_b200.ulysses import NodeLayout, UlyssesExchange
+
+    D = 16
+    lengths = [8 * d, 0, 3 * d, 20 * d]
+    for kind, H, seed in (("q", hq, 1), ("kv", hkv, 2)):
+        xs = _global(lengths, H, D, seed)
+        lays = [NodeLayout(lengths, d, r, hq, hkv, D) for r in range(d)]
+        _, h_loc, first = lays[0].heads(kind)
+        bufs = [torch.full((lays[0].t_full, h_loc, D), float("nan")) for _ in range(d)]
+        for r, lay in enumerate(lays):
+            UlyssesExchange(lay, list(range(d)), ops=TorchLayoutOps()).store_to_attention_layouts(
+                _local(xs, d, r).contiguous(), kind, bufs)
+        for r in range(d):
+            assert torch.equal(bufs[r], torch.cat([x[:, first[r]:first[r] + h_loc] for x in xs]))
 
 
 def test_layout_rejects_bad_shapes():
@@ -144,6 +173,17 @@ def test_cuda_layout_kernels_and_one_process_emulation(d, hq, hkv, dtype):
                     a = int(lay.full_off[j]) + s * lay.tok_loc[j]
                     full[a:a + lay.tok_loc[j]] = sends[kind, s][r, int(lay.loc_off[j]):int(lay.loc_off[j + 1])]
             assert torch.equal(full, torch.cat([x[:, first[r]:first[r] + h_loc] for x in xs]))
+    # the fused send side: every "rank" stores its slices straight into the attention buffers of all ranks (all of
+    # them local here: one GPU stands for the node); the buffers must equal the global slicing bit for bit
+    from paper_2609_22755_b200.ulysses import UlyssesExchange
+
+    for kind, xs in (("q", q), ("kv", kv)):
+        H, h_loc, first = lays[0].heads(kind)
+        bufs = [torch.full((lays[0].t_full, h_loc, D), float("nan"), dtype=dtype, device=dev) for _ in range(d)]
+        for r, lay in enumerate(lays):
+            UlyssesExchange(lay, list(range(d))).store_to_attention_layouts(_local(xs, d, r).contiguous(), kind, bufs)
+        for r in range(d):
+            assert torch.equal(bufs[r], torch.cat([x[:, first[r]:first[r] + h_loc] for x in xs]))
     # scatter: inverse for q; sums for shared KV heads
     for kind in ("q", "kv"):
         lay = lays[0]
