@@ -75,7 +75,12 @@ typedef struct {
   int32_t seg, head, tile, cost;
 } nsp_tile_t;
 
-/* bm / bn: query / key tile rows (built: 128 / 128). order_version: 1. flags: 0. */
+/* bm / bn: query / key tile rows (built: 128 / 128). order_version: 1. flags: 0, or NSP_PLAN_DETERMINISTIC_DQ:
+ * the backward pass then adds the dQ tiles of a (segment, q head, q tile) in key-tile order (a turn counter per tile,
+ * taken with the library's bounded wait), so that dQ, like O, LSE, dK and dV, comes out bit for bit the same in every
+ * run and for every packing order; bwd_ws_bytes grows by 4 bytes per (q head, q tile). Without the flag the tiles
+ * are added in arrival order with floating-point reductions: equal up to the rounding of an fp32 sum. */
+#define NSP_PLAN_DETERMINISTIC_DQ 1
 typedef struct {
   int32_t bm, bn, order_version, flags;
 } nsp_plan_opts;

@@ -32,6 +32,7 @@ struct nsp_plan {
   nsp_tile_t* d_bwd_exec = nullptr;  // the backward items in the order the kernel walks them (see build_bwd_exec_order)
   nsp_tile_t* d_bwd_first = nullptr;  // one item per (segment, kv head): the first-tile kernel's list
   int64_t n_first = 0;
+  bool deterministic = false;         // plan option: dQ tiles added in key-tile order
   int32_t max_len = 0;                // longest segment: no preprocess / main / postprocess launch when <= 128
   int32_t* d_front = nullptr;        // [n_bwd / kFrontBlock + 1] start-alignment counters of the backward kernel
   int32_t* d_counters = nullptr;  // [0] forward cursor, [1] backward cursor
@@ -191,7 +192,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     if (opts->bm <= 0 || opts->bn <= 0) return NSP_ERR_INVALID_ARG;
     bm = opts->bm;
     bn = opts->bn;
-    if (opts->order_version != 1 || opts->flags != 0) return NSP_ERR_UNSUPPORTED;
+    if (opts->order_version != 1 || (opts->flags & ~NSP_PLAN_DETERMINISTIC_DQ) != 0) return NSP_ERR_UNSUPPORTED;
   }
   if (head_dim != kHeadDim) return NSP_ERR_UNSUPPORTED;
   if (bm != kBM || bn != kBN) return NSP_ERR_UNSUPPORTED;
@@ -200,6 +201,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
   nsp_plan* p = new (std::nothrow) nsp_plan;
   if (!p) return NSP_ERR_ALLOC;
   p->n_seg = n_seg;
+  p->deterministic = opts && (opts->flags & NSP_PLAN_DETERMINISTIC_DQ) != 0;
   p->bm = bm;
   p->bn = bn;
   std::vector<int64_t> row_base, fwd_base, bwd_base;
@@ -239,6 +241,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     sg.hkv = hkv[s];
     sg.run = static_cast<int32_t>(p->runs.size() - 1);
     sg.tok_in_run = static_cast<int32_t>(run.tokens);
+    sg.turn_off = static_cast<int32_t>(nf);  // one turn counter per forward item = (q head, q tile) of the segment
     run.tokens += L;
     row_base[s] = lse_off;
     fwd_base[s] = nf;
@@ -366,8 +369,10 @@ int nsp_plan_sizes(const nsp_plan_t* plan, int64_t* q_elems, int64_t* kv_elems, 
   if (kv_elems) *kv_elems = plan->kv_elems;
   if (lse_elems) *lse_elems = plan->lse_elems;
   if (fwd_ws_bytes) *fwd_ws_bytes = 0;
-  if (bwd_ws_bytes)
-    *bwd_ws_bytes = align_up(static_cast<size_t>(plan->q_elems) * 4, 256) + align_up(static_cast<size_t>(plan->lse_elems) * 4, 256);
+  if (bwd_ws_bytes)  // fp32 dQ accumulator, delta, and (deterministic dQ) one turn counter per (q head, q tile)
+    *bwd_ws_bytes = align_up(static_cast<size_t>(plan->q_elems) * 4, 256) +
+                    align_up(static_cast<size_t>(plan->lse_elems) * 4, 256) +
+                    (plan->deterministic ? align_up(static_cast<size_t>(plan->n_fwd) * 4, 256) : 0);
   return NSP_OK;
 }
 
@@ -454,6 +459,10 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   char* wsb = static_cast<char*>(ws);
   float* dq_acc = static_cast<float*>(ws);
   float* delta = reinterpret_cast<float*>(wsb + align_up(static_cast<size_t>(plan->q_elems) * 4, 256));
+  int32_t* dq_turn = plan->deterministic
+                         ? reinterpret_cast<int32_t*>(wsb + align_up(static_cast<size_t>(plan->q_elems) * 4, 256) +
+                                                      align_up(static_cast<size_t>(plan->lse_elems) * 4, 256))
+                         : nullptr;
   float* lse_ws = reinterpret_cast<float*>(wsb + base);
   uint8_t* d_mask = reinterpret_cast<uint8_t*>(wsb + base + align_up(static_cast<size_t>(plan->lse_elems) * 4, 256));
 
@@ -498,6 +507,9 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   // Segments of at most 128 tokens are finished by the first-tile kernel alone; a batch made only of such segments
   // needs no accumulator, no delta and no conversion pass.
   const bool multi = plan->max_len > kBM;
+  if (dq_turn && multi &&
+      cudaMemsetAsync(dq_turn, 0, static_cast<size_t>(plan->n_fwd) * 4, st) != cudaSuccess)
+    return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_PRE, 0, st);
   if (multi || recompute) {
     if (launch_bwd_preprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems,
@@ -515,6 +527,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   a.dq_acc = dq_acc;
   a.dq = dq;
   a.dq_f32 = dq_dtype == NSP_F32;
+  a.dq_turn = dq_turn;
   a.front = plan->d_front;
   a.dk = dk;
   a.dv = dv;

@@ -64,6 +64,7 @@ struct ItemCtx {
   int32_t len, hq, hkv, run, tok0;
   int32_t g, n;                    // kv head, key tile
   int32_t G;                       // q heads per kv head
+  int32_t turn_off, mt;            // deterministic dQ: the segment's first turn counter, its q tiles
   int32_t first;                   // key tile 0
   int32_t m0;                      // first (lowest) q tile of the walk
   int32_t per_head;                // steps per q head
@@ -155,7 +156,11 @@ struct QRing {
 // bf16-rounded O. Its dQ rows are complete (no other key tile reaches q tile 0) and are stored directly; its dK / dV
 // rows are the whole result for a one-tile segment and otherwise the part the main kernel, which runs after it, adds
 // its own sum to.
-template <bool FIRST>
+// DET (main kernel only): the dQ tiles of the key tiles 0, 1, 2, ... of a (segment, q head, q tile) are added to the
+// accumulator in exactly that order: a dQ warp waits (bounded) until the turn counter of its q tile says that the key
+// tiles before its own are done, adds, and passes the turn on. In lock-step the CTAs of neighbouring key tiles then
+// follow one another a reduction apart instead of all adding at once.
+template <bool FIRST, bool DET>
 __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   BwdSmem<FIRST>& s = *reinterpret_cast<BwdSmem<FIRST>*>(smem_raw);
@@ -228,6 +233,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         x.len = sg.len, x.hq = sg.hq, x.hkv = sg.hkv, x.run = sg.run, x.tok0 = sg.tok_in_run;
         x.g = item.head, x.n = item.tile;
         x.G = sg.hq / sg.hkv;
+        x.turn_off = sg.turn_off, x.mt = (sg.len + kBM - 1) / kBM;
         x.first = (item.tile == 0);
         if constexpr (FIRST) {
           x.m0 = 0;
@@ -564,6 +570,25 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           continue;
         }
         float* p0 = tile0 + colhalf * 64 * q_stride;
+        int32_t* turn = nullptr;
+        if constexpr (DET) turn = a.dq_turn + c.turn_off + h * c.mt + m;
+        auto wait_turn = [&]() -> bool {  // key tiles 0 .. n-1 have added their tiles (eight dQ warps each)
+          bool okt = true;
+          if (lane == 0) {
+            const long long t0 = clock64();
+            while (*reinterpret_cast<volatile int32_t*>(turn) < 8 * c.n) {
+              if (clock64() - t0 > NSP_WAIT_CYCLES) { okt = false; break; }
+              __nanosleep(64);
+            }
+            __threadfence();
+          }
+          return __shfl_sync(0xffffffffu, okt, 0);
+        };
+        auto pass_turn = [&]() {
+          __threadfence();  // this lane's reductions are performed before the counter moves
+          __syncwarp();
+          if (lane == 0) atomicAdd(turn, 1);
+        };
         if (n_valid >= 64) {  // interior tile: no row checks
           uint32_t v0[32], v1[32];
           tmem_ld32(tR1 + lane_off + colhalf * 64, v0);
@@ -571,6 +596,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           tmem_wait_ld();
           tc_fence_before_sync();
           mbar_arrive(&s.bar_dq_empty);  // R1 is drained: the next dP^T may overwrite it
+          if constexpr (DET) {
+            if (!wait_turn()) {
+              if (lane == 0) {
+                report_timeout(a.status, c.it, kWhereBwdTurn, vt);
+                *abort_flag = 1;
+              }
+              break;
+            }
+          }
           // The reductions sit in a conditional region on purpose (the condition always holds): as straight-line
           // code the compiler computes all 64 row addresses ahead of the TMEM loads, runs out of the 80 registers
           // this role has and spills inside the loop (measured: the whole kernel 25 % slower).
@@ -584,7 +618,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               p1 += q_stride;
             }
           }
+          if constexpr (DET) pass_turn();
         } else {  // ragged tail: 16 columns at a time, each row checked
+          bool okt = true;
 #pragma unroll 1
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t v[16];
@@ -594,11 +630,25 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               tc_fence_before_sync();
               mbar_arrive(&s.bar_dq_empty);
             }
+            if constexpr (DET) {
+              if (ch == 0) okt = wait_turn();
+              if (!okt) continue;
+            }
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
               if (c.hq > 0 && ch * 16 + e < n_valid) red_add_f32(p0, __uint_as_float(v[e]));
               p0 += q_stride;
             }
+          }
+          if constexpr (DET) {
+            if (!okt) {
+              if (lane == 0) {
+                report_timeout(a.status, c.it, kWhereBwdTurn, vt);
+                *abort_flag = 1;
+              }
+              break;
+            }
+            pass_turn();
           }
         }
       }
@@ -1050,24 +1100,25 @@ cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t
 }
 
 namespace {
-template <bool FIRST>
+template <bool FIRST, bool DET>
 cudaError_t launch_bwd_t(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
   if (args.n_items == 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(bwd_kernel<FIRST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(bwd_kernel<FIRST, DET>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(sizeof(BwdSmem<FIRST>)));
   if (e != cudaSuccess) return e;
   const int grid = args.n_items < num_sms ? args.n_items : num_sms;
-  bwd_kernel<FIRST><<<grid, kBwdThreads, sizeof(BwdSmem<FIRST>), st>>>(maps, args);
+  bwd_kernel<FIRST, DET><<<grid, kBwdThreads, sizeof(BwdSmem<FIRST>), st>>>(maps, args);
   count_launches(1);
   return cudaGetLastError();
 }
 }  // namespace
 
 cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
-  return launch_bwd_t<false>(maps, args, num_sms, st);
+  return args.dq_turn ? launch_bwd_t<false, true>(maps, args, num_sms, st)
+                      : launch_bwd_t<false, false>(maps, args, num_sms, st);
 }
 cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
-  return launch_bwd_t<true>(maps, args, num_sms, st);
+  return launch_bwd_t<true, false>(maps, args, num_sms, st);
 }
 
 cudaError_t launch_bwd_postprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,

@@ -22,7 +22,8 @@ struct SegInfo {
   int32_t run;         // index of the run (dense [T, H, D] tensor) the segment belongs to
   int32_t tok_in_run;  // first token of the segment, relative to the run
   int32_t run_tokens;  // tokens of the whole run (extent of its tensor maps)
-  int32_t pad_[2];
+  int32_t turn_off;    // index of the segment's first (q head, q tile) turn counter (deterministic dQ): + h * Mt + m
+  int32_t pad_;
 };
 static_assert(sizeof(SegInfo) == 56 || sizeof(SegInfo) == 64, "SegInfo layout");
 
@@ -71,6 +72,7 @@ enum DeviceWhere : int32_t {
   kWhereBwdDsReady = 24,
   kWhereBwdItemBarrier = 25,
   kWhereBwdTmemBase = 26,
+  kWhereBwdTurn = 27,  // deterministic dQ: the key tiles before this one did not finish their additions
   kWhereSelfTest = 90,
 };
 
@@ -124,6 +126,7 @@ struct BwdArgs {
   float* dq_acc;  // fp32 [q_elems]; rows 128.. of every segment zeroed before the launch (main kernel)
   void* dq;       // first-tile kernel: rows 0..127 of every segment are stored here directly
   int32_t dq_f32;
+  int32_t* dq_turn;  // deterministic dQ: one counter per (segment, q head, q tile), zeroed before the launch; else null
   void* dk;
   void* dv;
   int32_t dkv_f32;
@@ -147,7 +150,7 @@ cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t
                                   const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, float* dq_acc,
                                   const uint8_t* seg_skip, const float* lse_in, float* lse_out, cudaStream_t st);
 cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st);
-cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st);
+cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st);  // args.dq_turn selects the deterministic variant
 cudaError_t launch_bwd_postprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
                                    const float* dq_acc, void* dq, int dq_f32, float scale, cudaStream_t st);
 void count_launches(int n);

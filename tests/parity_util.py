@@ -35,7 +35,7 @@ def check(name, got, want, max_abs_tol=MAX_ABS_TOL, rel_tol=REL_L2_TOL):
 class GpuRun:
     """Device buffers + one forward/backward through the C ABI for a workload."""
 
-    def __init__(self, w, tensors=None, dq_dtype="bf16", dkv_dtype="f32", device="cuda:0"):
+    def __init__(self, w, tensors=None, dq_dtype="bf16", dkv_dtype="f32", device="cuda:0", deterministic=False):
         import torch
 
         from paper_2609_22755_b200 import binding as B
@@ -45,7 +45,8 @@ class GpuRun:
         self.dev = torch.device(device)
         self.host = tensors if tensors is not None else W.make_tensors(w)
         self.q, self.k, self.v, self.do = (self.host[n].to(self.dev) for n in ("q", "k", "v", "do"))
-        self.plan = B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, w.head_dim)
+        opts = (128, 128, 1, B.NSP_PLAN_DETERMINISTIC_DQ) if deterministic else None
+        self.plan = B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, w.head_dim, opts=opts)
         assert self.plan.q_elems == w.q_elems() and self.plan.kv_elems == w.kv_elems()
         assert self.plan.lse_elems == w.lse_elems()
         # Every buffer the library writes sits between two 4 KiB guard bands filled with a byte pattern; results()

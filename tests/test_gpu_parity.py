@@ -340,6 +340,40 @@ def test_packing_order_invariance_and_reproducibility(env):
         assert np.max(np.abs(x - y) / np.maximum(np.abs(y), 1e-3)) <= 2.0 ** -7
 
 
+def test_deterministic_dq_option_is_bitwise_reproducible(env):
+    """Plan flag NSP_PLAN_DETERMINISTIC_DQ: the dQ tiles are added in key-tile order, so every output, dQ included, is
+    bit for bit the same in two runs and under a permuted packing; and it still matches the oracle."""
+    W, P, torch = env["W"], env["P"], env["torch"]
+    lengths, hq, hkv = [3000, 130, 2048, 700, 64], [8, 8, 4, 4, 4], [2, 2, 1, 1, 1]
+    w = W.custom(lengths, hq, hkv, seed=23)
+    run = P.GpuRun(w, dq_dtype="f32", deterministic=True)
+    outs = []
+    for _ in range(3):
+        for t in (run.dq, run.dk, run.dv):
+            t.fill_(float("nan"))
+        run.forward()
+        run.backward()
+        assert run.status()[0] == 0
+        outs.append(run.results())
+    for n in ("o", "lse", "dq", "dk", "dv"):
+        assert np.array_equal(outs[0][n], outs[1][n]) and np.array_equal(outs[0][n], outs[2][n]), n
+    P.compare_full(w, outs[0], P.oracle_full(w, run.host))
+    qo, kvo, lo = w.q_offsets(), w.kv_offsets(), w.lse_offsets()
+    perm = [2, 3, 4, 0, 1]
+    wp = W.custom([lengths[p] for p in perm], [hq[p] for p in perm], [hkv[p] for p in perm], seed=23)
+    host = {}
+    for name, off in (("q", qo), ("do", qo), ("k", kvo), ("v", kvo)):
+        host[name] = torch.cat([run.host[name][off[p]:off[p + 1]] for p in perm])
+    runp = P.GpuRun(wp, tensors=host, dq_dtype="f32", deterministic=True)
+    runp.forward()
+    runp.backward()
+    c = runp.results()
+    pqo, pkvo, plo = wp.q_offsets(), wp.kv_offsets(), wp.lse_offsets()
+    for new, p in enumerate(perm):
+        for n, off, poff in (("o", qo, pqo), ("lse", lo, plo), ("dq", qo, pqo), ("dk", kvo, pkvo), ("dv", kvo, pkvo)):
+            assert np.array_equal(outs[0][n][off[p]:off[p + 1]], c[n][poff[new]:poff[new + 1]]), (n, p)
+
+
 def _sample_rows(w, rng, per_seg):
     rows = []
     for s in range(w.n_seg):
