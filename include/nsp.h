@@ -17,7 +17,7 @@
  *         LSE_i = ln sum_j exp(S_ij);  P_ij = exp(S_ij - LSE_i);  O[i,h] = sum_j P_ij V[j,g]
  *         dQ, dK, dV = gradients of sum(O * dO); dK/dV are summed over the Hq/Hkv query heads of a KV head.
  *
- * Packed layout ("ragged token-major"), head_dim D = 128:
+ * Packed layout ("ragged token-major"), head_dim D = 128 or 64 (one value per plan):
  *   segment s has L_s = cu_seqlens[s+1]-cu_seqlens[s] tokens, hq[s] query heads and hkv[s] KV heads.
  *   Q, O, dO, dQ : segment s is a contiguous [L_s, hq[s], D] block at element offset D * sum_{t<s} L_t*hq[t].
  *   K, V, dK, dV : segment s is a contiguous [L_s, hkv[s], D] block at element offset D * sum_{t<s} L_t*hkv[t].
@@ -55,7 +55,7 @@ extern "C" {
 enum {
   NSP_OK = 0,
   NSP_ERR_INVALID_ARG = 1,    /* null pointer, bad metadata, misaligned tensor, bad dtype, bad scale */
-  NSP_ERR_UNSUPPORTED = 2,    /* head_dim != 128, too many runs, tile sizes not built, counts out of range */
+  NSP_ERR_UNSUPPORTED = 2,    /* head_dim not 128 or 64, too many runs, tile sizes not built, counts out of range */
   NSP_ERR_ALLOC = 3,          /* host or device allocation failed (plan construction only) */
   NSP_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (including: no device) */
   NSP_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait expired (sticky, see nsp_device_status) */
@@ -94,7 +94,7 @@ typedef struct {
  * cu_seqlens [n_seg+1], hq [n_seg], hkv [n_seg]: host arrays, copied. Zero-length segments and n_seg == 0 are legal.
  * opts may be NULL (= {128,128,1,0}). The lists are built by kernels enqueued on `stream`.
  * Errors: INVALID_ARG (null, n_seg < 0, cu_seqlens[0] != 0, decreasing cu_seqlens, hq/hkv <= 0, hq % hkv != 0),
- * UNSUPPORTED (head_dim != 128, > NSP_MAX_RUNS runs, unsupported tile sizes, >= 65536 segments, > 256 heads,
+ * UNSUPPORTED (head_dim other than 128 or 64, > NSP_MAX_RUNS runs, unsupported tile sizes, >= 65536 segments, > 256 heads,
  * >= 65536 tiles in a segment), ALLOC, CUDA. On error *out_plan is NULL.
  */
 int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* hkv, int32_t n_seg, int32_t head_dim,

@@ -19,7 +19,7 @@ void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed);
 using namespace nsp;
 
 struct nsp_plan {
-  int32_t n_seg = 0, bm = kBM, bn = kBN;
+  int32_t n_seg = 0, bm = kBM, bn = kBN, head_dim = kHeadDim;
   int device = 0, num_sms = 0;
   int64_t q_elems = 0, kv_elems = 0, lse_elems = 0, n_fwd = 0, n_bwd = 0;
   std::vector<SegInfo> seg;
@@ -66,16 +66,16 @@ EncodeTiledFn get_encode_fn() {
 
 // Tensor map of one run: a dense bf16 [tokens, heads, 128] tensor; tiles are {64 dims, 1 head, 128 tokens}
 // with 128-byte swizzle, rows past the run read as zero.
-bool encode_run_map(CUtensorMap* out, const void* base, int64_t elem_off, int64_t tokens, int heads) {
+bool encode_run_map(CUtensorMap* out, const void* base, int64_t elem_off, int64_t tokens, int heads, int head_dim) {
   EncodeTiledFn enc = get_encode_fn();
   if (!enc) return false;
   if (tokens <= 0) {
     std::memset(out, 0, sizeof(*out));
     return true;
   }
-  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(kHeadDim), static_cast<cuuint64_t>(heads),
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(head_dim), static_cast<cuuint64_t>(heads),
                               static_cast<cuuint64_t>(tokens)};
-  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(kHeadDim) * 2, static_cast<cuuint64_t>(heads) * kHeadDim * 2};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(head_dim) * 2, static_cast<cuuint64_t>(heads) * head_dim * 2};
   const cuuint32_t box[3] = {64, 1, 128};
   const cuuint32_t estr[3] = {1, 1, 1};
   void* ptr = const_cast<char*>(static_cast<const char*>(base)) + elem_off * 2;
@@ -194,13 +194,14 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     bn = opts->bn;
     if (opts->order_version != 1 || (opts->flags & ~NSP_PLAN_DETERMINISTIC_DQ) != 0) return NSP_ERR_UNSUPPORTED;
   }
-  if (head_dim != kHeadDim) return NSP_ERR_UNSUPPORTED;
+  if (head_dim != 128 && head_dim != 64) return NSP_ERR_UNSUPPORTED;
   if (bm != kBM || bn != kBN) return NSP_ERR_UNSUPPORTED;
   if (n_seg >= 65536) return NSP_ERR_UNSUPPORTED;
 
   nsp_plan* p = new (std::nothrow) nsp_plan;
   if (!p) return NSP_ERR_ALLOC;
   p->n_seg = n_seg;
+  p->head_dim = head_dim;
   p->deterministic = opts && (opts->flags & NSP_PLAN_DETERMINISTIC_DQ) != 0;
   p->bm = bm;
   p->bn = bn;
@@ -246,8 +247,8 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     row_base[s] = lse_off;
     fwd_base[s] = nf;
     bwd_base[s] = nb;
-    q_off += L * hq[s] * kHeadDim;
-    kv_off += L * hkv[s] * kHeadDim;
+    q_off += L * hq[s] * head_dim;
+    kv_off += L * hkv[s] * head_dim;
     lse_off += L * hq[s];
     nf += Mt * hq[s];
     nb += Nt * hkv[s];
@@ -404,9 +405,9 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   std::memset(&maps, 0, sizeof(maps));
   for (size_t r = 0; r < plan->runs.size(); ++r) {
     const RunInfo& run = plan->runs[r];
-    if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq) ||
-        !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv) ||
-        !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv))
+    if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq, plan->head_dim) ||
+        !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv, plan->head_dim) ||
+        !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv, plan->head_dim))
       return NSP_ERR_CUDA;
   }
   if (cudaMemsetAsync(plan->d_counters, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
@@ -423,7 +424,7 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.d_o = nullptr;
   a.delta = nullptr;
   prof_mark(plan, NSP_KERNEL_FWD, 0, st);
-  if (launch_fwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (launch_fwd(maps, a, plan->head_dim, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_FWD, 1, st);
   return NSP_OK;
 }
@@ -472,10 +473,10 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   if (recompute) std::memset(&fmaps, 0, sizeof(fmaps));
   for (size_t r = 0; r < plan->runs.size(); ++r) {
     const RunInfo& run = plan->runs[r];
-    if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq) ||
-        !encode_run_map(&maps.d_o[r], d_o, run.q_off, run.tokens, run.hq) ||
-        !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv) ||
-        !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv))
+    if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq, plan->head_dim) ||
+        !encode_run_map(&maps.d_o[r], d_o, run.q_off, run.tokens, run.hq, plan->head_dim) ||
+        !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv, plan->head_dim) ||
+        !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv, plan->head_dim))
       return NSP_ERR_CUDA;
     if (recompute) fmaps.q[r] = maps.q[r], fmaps.k[r] = maps.k[r], fmaps.v[r] = maps.v[r];
   }
@@ -501,7 +502,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
     fa.d_o = static_cast<const __nv_bfloat16*>(d_o);
     fa.delta = delta;
     prof_mark(plan, NSP_KERNEL_FWD, 0, st);
-    if (launch_fwd(fmaps, fa, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+    if (launch_fwd(fmaps, fa, plan->head_dim, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
     prof_mark(plan, NSP_KERNEL_FWD, 1, st);
   }
   // Segments of at most 128 tokens are finished by the first-tile kernel alone; a batch made only of such segments
@@ -512,7 +513,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
     return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_PRE, 0, st);
   if (multi || recompute) {
-    if (launch_bwd_preprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems,
+    if (launch_bwd_preprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems, plan->head_dim,
                               static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta,
                               dq_acc, recompute ? d_mask : nullptr, recompute ? lse : nullptr,
                               recompute ? lse_ws : nullptr, st) != cudaSuccess)
@@ -539,17 +540,17 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   a.n_items = static_cast<int32_t>(plan->n_first);
   a.counter = plan->d_counters + 2;
   prof_mark(plan, NSP_KERNEL_BWD_FIRST, 0, st);
-  if (launch_bwd_first(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (launch_bwd_first(maps, a, plan->head_dim, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_FIRST, 1, st);
   // main kernel: everything else
   a.items = plan->d_bwd_exec;
   a.n_items = static_cast<int32_t>(plan->n_bwd);
   a.counter = plan->d_counters + 1;
   prof_mark(plan, NSP_KERNEL_BWD_MAIN, 0, st);
-  if (multi && launch_bwd(maps, a, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (multi && launch_bwd(maps, a, plan->head_dim, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_MAIN, 1, st);
   prof_mark(plan, NSP_KERNEL_BWD_POST, 0, st);
-  if (multi && launch_bwd_postprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems, dq_acc, dq,
+  if (multi && launch_bwd_postprocess(plan->d_seg, plan->n_seg, plan->d_row_base, plan->lse_elems, plan->head_dim, dq_acc, dq,
                                       dq_dtype == NSP_F32, softmax_scale, st) != cudaSuccess)
     return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_BWD_POST, 1, st);

@@ -47,7 +47,6 @@ namespace {
 
 constexpr int kBwdThreads = 640;  // 8 softmax warps, 8 dQ warps, one auxiliary warpgroup
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;
-constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 // setmaxnreg redistributes the launch-time allocation (96 per thread): 256*136 + 256*80 + 128*48 = 640*96
@@ -74,14 +73,14 @@ struct ItemCtx {
 // FIRST: the first-tile kernel also keeps the bf16 residual of dS^T. The main kernel does without those 32 KB on
 // purpose: shared memory it does not claim stays with the L1 cache, and the kernel ran 3 % slower with the larger
 // carve-out (the same 3 % the step from a three-stage to a two-stage Q ring gained).
-template <bool FIRST>
+template <bool FIRST, int D>
 struct BwdSmem {
-  uint8_t k[2][kHalfTileBytes];
-  uint8_t v[2][kHalfTileBytes];
-  uint8_t q[kQStages][2][kHalfTileBytes];  // [stage][64-column half]: ring, loaded a whole step ahead
-  uint8_t d_o[2][kHalfTileBytes];     // [half]: single buffer (its consumers leave a long window for the refill)
+  uint8_t k[D / 64][kHalfTileBytes];  // K, V, Q, dO tiles: D / 64 sub-tiles of 64 columns (D = head dimension)
+  uint8_t v[D / 64][kHalfTileBytes];
+  uint8_t q[kQStages][D / 64][kHalfTileBytes];  // [stage][64-column half]: ring, loaded a whole step ahead
+  uint8_t d_o[D / 64][kHalfTileBytes];  // [half]: single buffer (its consumers leave a long window for the refill)
   uint8_t ds[2][kHalfTileBytes];      // dS^T, [key row][query col], two 64-column halves
-  uint8_t ds_lo[FIRST ? kTileBytes : 16];  // first-tile kernel: the bf16 residual of dS^T, same layout, right behind it
+  uint8_t ds_lo[FIRST ? 2 * kHalfTileBytes : 16];  // first-tile kernel: the bf16 residual of dS^T, same layout, right behind it
   float lse[2][128];                  // [stage] LSE * log2(e) of the q tile (+inf for rows past the segment)
   float delta[2][128];                // [stage]
   ItemCtx ctx[2];
@@ -100,7 +99,7 @@ struct BwdSmem {
   uint32_t tmem_base;
   int32_t abort;
 };
-static_assert(sizeof(BwdSmem<true>) <= 232448, "shared memory budget (227 KB)");
+static_assert(sizeof(BwdSmem<true, 128>) <= 232448, "shared memory budget (227 KB)");
 
 __device__ __forceinline__ void red_add_f32(float* addr, float v) {
   asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
@@ -160,10 +159,13 @@ struct QRing {
 // accumulator in exactly that order: a dQ warp waits (bounded) until the turn counter of its q tile says that the key
 // tiles before its own are done, adds, and passes the turn on. In lock-step the CTAs of neighbouring key tiles then
 // follow one another a reduction apart instead of all adding at once.
-template <bool FIRST, bool DET>
+template <bool FIRST, bool DET, int D>
 __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  BwdSmem<FIRST>& s = *reinterpret_cast<BwdSmem<FIRST>*>(smem_raw);
+  BwdSmem<FIRST, D>& s = *reinterpret_cast<BwdSmem<FIRST, D>*>(smem_raw);
+  constexpr int kHalves = D / 64;  // 64-column sub-tiles of a K / V / Q / dO tile
+  constexpr uint32_t kOpBytes = kHalves * kHalfTileBytes;  // bytes of such a tile
+  constexpr int kHeadDim = D;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
   // swizzled tiles need a 1024-byte aligned base
   const bool misaligned = (smem_u32(smem_raw) & 1023u) != 0;
@@ -292,11 +294,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           const ItemCtx c = *cx;
           const CUtensorMap* mq = &maps.q[c.run];
           const CUtensorMap* mdo = &maps.d_o[c.run];
-          mbar_expect_tx(&s.bar_kv, 2 * kTileBytes);
-          tma_load_3d(s.k[0], &maps.k[c.run], &s.bar_kv, 0, c.g, c.tok0 + c.n * kBN);
-          tma_load_3d(s.k[1], &maps.k[c.run], &s.bar_kv, 64, c.g, c.tok0 + c.n * kBN);
-          tma_load_3d(s.v[0], &maps.v[c.run], &s.bar_kv, 0, c.g, c.tok0 + c.n * kBN);
-          tma_load_3d(s.v[1], &maps.v[c.run], &s.bar_kv, 64, c.g, c.tok0 + c.n * kBN);
+          mbar_expect_tx(&s.bar_kv, 2 * kOpBytes);
+#pragma unroll
+          for (int hf = 0; hf < kHalves; ++hf) {
+            tma_load_3d(s.k[hf], &maps.k[c.run], &s.bar_kv, 64 * hf, c.g, c.tok0 + c.n * kBN);
+            tma_load_3d(s.v[hf], &maps.v[c.run], &s.bar_kv, 64 * hf, c.g, c.tok0 + c.n * kBN);
+          }
           StepWalk w;
           w.reset();
 #pragma unroll 1
@@ -311,18 +314,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               *abort_flag = 1;
               break;
             }
-            mbar_expect_tx(&s.bar_q_full[qr.st], kTileBytes);
-            tma_load_3d(s.q[qr.st][0], mq, &s.bar_q_full[qr.st], 0, h, c.tok0 + m * kBM);
-            tma_load_3d(s.q[qr.st][1], mq, &s.bar_q_full[qr.st], 64, h, c.tok0 + m * kBM);
+            mbar_expect_tx(&s.bar_q_full[qr.st], kOpBytes);
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf)
+              tma_load_3d(s.q[qr.st][hf], mq, &s.bar_q_full[qr.st], 64 * hf, h, c.tok0 + m * kBM);
             qr.next();
             if (!mbar_wait(&s.bar_do_empty[0], (cs & 1) ^ 1) || !mbar_wait(&s.bar_do_empty[1], (cs & 1) ^ 1)) {
               report_timeout(a.status, c.it, kWhereBwdQEmpty, 100000 + vt);
               *abort_flag = 1;
               break;
             }
-            mbar_expect_tx(&s.bar_do_full, kTileBytes);
-            tma_load_3d(s.d_o[0], mdo, &s.bar_do_full, 0, h, c.tok0 + m * kBM);
-            tma_load_3d(s.d_o[1], mdo, &s.bar_do_full, 64, h, c.tok0 + m * kBM);
+            mbar_expect_tx(&s.bar_do_full, kOpBytes);
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.d_o[hf], mdo, &s.bar_do_full, 64 * hf, h, c.tok0 + m * kBM);
           }
         }
         item_done();
@@ -339,16 +343,20 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       while (next_item()) {
         {
           const bool leader = elect_one();
-          constexpr uint32_t idesc_kk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
-          constexpr uint32_t idesc_kn = make_idesc_bf16(128, 128, 0, 1);  // A K-major (or TMEM), B MN-major
-          constexpr uint32_t idesc_nn = make_idesc_bf16(128, 128, 1, 1);  // A MN-major, B MN-major
+          constexpr uint32_t idesc_kk = make_idesc_bf16(128, 128, 0, 0);  // S^T, dP^T: A K-major, B K-major, contraction over D
+          constexpr uint32_t idesc_kn = make_idesc_bf16(128, D, 0, 1);    // dV, dK: A K-major (or TMEM), B MN-major, N = D
+          constexpr uint32_t idesc_nn = make_idesc_bf16(128, 128, 1, 1);  // dQ^T: A MN-major (M = head dimension), B MN-major
           // Descriptors are {low word, high word}; an operand advances inside its tile by adding the byte offset
           // (in 16-byte units) to the low word (the 14-bit address field cannot overflow: every tile sits below
           // 256 KB). K-major operands step 32 bytes per 16 contraction elements inside a 64-column half;
           // MN-major operands step 16 rows = 2048 bytes. The high word is the same for both kinds.
           const uint32_t hi = static_cast<uint32_t>(make_smem_desc_sw128(0, 16, 1024) >> 32);
           constexpr uint32_t lbo_km = (16u >> 4) << 16, lbo_mn = (kHalfTileBytes >> 4) << 16;
-          constexpr uint32_t kStageStep = kTileBytes >> 4;  // descriptor distance between Q stages
+          // K read MN-major as the A operand of dQ^T has M = head dimension. With D = 64 the product still runs with
+          // M = 128: the second half of the rows repeats the first (leading byte offset 0) and lands in TMEM lanes
+          // 64..127, which nobody reads.
+          constexpr uint32_t lbo_kt = D == 128 ? lbo_mn : 0u;
+          constexpr uint32_t kStageStep = kOpBytes >> 4;  // descriptor distance between Q stages
           const int steps = cx->steps, item_it = cx->it;
           int where = 0;
           bool okm = mbar_wait(&s.bar_kv, gi & 1);
@@ -362,7 +370,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               tc_fence_after_sync();
               const uint32_t b_lo = (q0_lo + qr.st * kStageStep) | lbo_km;
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk) {
+              for (int kk = 0; kk < D / 16; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
                 if (leader) umma_ss_lh(tR0, k_km + off, hi, b_lo + off, hi, idesc_kk, kk > 0);
               }
@@ -406,9 +414,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
 #pragma unroll 1
             for (int vt = 0; okm && vt < steps; ++vt) okm = step_a(vt);
           } else {
-            const uint32_t v_km = smem_desc_addr(s.v[0]) | lbo_km, k_mn = smem_desc_addr(s.k[0]) | lbo_mn;
+            const uint32_t v_km = smem_desc_addr(s.v[0]) | lbo_km, k_mn = smem_desc_addr(s.k[0]) | lbo_kt;
             const uint32_t ds_km = smem_desc_addr(s.ds[0]) | lbo_km, ds_mn = smem_desc_addr(s.ds[0]) | lbo_mn;
-            constexpr uint32_t kLoStep = kTileBytes >> 4;  // descriptor distance from dS^T to its residual
+            constexpr uint32_t kLoStep = (2 * kHalfTileBytes) >> 4;  // descriptor distance from dS^T to its residual
             // dP^T of step vt -> R1, once the dQ warps have drained dQ^T of the previous step from it
             auto issue_dp = [&](int vt) -> bool {
               const uint32_t cs = gs + vt;
@@ -416,7 +424,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               if (!mbar_wait(&s.bar_dq_empty, (cs & 1) ^ 1)) { where = kWhereBwdDqEmpty; return false; }
               tc_fence_after_sync();
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk) {
+              for (int kk = 0; kk < D / 16; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
                 if (leader) umma_ss_lh(tR1, v_km + off, hi, (do_lo | lbo_km) + off, hi, idesc_kk, kk > 0);
               }
@@ -543,6 +551,23 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         const int rows_left = c.len - m * kBM;  // valid query rows of this q tile (>= 128 for an interior tile)
         float* const tile0 = a.dq_acc + c.q_off + (static_cast<int64_t>(m) * kBM * c.hq + h) * kHeadDim + d;
         const int n_valid = min(kBM, rows_left) - colhalf * 64;
+        if constexpr (D < 128) {
+          // dQ^T has D rows: the warps of TMEM lanes D..127 have nothing to drain, they only keep the barrier counts
+          // (and, with ordered additions, the turn counts)
+          if (d >= D) {
+            tc_fence_before_sync();
+            mbar_arrive(&s.bar_dq_empty);
+            if constexpr (DET) {
+              int32_t* turn = a.dq_turn + c.turn_off + h * c.mt + m;
+              if (lane == 0) {
+                const long long t0 = clock64();
+                while (*reinterpret_cast<volatile int32_t*>(turn) < 8 * c.n && clock64() - t0 < NSP_WAIT_CYCLES) __nanosleep(64);
+                atomicAdd(turn, 1);
+              }
+            }
+            continue;
+          }
+        }
         if constexpr (FIRST) {
           // q tile 0 gets nothing from any other key tile: scale and store the rows directly, no accumulator
           uint32_t v0[32], v1[32];
@@ -851,7 +876,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           }
           // Sweep 2: dS^T = P^T o (dP^T - delta), value and residual; P^T (value + residual = P to 2^-17) is read back
           // from R0, which the next S^T does not overwrite before bar_ds_ready.
-          uint8_t* const ds_row_lo = ds_row + kTileBytes;
+          uint8_t* const ds_row_lo = ds_row + 2 * kHalfTileBytes;
 #pragma unroll 1
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t pk[16], dpv[16], dsp[8], dsl[8];
@@ -895,14 +920,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         tc_fence_after_sync();
         const int kj = c.n * kBN + r;
         const bool valid = kj < c.len;
-        const int64_t off = c.kv_off + (static_cast<int64_t>(kj) * c.hkv + c.g) * kHeadDim + half * 64;
+        constexpr int kCols = D / 2;  // this thread's columns of a dK / dV row
+        const int64_t off = c.kv_off + (static_cast<int64_t>(kj) * c.hkv + c.g) * kHeadDim + half * kCols;
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {  // (dK, dV) x two 32-column chunks
-          const int which = part >> 1, cc = part & 1;
+        for (int part = 0; part < 2 * (kCols / 32); ++part) {  // (dK, dV) x 32-column chunks
+          const int which = part / (kCols / 32), cc = part % (kCols / 32);
           const float mul = which == 0 ? a.scale : 1.f;
           void* outp = which == 0 ? a.dk : a.dv;
           uint32_t v[32];
-          tmem_ld32(tDK + which * 128 + lane_off + half * 64 + cc * 32, v);
+          tmem_ld32(tDK + which * 128 + lane_off + half * kCols + cc * 32, v);
           tmem_wait_ld();
           // Key tile 0 in the main kernel: the first-tile kernel, which ran before, left its part (q tile 0) in the
           // output; this item's sum over the q tiles 1 .. Mt-1 is added to it (one fixed order: reproducible).
@@ -968,13 +994,14 @@ __device__ __forceinline__ int find_segment(const int64_t* __restrict__ row_base
 }
 
 // Preprocess, for the rows the main kernel works on (tokens 128.. of every segment; the first 128 tokens belong to
-// the first-tile kernel, which needs neither): delta[h, i] = <dO[i,h,:], O[i,h,:]> and the row's 128 floats of the dQ
-// accumulator set to zero. Rows (token, head) are packed one after the other, 256 bytes each, so the kernel streams
-// O and dO as flat arrays: a warp takes eight consecutive rows per pass, sixteen lanes per row with one 16-byte load
-// per tensor (eight loads in flight per thread), and only the index of the result needs the segment table (delta is
-// stored [head][token] inside a segment): lanes 0..7 look up one row each.
+// the first-tile kernel, which needs neither): delta[h, i] = <dO[i,h,:], O[i,h,:]> and the row's D floats of the dQ
+// accumulator set to zero. Rows (token, head) are packed one after the other, 2 D bytes each, so the kernel streams
+// O and dO as flat arrays: D / 8 lanes per row with one 16-byte load per tensor, four loads in flight per thread
+// and tensor (a warp pass covers 8 rows at D = 128, 16 at D = 64), and only the index of the result needs the
+// segment table (delta is stored [head][token] inside a segment): one lane per row looks it up.
 // With seg_skip, no delta is written for the rows of marked segments (it comes from the recomputation); with lse_out,
-// the LSE of every row whose delta is written is copied from lse_in (same index as delta).
+// the LSE of every row of the other segments is copied from lse_in (same index as delta).
+template <int D>
 __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __restrict__ seg, int n_seg,
                                                              const int64_t* __restrict__ row_base, int64_t total_rows,
                                                              const __nv_bfloat16* __restrict__ o,
@@ -983,27 +1010,28 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
                                                              const uint8_t* __restrict__ seg_skip,
                                                              const float* __restrict__ lse_in,
                                                              float* __restrict__ lse_out) {
-  const int lane = threadIdx.x & 31, sub = lane >> 4, l16 = lane & 15;
-  const int64_t n_groups = (total_rows + 7) >> 3;
+  constexpr int kLanesPerRow = D / 8, kRowsPerLoad = 32 / kLanesPerRow, kRowsPerPass = 4 * kRowsPerLoad;
+  const int lane = threadIdx.x & 31, sub = lane / kLanesPerRow, l = lane % kLanesPerRow;
+  const int64_t n_groups = (total_rows + kRowsPerPass - 1) / kRowsPerPass;
   const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
   for (int64_t grp = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; grp < n_groups; grp += n_warps) {
-    const int64_t row0 = grp * 8;
+    const int64_t row0 = grp * kRowsPerPass;
     uint4 va[4], vb[4];
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
-      const int64_t row = row0 + 2 * p + sub;
+      const int64_t row = row0 + kRowsPerLoad * p + sub;
       if (row < total_rows) {
-        va[p] = __ldg(reinterpret_cast<const uint4*>(o + row * kHeadDim) + l16);
-        vb[p] = __ldg(reinterpret_cast<const uint4*>(d_o + row * kHeadDim) + l16);
+        va[p] = __ldg(reinterpret_cast<const uint4*>(o + row * D) + l);
+        vb[p] = __ldg(reinterpret_cast<const uint4*>(d_o + row * D) + l);
       } else {
         va[p] = vb[p] = make_uint4(0u, 0u, 0u, 0u);
       }
     }
-    // row row0 + (lane & 7): where its delta goes (-1: nowhere), and whether it is one of the main kernel's rows
+    // row row0 + (lane % kRowsPerPass): where its delta goes (-1: nowhere), and whether it is one of the main kernel's rows
     int64_t dst = -1;
     int mine = 0;
     {
-      const int64_t row = row0 + (lane & 7);
+      const int64_t row = row0 + (lane % kRowsPerPass);
       if (row < total_rows) {
         const int sgi = find_segment(row_base, n_seg, row);
         const SegInfo sg = seg[sgi];
@@ -1014,7 +1042,7 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
         // segments the LSE copy covers every row (the first-tile kernel reads it too)
         if (seg_skip == nullptr || seg_skip[sgi] == 0) {
           const int64_t at = sg.lse_off + h * sg.len + i;
-          if (lse_out != nullptr && lane < 8) lse_out[at] = lse_in[at];
+          if (lse_out != nullptr && lane < kRowsPerPass) lse_out[at] = lse_in[at];
           if (mine) dst = at;
         }
       }
@@ -1031,12 +1059,12 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
         acc = fmaf(fa.y, fb.y, acc);
       }
 #pragma unroll
-      for (int sft = 8; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
-      const int64_t dst_p = __shfl_sync(0xffffffffu, dst, 2 * p + sub);
-      const int mine_p = __shfl_sync(0xffffffffu, mine, 2 * p + sub);
-      if (l16 == 0 && dst_p >= 0) delta[dst_p] = acc;
+      for (int sft = kLanesPerRow / 2; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+      const int64_t dst_p = __shfl_sync(0xffffffffu, dst, kRowsPerLoad * p + sub);
+      const int mine_p = __shfl_sync(0xffffffffu, mine, kRowsPerLoad * p + sub);
+      if (l == 0 && dst_p >= 0) delta[dst_p] = acc;
       if (mine_p) {
-        float4* z = reinterpret_cast<float4*>(dq_acc + (row0 + 2 * p + sub) * kHeadDim) + 2 * l16;
+        float4* z = reinterpret_cast<float4*>(dq_acc + (row0 + kRowsPerLoad * p + sub) * D) + 2 * l;
         z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
         z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
@@ -1046,18 +1074,20 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
 
 // Postprocess: dQ = scale * accumulator, in the output dtype, for the rows the main kernel works on (tokens 128.. of
 // every segment; the rows before were stored by the first-tile kernel). Same row walk as the preprocess kernel.
+template <int D>
 __global__ void __launch_bounds__(256) bwd_postprocess_kernel(const SegInfo* __restrict__ seg, int n_seg,
                                                               const int64_t* __restrict__ row_base, int64_t total_rows,
                                                               const float* __restrict__ acc, void* __restrict__ dq,
                                                               int dq_f32, float scale) {
-  const int lane = threadIdx.x & 31, sub = lane >> 4, l16 = lane & 15;
-  const int64_t n_groups = (total_rows + 7) >> 3;
+  constexpr int kLanesPerRow = D / 8, kRowsPerLoad = 32 / kLanesPerRow, kRowsPerPass = 4 * kRowsPerLoad;
+  const int lane = threadIdx.x & 31, sub = lane / kLanesPerRow, l = lane % kLanesPerRow;
+  const int64_t n_groups = (total_rows + kRowsPerPass - 1) / kRowsPerPass;
   const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
   for (int64_t grp = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; grp < n_groups; grp += n_warps) {
-    const int64_t row0 = grp * 8;
+    const int64_t row0 = grp * kRowsPerPass;
     int mine = 0;
     {
-      const int64_t row = row0 + (lane & 7);
+      const int64_t row = row0 + (lane % kRowsPerPass);
       if (row < total_rows) {
         const int sgi = find_segment(row_base, n_seg, row);
         mine = (row - row_base[sgi]) / seg[sgi].hq >= kBM;
@@ -1065,12 +1095,12 @@ __global__ void __launch_bounds__(256) bwd_postprocess_kernel(const SegInfo* __r
     }
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
-      const int64_t row = row0 + 2 * p + sub;
-      if (!__shfl_sync(0xffffffffu, mine, 2 * p + sub)) continue;
-      const float4* src = reinterpret_cast<const float4*>(acc + row * kHeadDim) + 2 * l16;
+      const int64_t row = row0 + kRowsPerLoad * p + sub;
+      if (!__shfl_sync(0xffffffffu, mine, kRowsPerLoad * p + sub)) continue;
+      const float4* src = reinterpret_cast<const float4*>(acc + row * D) + 2 * l;
       const float4 v0 = src[0], v1 = src[1];
       if (dq_f32) {
-        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(dq) + row * kHeadDim) + 2 * l16;
+        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(dq) + row * D) + 2 * l;
         dst[0] = make_float4(v0.x * scale, v0.y * scale, v0.z * scale, v0.w * scale);
         dst[1] = make_float4(v1.x * scale, v1.y * scale, v1.z * scale, v1.w * scale);
       } else {
@@ -1079,7 +1109,7 @@ __global__ void __launch_bounds__(256) bwd_postprocess_kernel(const SegInfo* __r
         w.y = pack_bf16x2(v0.z * scale, v0.w * scale);
         w.z = pack_bf16x2(v1.x * scale, v1.y * scale);
         w.w = pack_bf16x2(v1.z * scale, v1.w * scale);
-        reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(dq) + row * kHeadDim)[l16] = w;
+        reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(dq) + row * D)[l] = w;
       }
     }
   }
@@ -1088,46 +1118,60 @@ __global__ void __launch_bounds__(256) bwd_postprocess_kernel(const SegInfo* __r
 }  // namespace
 
 cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
-                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, float* dq_acc,
-                                  const uint8_t* seg_skip, const float* lse_in, float* lse_out, cudaStream_t st) {
+                                  int head_dim, const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta,
+                                  float* dq_acc, const uint8_t* seg_skip, const float* lse_in, float* lse_out,
+                                  cudaStream_t st) {
   if (total_rows == 0) return cudaSuccess;
-  int64_t blocks = ((total_rows + 7) / 8 * 32 + 255) / 256;  // one warp per eight rows, grid-stride beyond 16 waves
+  int64_t blocks = ((total_rows + 7) / 8 * 32 + 255) / 256;  // about one warp per eight rows, grid-stride beyond 16 waves
   if (blocks > 148 * 8 * 16) blocks = 148 * 8 * 16;
-  bwd_preprocess_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows, o, d_o,
-                                                                       delta, dq_acc, seg_skip, lse_in, lse_out);
+  if (head_dim == 64)
+    bwd_preprocess_kernel<64><<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows, o, d_o,
+                                                                             delta, dq_acc, seg_skip, lse_in, lse_out);
+  else
+    bwd_preprocess_kernel<128><<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows, o, d_o,
+                                                                              delta, dq_acc, seg_skip, lse_in, lse_out);
   count_launches(1);
   return cudaGetLastError();
 }
 
 namespace {
-template <bool FIRST, bool DET>
+template <bool FIRST, bool DET, int D>
 cudaError_t launch_bwd_t(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
   if (args.n_items == 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(bwd_kernel<FIRST, DET>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(sizeof(BwdSmem<FIRST>)));
+  cudaError_t e = cudaFuncSetAttribute(bwd_kernel<FIRST, DET, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(sizeof(BwdSmem<FIRST, D>)));
   if (e != cudaSuccess) return e;
   const int grid = args.n_items < num_sms ? args.n_items : num_sms;
-  bwd_kernel<FIRST, DET><<<grid, kBwdThreads, sizeof(BwdSmem<FIRST>), st>>>(maps, args);
+  bwd_kernel<FIRST, DET, D><<<grid, kBwdThreads, sizeof(BwdSmem<FIRST, D>), st>>>(maps, args);
   count_launches(1);
   return cudaGetLastError();
 }
 }  // namespace
 
-cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
-  return args.dq_turn ? launch_bwd_t<false, true>(maps, args, num_sms, st)
-                      : launch_bwd_t<false, false>(maps, args, num_sms, st);
+cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st) {
+  if (head_dim == 64)
+    return args.dq_turn ? launch_bwd_t<false, true, 64>(maps, args, num_sms, st)
+                        : launch_bwd_t<false, false, 64>(maps, args, num_sms, st);
+  return args.dq_turn ? launch_bwd_t<false, true, 128>(maps, args, num_sms, st)
+                      : launch_bwd_t<false, false, 128>(maps, args, num_sms, st);
 }
-cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
-  return launch_bwd_t<true, false>(maps, args, num_sms, st);
+cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st) {
+  return head_dim == 64 ? launch_bwd_t<true, false, 64>(maps, args, num_sms, st)
+                        : launch_bwd_t<true, false, 128>(maps, args, num_sms, st);
 }
 
 cudaError_t launch_bwd_postprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
-                                   const float* dq_acc, void* dq, int dq_f32, float scale, cudaStream_t st) {
+                                   int head_dim, const float* dq_acc, void* dq, int dq_f32, float scale,
+                                   cudaStream_t st) {
   if (total_rows == 0) return cudaSuccess;
   int64_t blocks = ((total_rows + 7) / 8 * 32 + 255) / 256;
   if (blocks > 148 * 8 * 16) blocks = 148 * 8 * 16;
-  bwd_postprocess_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows, dq_acc,
-                                                                        dq, dq_f32, scale);
+  if (head_dim == 64)
+    bwd_postprocess_kernel<64><<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows,
+                                                                              dq_acc, dq, dq_f32, scale);
+  else
+    bwd_postprocess_kernel<128><<<static_cast<unsigned>(blocks), 256, 0, st>>>(d_seg, n_seg, d_row_base, total_rows,
+                                                                               dq_acc, dq, dq_f32, scale);
   count_launches(1);
   return cudaGetLastError();
 }

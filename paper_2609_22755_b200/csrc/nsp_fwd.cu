@@ -25,7 +25,6 @@ namespace {
 
 constexpr int kFwdThreads = 640;  // 16 softmax warps (two threads per query row) + one auxiliary warpgroup
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;  // one [128 rows x 64 cols] bf16 sub-tile
-constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;
 constexpr uint32_t kFwdTmemCols = 512;  // S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512)
 constexpr int kFwdRegsSoftmax = 104, kFwdRegsAux = 64;  // 4*104 + 64 = 480 = 5 * 96, the launch-time allocation
 
@@ -37,10 +36,12 @@ struct FwdPop {
   int32_t it0, joint, n_rounds, pad_;
 };
 
+// D = head dimension (128 or 64): a Q / K / V tile is D / 64 sub-tiles of 64 columns.
+template <int D>
 struct FwdSmem {
-  uint8_t q[2][2][kHalfTileBytes];  // [A/B][64-column half]
-  uint8_t k[2][2][kHalfTileBytes];  // [stage][half]
-  uint8_t v[2][2][kHalfTileBytes];  // [stage][half]
+  uint8_t q[2][D / 64][kHalfTileBytes];  // [A/B][64-column half]
+  uint8_t k[2][D / 64][kHalfTileBytes];  // [stage][half]
+  uint8_t v[2][D / 64][kHalfTileBytes];  // [stage][half]
   uint64_t bar_q;
   uint64_t bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2];
   uint64_t bar_s_full[2];   // [A/B] S_x of a key tile is in TMEM
@@ -54,8 +55,7 @@ struct FwdSmem {
   FwdPop pop[2];
   int32_t abort;
 };
-static_assert(sizeof(FwdSmem) <= 232448, "shared memory budget (227 KB)");
-constexpr size_t kFwdSmemBytes = sizeof(FwdSmem);
+static_assert(sizeof(FwdSmem<128>) <= 232448, "shared memory budget (227 KB)");
 
 template <int N>
 __device__ __forceinline__ void fwd_setmaxnreg_inc() {
@@ -78,9 +78,14 @@ struct FwdRound {
   nsp_tile_t a, b;
   int joint;
 };
+template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  FwdSmem& s = *reinterpret_cast<FwdSmem*>(smem_raw);
+  FwdSmem<D>& s = *reinterpret_cast<FwdSmem<D>*>(smem_raw);
+  constexpr int kHalves = D / 64;                              // 64-column sub-tiles of a Q / K / V tile
+  constexpr uint32_t kTileBytes = kHalves * kHalfTileBytes;
+  constexpr int kOCols = D / 2;                                // output columns of one of the two threads of a row
+  constexpr int kHeadDim = D;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
   if ((smem_u32(smem_raw) & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
     if (tid == 0) report_timeout(a.status, -1, kWhereFwdSmemAlign, 0);
@@ -185,11 +190,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             const CUtensorMap* mk = &maps.k[sg.run];
             const CUtensorMap* mv = &maps.v[sg.run];
             mbar_expect_tx(&s.bar_q, rd.joint ? 2 * kTileBytes : kTileBytes);
-            tma_load_3d(s.q[0][0], mq, &s.bar_q, 0, ia.head, tok0 + q_row0);
-            tma_load_3d(s.q[0][1], mq, &s.bar_q, 64, ia.head, tok0 + q_row0);
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[0][hf], mq, &s.bar_q, 64 * hf, ia.head, tok0 + q_row0);
             if (rd.joint) {
-              tma_load_3d(s.q[1][0], mq, &s.bar_q, 0, rd.b.head, tok0 + q_row0);
-              tma_load_3d(s.q[1][1], mq, &s.bar_q, 64, rd.b.head, tok0 + q_row0);
+#pragma unroll
+              for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[1][hf], mq, &s.bar_q, 64 * hf, rd.b.head, tok0 + q_row0);
             }
             for (int j = 0; j < n_kv; ++j) {
               if (*abort_flag) break;
@@ -200,8 +205,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 break;
               }
               mbar_expect_tx(&s.bar_k_full[st], kTileBytes);
-              tma_load_3d(s.k[st][0], mk, &s.bar_k_full[st], 0, g, tok0 + j * kBN);
-              tma_load_3d(s.k[st][1], mk, &s.bar_k_full[st], 64, g, tok0 + j * kBN);
+#pragma unroll
+              for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.k[st][hf], mk, &s.bar_k_full[st], 64 * hf, g, tok0 + j * kBN);
               ++kn;
               st = vn & 1;
               if (!mbar_wait(&s.bar_v_empty[st], ((vn >> 1) & 1) ^ 1)) {
@@ -210,8 +215,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 break;
               }
               mbar_expect_tx(&s.bar_v_full[st], kTileBytes);
-              tma_load_3d(s.v[st][0], mv, &s.bar_v_full[st], 0, g, tok0 + j * kBN);
-              tma_load_3d(s.v[st][1], mv, &s.bar_v_full[st], 64, g, tok0 + j * kBN);
+#pragma unroll
+              for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.v[st][hf], mv, &s.bar_v_full[st], 64 * hf, g, tok0 + j * kBN);
               ++vn;
             }
           }
@@ -221,7 +226,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     } else if (warp == 17) {
       // ================================================================ MMA issuer
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);  // A K-major, B K-major
-      constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);  // A from TMEM, B MN-major
+      constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);    // A from TMEM, B MN-major, N = head dimension
       uint32_t qn = 0, kn = 0, vn = 0, pn[2] = {0, 0};
       while (next_pop()) {
         for (int r = 0; r < n_rounds; ++r) {
@@ -244,7 +249,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             auto issue_s = [&](int x, uint32_t kst) {
               const uint32_t a_lo = q_lo + x * kTileStep, b_lo = k_lo + kst * kTileStep;
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk) {
+              for (int kk = 0; kk < D / 16; ++kk) {
                 const uint32_t off = ((kk >> 2) * kHalfTileBytes + (kk & 3) * 32) >> 4;
                 if (leader) umma_ss_lh(tmem + 128 * x, a_lo + off, hi, b_lo + off, hi, idesc_qk, kk > 0);
               }
@@ -427,13 +432,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               if (!ok) { where = kWhereFwdO; break; }
               tc_fence_after_sync();
 #pragma unroll
-              for (int c = 0; c < 2; ++c) {
+              for (int c = 0; c < kOCols / 32; ++c) {
                 uint32_t orow[32];
-                tmem_ld32(tO + lane_off + ch * 64 + c * 32, orow);
+                tmem_ld32(tO + lane_off + ch * kOCols + c * 32, orow);
                 tmem_wait_ld();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) orow[e] = __float_as_uint(__uint_as_float(orow[e]) * alpha);
-                tmem_st32(tO + lane_off + ch * 64 + c * 32, orow);
+                tmem_st32(tO + lane_off + ch * kOCols + c * 32, orow);
               }
             }
             tmem_wait_st();
@@ -463,12 +468,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             // sum.
             tc_fence_after_sync();
             const __nv_bfloat16* dptr =
-                a.d_o + sg.q_off + (static_cast<int64_t>(valid ? row : 0) * sg.hq + h) * kHeadDim + ch * 64;
+                a.d_o + sg.q_off + (static_cast<int64_t>(valid ? row : 0) * sg.hq + h) * kHeadDim + ch * kOCols;
             float part = 0.f;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < kOCols / 32; ++c) {
               uint32_t orow[32];
-              tmem_ld32(tO + lane_off + ch * 64 + c * 32, orow);
+              tmem_ld32(tO + lane_off + ch * kOCols + c * 32, orow);
               uint4 dv4[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) dv4[e] = __ldg(reinterpret_cast<const uint4*>(dptr + c * 32) + e);
@@ -517,11 +522,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             l += partner_slot[256];
             tc_fence_after_sync();
             const float inv_l = 1.f / l;
-            __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim + ch * 64;
+            __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim + ch * kOCols;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < kOCols / 32; ++c) {
               uint32_t orow[32];
-              tmem_ld32(tO + lane_off + ch * 64 + c * 32, orow);
+              tmem_ld32(tO + lane_off + ch * kOCols + c * 32, orow);
               tmem_wait_ld();
               if (valid) {
 #pragma unroll
@@ -554,16 +559,23 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
 
 }  // namespace
 
-cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st) {
-  if (args.n_items == 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kFwdSmemBytes));
+namespace {
+template <int D>
+cudaError_t launch_fwd_t(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(sizeof(FwdSmem<D>)));
   if (e != cudaSuccess) return e;
   const int pops = (args.n_items + 1) / 2;
   const int grid = pops < num_sms ? pops : num_sms;
-  fwd_kernel<<<grid, kFwdThreads, kFwdSmemBytes, st>>>(maps, args);
+  fwd_kernel<D><<<grid, kFwdThreads, sizeof(FwdSmem<D>), st>>>(maps, args);
   count_launches(1);
   return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int head_dim, int num_sms, cudaStream_t st) {
+  if (args.n_items == 0) return cudaSuccess;
+  return head_dim == 64 ? launch_fwd_t<64>(maps, args, num_sms, st) : launch_fwd_t<128>(maps, args, num_sms, st);
 }
 
 }  // namespace nsp

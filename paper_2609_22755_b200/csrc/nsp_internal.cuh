@@ -141,18 +141,20 @@ cudaError_t launch_plan_build(const SegInfo* d_seg, int n_seg, int bm, int bn, n
                               size_t sort_tmp_bytes, const int64_t* d_fwd_base, const int64_t* d_bwd_base,
                               cudaStream_t st);
 size_t plan_sort_tmp_bytes(int64_t max_items);
-cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st);
+cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int head_dim, int num_sms, cudaStream_t st);
 // The backward launches, in the order they run: preprocess (delta and zeroed accumulator rows for tokens 128.. of
 // every segment), first-tile kernel (q tile 0 of every segment: its dQ rows, and its part of dK / dV), main kernel,
 // postprocess (tokens 128..). seg_skip (may be null): segments whose delta is left alone; lse_in / lse_out (may be
 // null): LSE copied for the rows whose delta is written.
 cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
-                                  const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta, float* dq_acc,
-                                  const uint8_t* seg_skip, const float* lse_in, float* lse_out, cudaStream_t st);
-cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st);
-cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st);  // args.dq_turn selects the deterministic variant
+                                  int head_dim, const __nv_bfloat16* o, const __nv_bfloat16* d_o, float* delta,
+                                  float* dq_acc, const uint8_t* seg_skip, const float* lse_in, float* lse_out,
+                                  cudaStream_t st);
+cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st);
+cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st);  // args.dq_turn selects the deterministic variant
 cudaError_t launch_bwd_postprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
-                                   const float* dq_acc, void* dq, int dq_f32, float scale, cudaStream_t st);
+                                   int head_dim, const float* dq_acc, void* dq, int dq_f32, float scale,
+                                   cudaStream_t st);
 void count_launches(int n);
 
 }  // namespace nsp

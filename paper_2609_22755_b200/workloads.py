@@ -99,10 +99,10 @@ def lognormal_lengths(seed: int, budget: int, median: float, sigma: float, lo: i
     return out
 
 
-def _mk(name, lengths, hq, hkv, seed, note=""):
+def _mk(name, lengths, hq, hkv, seed, note="", head_dim=HEAD_DIM):
     cu = np.concatenate([[0], np.cumsum(np.asarray(lengths, dtype=np.int64))])
     assert cu[-1] < 2**31
-    return Workload(name, cu.astype(np.int32), np.asarray(hq, np.int32), np.asarray(hkv, np.int32), HEAD_DIM, seed, note)
+    return Workload(name, cu.astype(np.int32), np.asarray(hq, np.int32), np.asarray(hkv, np.int32), head_dim, seed, note)
 
 
 def config(idx: int, seed: int | None = None, twin: bool = False) -> Workload:
@@ -176,11 +176,11 @@ def ragged(seed: int = 11) -> Workload:
     return _mk("ragged_tails", lengths, hq, hkv, seed, "tail tiles, MQA/GQA/MHA runs, empty segment")
 
 
-def custom(lengths, hq, hkv, seed: int = 0, name: str = "custom") -> Workload:
+def custom(lengths, hq, hkv, seed: int = 0, name: str = "custom", head_dim: int = HEAD_DIM) -> Workload:
     n = len(lengths)
     hq = [hq] * n if np.isscalar(hq) else hq
     hkv = [hkv] * n if np.isscalar(hkv) else hkv
-    return _mk(name, lengths, hq, hkv, seed)
+    return _mk(name, lengths, hq, hkv, seed, head_dim=head_dim)
 
 
 def make_tensors(w: Workload, seed: int | None = None, which=("q", "k", "v", "do")):

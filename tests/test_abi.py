@@ -72,7 +72,7 @@ def test_plan_argument_validation(B):
     assert _plan_rc(B, good[0], [4, 3], good[2]) == B.NSP_ERR_INVALID_ARG  # hq % hkv != 0
     for null in (0, 1, 2):
         assert _plan_rc(B, *good, null=null) == B.NSP_ERR_INVALID_ARG
-    assert _plan_rc(B, *good, head_dim=64) == B.NSP_ERR_UNSUPPORTED
+    assert _plan_rc(B, *good, head_dim=96) == B.NSP_ERR_UNSUPPORTED  # built: 128 and 64
     assert _plan_rc(B, *good, opts=(64, 128, 1, 0)) == B.NSP_ERR_UNSUPPORTED  # tile size not built
     assert _plan_rc(B, *good, opts=(0, 128, 1, 0)) == B.NSP_ERR_INVALID_ARG
     assert _plan_rc(B, *good, opts=(128, 128, 2, 0)) == B.NSP_ERR_UNSUPPORTED  # unknown order version

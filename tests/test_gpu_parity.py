@@ -78,6 +78,33 @@ def test_scaled_down_twins_every_element(env, idx):
     _full_case(env, env["W"].config(idx, twin=True))
 
 
+@pytest.mark.parametrize("case", ["cfg1", "ragged", 2, 3, 4, 5, 6])
+def test_head_dim_64_every_element(env, case):
+    """The same segment structures with head_dim = 64 (softmax scale 1/8): cfg1, the ragged case and the scaled-down
+    twins, every element of every output against the oracle; the tile plan does not depend on the head dimension."""
+    W, P, B, oracle = env["W"], env["P"], env["B"], env["oracle"]
+    base = W.config(1) if case == "cfg1" else W.ragged() if case == "ragged" else W.config(case, twin=True)
+    w = W.custom(base.lengths.tolist(), base.hq.tolist(), base.hkv.tolist(), seed=base.seed, name=base.name + "_d64",
+                 head_dim=64)
+    errs, run, res, ref = _full_case(env, w)
+    for p_ in (0, 1, 2):
+        assert np.array_equal(B.nsp_plan_get(run.plan, p_), oracle.plan_tiles(w.cu_seqlens, w.hq, w.hkv, 128, 128, p_))
+    if case in ("ragged", 6):  # and through the recomputing backward, every second segment dropped
+        torch = env["torch"]
+        flags = (np.arange(w.n_seg) % 2).astype(np.uint8)
+        qo, lo = w.q_offsets(), w.lse_offsets()
+        for s_ in np.nonzero(flags)[0]:
+            run.o[qo[s_]:qo[s_ + 1]] = float("nan")
+            run.lse[lo[s_]:lo[s_ + 1]] = float("nan")
+        ws = torch.empty(B.nsp_plan_recompute_ws_bytes(run.plan), dtype=torch.uint8, device=run.dev)
+        B.nsp_attn_bwd_recompute(run.plan, flags, run.q, run.k, run.v, run.o, run.do, run.lse, run.dq, run.dk, run.dv,
+                                 w.softmax_scale, ws)
+        assert run.status()[0] == 0
+        got = run.results()
+        for name in ("dq", "dk", "dv"):
+            P.check(f"{w.name}:recompute:{name}", got[name], ref[name])
+
+
 def test_peaked_scores_exercise_the_rescale_path(env):
     """Q and K three times larger than in the benchmark data: scores spread over +-40 in log2 units, so the running
     maximum of a row keeps jumping by far more than the lazy-rescale threshold (2^8) from one key tile to the next.
