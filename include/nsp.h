@@ -274,6 +274,20 @@ int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]);
  * Errors: INVALID_ARG, CUDA, or the plan's sticky status. */
 int nsp_selftest_wait_timeout(const nsp_plan_t* plan, int64_t limit_clk, void* stream);
 
+/* How long a device-side wait of this plan's kernels may take before it gives up, in SM clocks (default 4e9, about
+ * two seconds; at least 1000). Every wait on a barrier inside the kernels is bounded by it; when one runs out the kernel
+ * records NSP_ERR_DEVICE_TIMEOUT with the work item and the place, all its roles unwind and the launch ends. Errors:
+ * INVALID_ARG. */
+int nsp_plan_set_wait_limit(nsp_plan_t* plan, int64_t sm_clocks);
+
+#ifdef NSP_CHECKED
+/* Checked build only (libnsp_checked.so, compiled with -DNSP_CHECKED: every index a kernel computes for a global
+ * access is verified first, a failing one is recorded as NSP_ERR_DEVICE_ASSERT and the access skipped). Test switch for
+ * the failure path: with enable != 0 the next forward launch leaves out one V tile load, so that the waits behind it
+ * run out (use a small nsp_plan_set_wait_limit); nothing faults, the launch ends with NSP_ERR_DEVICE_TIMEOUT. */
+int nsp_checked_withhold_load(nsp_plan_t* plan, int enable);
+#endif
+
 /* Kernels of the path, for nsp_plan_kernel_ms. */
 enum {
   NSP_KERNEL_FWD = 0,

@@ -30,8 +30,9 @@ EXPORTS = [
     "nsp_launch_count", "nsp_plan_destroy", "nsp_status_string", "nsp_plan_set_profiling", "nsp_plan_kernel_ms",
     "nsp_attn_bwd_static", "nsp_recompute_mark", "nsp_plan_recompute_ws_bytes", "nsp_attn_bwd_recompute",
     "nsp_cost_table", "nsp_route_sp_tree", "nsp_a2a_gather_heads", "nsp_a2a_scatter_heads",
-    "nsp_selftest_wait_timeout", "nsp_a2a_gather_heads_to",
+    "nsp_selftest_wait_timeout", "nsp_a2a_gather_heads_to", "nsp_plan_set_wait_limit",
 ]
+CHECKED_EXPORTS = ["nsp_checked_withhold_load"]  # libnsp_checked.so only
 NSP_COST_BUCKETS = 16
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
 KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST, KERNEL_BWD_FIRST = 0, 1, 2, 3, 4
@@ -98,6 +99,11 @@ def lib() -> ctypes.CDLL:
         L.nsp_a2a_gather_heads_to.argtypes = [vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
                                               ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
         L.nsp_a2a_gather_heads_to.restype = ctypes.c_int
+        L.nsp_plan_set_wait_limit.argtypes = [vp, ctypes.c_int64]
+        L.nsp_plan_set_wait_limit.restype = ctypes.c_int
+        if hasattr(L, "nsp_checked_withhold_load"):
+            L.nsp_checked_withhold_load.argtypes = [vp, ctypes.c_int]
+            L.nsp_checked_withhold_load.restype = ctypes.c_int
         L.nsp_selftest_wait_timeout.argtypes = [vp, ctypes.c_int64, vp]
         L.nsp_selftest_wait_timeout.restype = ctypes.c_int
         L.nsp_device_status.argtypes = [vp, i32p]
@@ -433,6 +439,21 @@ def nsp_selftest_wait_timeout(plan: Plan, limit_clk: int = 1_000_000, stream=Non
     rc = lib().nsp_selftest_wait_timeout(plan.handle, int(limit_clk), _stream_ptr(stream))
     if rc != NSP_OK:
         raise NspError(rc, "nsp_selftest_wait_timeout")
+
+
+def nsp_plan_set_wait_limit(plan: Plan, sm_clocks: int):
+    rc = lib().nsp_plan_set_wait_limit(plan.handle, int(sm_clocks))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_plan_set_wait_limit")
+
+
+def nsp_checked_withhold_load(plan: Plan, enable: bool):
+    """Checked build only: the next forward launch leaves out one V tile load (failure-detection test)."""
+    if not hasattr(lib(), "nsp_checked_withhold_load"):
+        raise NspError(NSP_ERR_UNSUPPORTED, "nsp_checked_withhold_load (needs libnsp_checked.so)")
+    rc = lib().nsp_checked_withhold_load(plan.handle, int(bool(enable)))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_checked_withhold_load")
 
 
 def nsp_device_status(plan: Plan):

@@ -16,6 +16,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libnsp.so"
+LIB_CHECKED = PKG / "libnsp_checked.so"  # the same sources with -DNSP_CHECKED: index checks inside the kernels
 OBJ_DIR = PKG / "build"
 
 NVCC_FLAGS = [
@@ -41,18 +42,20 @@ def _stale(target: Path, deps) -> bool:
     return any(Path(d).stat().st_mtime > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> Path:
+def build_library(force: bool = False, verbose: bool = False, checked: bool = False) -> Path:
+    """Build libnsp.so, or with checked=True libnsp_checked.so (kernels verify every index they compute; for tests)."""
     nvcc = _nvcc()
+    lib, tag, extra = (LIB_CHECKED, "_checked", ["-DNSP_CHECKED"]) if checked else (LIB, "", [])
     sources = sorted(CSRC.glob("*.cu"))
     headers = sorted(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "nsp.h"]
     OBJ_DIR.mkdir(exist_ok=True)
 
     def compile_one(src: Path):
-        obj = OBJ_DIR / (src.stem + ".o")
+        obj = OBJ_DIR / (src.stem + tag + ".o")
         if force or _stale(obj, [src, *headers]):
-            cmd = [nvcc, *NVCC_FLAGS, "-c", str(src), "-o", str(obj)]
+            cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", str(src), "-o", str(obj)]
             r = subprocess.run(cmd, capture_output=True, text=True)
-            (OBJ_DIR / (src.stem + ".ptxas.log")).write_text(r.stderr)
+            (OBJ_DIR / (src.stem + tag + ".ptxas.log")).write_text(r.stderr)
             if r.returncode != 0:
                 raise RuntimeError(f"nvcc failed for {src.name}:\n{r.stdout}\n{r.stderr}")
             if verbose:
@@ -61,16 +64,17 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
 
     with ThreadPoolExecutor(max_workers=min(8, len(sources))) as ex:
         objs = list(ex.map(compile_one, sources))
-    if force or _stale(LIB, objs):
-        tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
+    if force or _stale(lib, objs):
+        tmp = lib.with_suffix(f".tmp{os.getpid()}.so")
         cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-cudart", "static",
                *map(str, objs), "-o", str(tmp)]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
     print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, checked=True))

@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -40,6 +41,8 @@ struct nsp_plan {
   int32_t* h_status = nullptr;    // the same record in mapped pinned host memory (written by the failing kernel)
   int32_t* h_status_dev = nullptr;  // device pointer to h_status
   int sticky = 0;
+  long long wait_limit = NSP_WAIT_CYCLES_DEFAULT;  // SM clocks a device-side wait may take
+  int withhold = 0;                                // checked build: failure-detection test switch
   // optional per-kernel timing (CUDA events on the launching stream)
   bool profiling = false;
   cudaEvent_t ev[2 * NSP_KERNEL_COUNT] = {};
@@ -127,6 +130,23 @@ int plan_failed(const nsp_plan* plan) {
   return plan->sticky;
 }
 StatusWord status_word(const nsp_plan* plan) { return StatusWord{plan->d_status, plan->h_status_dev}; }
+
+// Host-side call log: with NSP_LOG=1 in the environment (read once) every plan construction and every compute call
+// prints one line to stderr. Nothing on the device changes.
+bool log_on() {
+  static const bool on = [] {
+    const char* e = std::getenv("NSP_LOG");
+    return e && e[0] && e[0] != '0';
+  }();
+  return on;
+}
+#define NSP_LOGF(...)                        \
+  do {                                       \
+    if (log_on()) {                          \
+      std::fprintf(stderr, "[nsp] " __VA_ARGS__); \
+      std::fputc('\n', stderr);              \
+    }                                        \
+  } while (0)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -359,6 +379,10 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     free_plan(p);
     return rc;
   }
+  NSP_LOGF("plan %p: %d segments, %zu runs, head_dim %d, q_elems %lld, kv_elems %lld, fwd items %lld, bwd items %lld%s",
+           static_cast<void*>(p), n_seg, p->runs.size(), head_dim, static_cast<long long>(p->q_elems),
+           static_cast<long long>(p->kv_elems), static_cast<long long>(nf), static_cast<long long>(nb),
+           p->deterministic ? ", deterministic dQ" : "");
   *out_plan = p;
   return NSP_OK;
 }
@@ -420,9 +444,14 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  a.wait_limit = plan->wait_limit;
+  a.withhold = plan->withhold;
+  a.q_elems = plan->q_elems;
+  a.lse_elems = plan->lse_elems;
   a.seg_mask = nullptr;
   a.d_o = nullptr;
   a.delta = nullptr;
+  NSP_LOGF("fwd plan %p stream %p scale %g", static_cast<const void*>(plan), stream, softmax_scale);
   prof_mark(plan, NSP_KERNEL_FWD, 0, st);
   if (launch_fwd(maps, a, plan->head_dim, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_FWD, 1, st);
@@ -498,6 +527,10 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
     fa.o = nullptr;
     fa.lse = lse_ws;
     fa.scale_log2 = softmax_scale * 1.4426950408889634f;
+    fa.wait_limit = plan->wait_limit;
+    fa.withhold = 0;
+    fa.q_elems = plan->q_elems;
+    fa.lse_elems = plan->lse_elems;
     fa.seg_mask = d_mask;
     fa.d_o = static_cast<const __nv_bfloat16*>(d_o);
     fa.delta = delta;
@@ -508,6 +541,8 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   // Segments of at most 128 tokens are finished by the first-tile kernel alone; a batch made only of such segments
   // needs no accumulator, no delta and no conversion pass.
   const bool multi = plan->max_len > kBM;
+  NSP_LOGF("bwd plan %p stream %p scale %g%s%s", static_cast<const void*>(plan), stream, softmax_scale,
+           recompute ? ", recomputing marked segments" : "", multi ? "" : ", first-tile kernel only");
   if (dq_turn && multi &&
       cudaMemsetAsync(dq_turn, 0, static_cast<size_t>(plan->n_fwd) * 4, st) != cudaSuccess)
     return NSP_ERR_CUDA;
@@ -535,6 +570,10 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   a.dkv_f32 = dkv_dtype == NSP_F32;
   a.scale = softmax_scale;
   a.scale_log2 = softmax_scale * 1.4426950408889634f;
+  a.wait_limit = plan->wait_limit;
+  a.q_elems = plan->q_elems;
+  a.kv_elems = plan->kv_elems;
+  a.lse_elems = plan->lse_elems;
   // first-tile kernel: q tile 0 of every segment (its dQ rows; its part of, or all of, dK / dV rows 0..127)
   a.items = plan->d_bwd_first;
   a.n_items = static_cast<int32_t>(plan->n_first);
@@ -643,6 +682,20 @@ int nsp_device_status(const nsp_plan_t* plan, int32_t out[4]) {
   if (out[0] != 0 && !plan->sticky) const_cast<nsp_plan_t*>(plan)->sticky = out[0];
   return NSP_OK;
 }
+
+int nsp_plan_set_wait_limit(nsp_plan_t* plan, int64_t sm_clocks) {
+  if (!plan || sm_clocks < 1000) return NSP_ERR_INVALID_ARG;
+  plan->wait_limit = sm_clocks;
+  return NSP_OK;
+}
+
+#ifdef NSP_CHECKED
+int nsp_checked_withhold_load(nsp_plan_t* plan, int enable) {
+  if (!plan) return NSP_ERR_INVALID_ARG;
+  plan->withhold = enable != 0;
+  return NSP_OK;
+}
+#endif
 
 int nsp_plan_set_profiling(nsp_plan_t* plan, int enable) {
   if (!plan) return NSP_ERR_INVALID_ARG;

@@ -271,6 +271,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       }
     }
     tc_fence_before_sync();
+    // Every role gets here in bounded time: all its other waits are bounded, and none of them returns before the end
+    // of the kernel. (An mbarrier with a bounded wait in this place made the register allocation of the softmax role
+    // fail.)
     __syncthreads();
     tc_fence_after_sync();
     cx = &x;
@@ -309,7 +312,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             int h, m;
             w.get(c, h, m);
             w.next(c);
-            if (!mbar_wait(&s.bar_q_empty[qr.st][0], qr.ph ^ 1) || !mbar_wait(&s.bar_q_empty[qr.st][1], qr.ph ^ 1)) {
+            if (!mbar_wait(&s.bar_q_empty[qr.st][0], qr.ph ^ 1, a.wait_limit) || !mbar_wait(&s.bar_q_empty[qr.st][1], qr.ph ^ 1, a.wait_limit)) {
               report_timeout(a.status, c.it, kWhereBwdQEmpty, vt);
               *abort_flag = 1;
               break;
@@ -319,7 +322,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             for (int hf = 0; hf < kHalves; ++hf)
               tma_load_3d(s.q[qr.st][hf], mq, &s.bar_q_full[qr.st], 64 * hf, h, c.tok0 + m * kBM);
             qr.next();
-            if (!mbar_wait(&s.bar_do_empty[0], (cs & 1) ^ 1) || !mbar_wait(&s.bar_do_empty[1], (cs & 1) ^ 1)) {
+            if (!mbar_wait(&s.bar_do_empty[0], (cs & 1) ^ 1, a.wait_limit) || !mbar_wait(&s.bar_do_empty[1], (cs & 1) ^ 1, a.wait_limit)) {
               report_timeout(a.status, c.it, kWhereBwdQEmpty, 100000 + vt);
               *abort_flag = 1;
               break;
@@ -359,14 +362,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           constexpr uint32_t kStageStep = kOpBytes >> 4;  // descriptor distance between Q stages
           const int steps = cx->steps, item_it = cx->it;
           int where = 0;
-          bool okm = mbar_wait(&s.bar_kv, gi & 1);
+          bool okm = mbar_wait(&s.bar_kv, gi & 1, a.wait_limit);
           if (!okm) where = kWhereBwdLoadKV;
           const uint32_t q0_lo = smem_desc_addr(s.q[0][0]), do_lo = smem_desc_addr(s.d_o[0]);
           if (is_a) {
             const uint32_t k_km = smem_desc_addr(s.k[0]) | lbo_km;
             // S^T of the next step not yet issued -> R0 (A = K, B = Q of the ring stage, both K-major)
             auto issue_s = [&]() -> bool {
-              if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph)) { where = kWhereBwdLoadQ; return false; }
+              if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph, a.wait_limit)) { where = kWhereBwdLoadQ; return false; }
               tc_fence_after_sync();
               const uint32_t b_lo = (q0_lo + qr.st * kStageStep) | lbo_km;
 #pragma unroll
@@ -384,8 +387,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               constexpr bool fold = FIRST;
               const uint32_t cs = gs + vt;
               if (*abort_flag) return false;
-              if (!mbar_wait(&s.bar_do_full, cs & 1)) { where = kWhereBwdLoadQ; return false; }
-              if (!mbar_wait(&s.bar_p_ready, cs & 1)) { where = kWhereBwdPReady; return false; }
+              if (!mbar_wait(&s.bar_do_full, cs & 1, a.wait_limit)) { where = kWhereBwdLoadQ; return false; }
+              if (!mbar_wait(&s.bar_p_ready, cs & 1, a.wait_limit)) { where = kWhereBwdPReady; return false; }
               tc_fence_after_sync();
               const uint32_t acc = vt > 0;
               if constexpr (!fold) {
@@ -406,7 +409,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               if (leader) umma_commit(&s.bar_do_empty[0]);  // this thread is done with the dO buffer
               if constexpr (fold) {
                 // the softmax warps read P^T back from R0 while they form dS^T: S^T of the next step waits for them
-                if (!mbar_wait(&s.bar_ds_ready, cs & 1)) { where = kWhereBwdDsReady; return false; }
+                if (!mbar_wait(&s.bar_ds_ready, cs & 1, a.wait_limit)) { where = kWhereBwdDsReady; return false; }
               }
               if (vt + 1 < steps && !issue_s()) return false;
               return true;
@@ -420,8 +423,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             // dP^T of step vt -> R1, once the dQ warps have drained dQ^T of the previous step from it
             auto issue_dp = [&](int vt) -> bool {
               const uint32_t cs = gs + vt;
-              if (!mbar_wait(&s.bar_do_full, cs & 1)) { where = kWhereBwdLoadQ; return false; }
-              if (!mbar_wait(&s.bar_dq_empty, (cs & 1) ^ 1)) { where = kWhereBwdDqEmpty; return false; }
+              if (!mbar_wait(&s.bar_do_full, cs & 1, a.wait_limit)) { where = kWhereBwdLoadQ; return false; }
+              if (!mbar_wait(&s.bar_dq_empty, (cs & 1) ^ 1, a.wait_limit)) { where = kWhereBwdDqEmpty; return false; }
               tc_fence_after_sync();
 #pragma unroll
               for (int kk = 0; kk < D / 16; ++kk) {
@@ -437,8 +440,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               constexpr bool fold = FIRST;
               const uint32_t cs = gs + vt;
               if (*abort_flag) return false;
-              if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph)) { where = kWhereBwdLoadQ; return false; }
-              if (!mbar_wait(&s.bar_ds_ready, cs & 1)) { where = kWhereBwdDsReady; return false; }
+              if (!mbar_wait(&s.bar_q_full[qr.st], qr.ph, a.wait_limit)) { where = kWhereBwdLoadQ; return false; }
+              if (!mbar_wait(&s.bar_ds_ready, cs & 1, a.wait_limit)) { where = kWhereBwdDsReady; return false; }
               tc_fence_after_sync();
               const uint32_t acc = vt > 0;
               const uint32_t q_mn = (q0_lo + qr.st * kStageStep) | lbo_mn;
@@ -491,7 +494,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         for (int vt = 0; vt < c.steps; ++vt) {
           const uint32_t cs = gs + vt, st = cs & 1;
           if (*abort_flag) break;
-          bool okl = mbar_wait(&s.bar_ld_empty[st], ((cs >> 1) & 1) ^ 1);
+          bool okl = mbar_wait(&s.bar_ld_empty[st], ((cs >> 1) & 1) ^ 1, a.wait_limit);
           okl = __all_sync(0xffffffffu, okl);
           if (!okl) {
             if (lane == 0) {
@@ -508,8 +511,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           for (int x = 0; x < 4; ++x) {
             const int col = lane + 32 * x, qi = m * kBM + col;
             const bool valid = qi < c.len;
-            s.lse[st][col] = valid ? a.lse[base + qi] * kLog2e : INFINITY;
-            s.delta[st][col] = valid ? a.delta[base + qi] : 0.f;
+            float lv = INFINITY, dv_ = 0.f;
+            if (valid) {
+              NSP_CHECK(base + qi >= 0 && base + qi < a.lse_elems, a.status, c.it, kWhereCheckBwdLse, qi) {
+                lv = a.lse[base + qi] * kLog2e;
+                dv_ = a.delta[base + qi];
+              }
+            }
+            s.lse[st][col] = lv;
+            s.delta[st][col] = dv_;
           }
           mbar_arrive(&s.bar_ld_full[st]);
         }
@@ -531,7 +541,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       for (int vt = 0; vt < c.steps; ++vt) {
         const uint32_t cs = gs + vt;
         if (*abort_flag) break;
-        bool okr = mbar_wait(&s.bar_dq_full, cs & 1);
+        bool okr = mbar_wait(&s.bar_dq_full, cs & 1, a.wait_limit);
         okr = __all_sync(0xffffffffu, okr);
         if (!okr) {
           if (lane == 0) {
@@ -561,7 +571,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               int32_t* turn = a.dq_turn + c.turn_off + h * c.mt + m;
               if (lane == 0) {
                 const long long t0 = clock64();
-                while (*reinterpret_cast<volatile int32_t*>(turn) < 8 * c.n && clock64() - t0 < NSP_WAIT_CYCLES) __nanosleep(64);
+                while (*reinterpret_cast<volatile int32_t*>(turn) < 8 * c.n && clock64() - t0 < a.wait_limit) __nanosleep(64);
                 atomicAdd(turn, 1);
               }
             }
@@ -577,6 +587,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           tc_fence_before_sync();
           mbar_arrive(&s.bar_dq_empty);
           const int64_t o0 = c.q_off + (static_cast<int64_t>(colhalf * 64) * c.hq + h) * kHeadDim + d;
+          NSP_CHECK(n_valid <= 0 || (o0 >= 0 && o0 + (min(n_valid, 64) - 1) * q_stride < a.q_elems), a.status, c.it,
+                    kWhereCheckBwdDq, h) {
           if (a.dq_f32) {
             float* q0 = static_cast<float*>(a.dq) + o0;
 #pragma unroll
@@ -592,6 +604,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               if (e + 32 < n_valid) q0[(e + 32) * q_stride] = __float2bfloat16_rn(__uint_as_float(v1[e]) * a.scale);
             }
           }
+          }
           continue;
         }
         float* p0 = tile0 + colhalf * 64 * q_stride;
@@ -602,7 +615,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           if (lane == 0) {
             const long long t0 = clock64();
             while (*reinterpret_cast<volatile int32_t*>(turn) < 8 * c.n) {
-              if (clock64() - t0 > NSP_WAIT_CYCLES) { okt = false; break; }
+              if (clock64() - t0 > a.wait_limit) { okt = false; break; }
               __nanosleep(64);
             }
             __threadfence();
@@ -633,6 +646,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           // The reductions sit in a conditional region on purpose (the condition always holds): as straight-line
           // code the compiler computes all 64 row addresses ahead of the TMEM loads, runs out of the 80 registers
           // this role has and spills inside the loop (measured: the whole kernel 25 % slower).
+          NSP_CHECK(p0 >= a.dq_acc && p0 + 63 * q_stride < a.dq_acc + a.q_elems, a.status, c.it, kWhereCheckBwdDq, m)
           if (c.hq > 0) {
             float* p1 = p0 + 32 * q_stride;
 #pragma unroll
@@ -661,7 +675,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             }
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              if (c.hq > 0 && ch * 16 + e < n_valid) red_add_f32(p0, __uint_as_float(v[e]));
+              if (c.hq > 0 && ch * 16 + e < n_valid) {
+                NSP_CHECK(p0 >= a.dq_acc && p0 < a.dq_acc + a.q_elems, a.status, c.it, kWhereCheckBwdDq, m)
+                red_add_f32(p0, __uint_as_float(v[e]));
+              }
               p0 += q_stride;
             }
           }
@@ -701,7 +718,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         int h, m;
         w.get(c, h, m);
         w.next(c);
-        oks = mbar_wait(&s.bar_ld_full[st], (cs >> 1) & 1) && mbar_wait(&s.bar_s_full, cs & 1);
+        oks = mbar_wait(&s.bar_ld_full[st], (cs >> 1) & 1, a.wait_limit) && mbar_wait(&s.bar_s_full, cs & 1, a.wait_limit);
         oks = __all_sync(0xffffffffu, oks);
         if (!oks) { where = kWhereBwdS; break; }
         tc_fence_after_sync();
@@ -763,7 +780,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           // previous step, so bar_dp_full implies they have completed.
 #pragma unroll
           for (int i = 0; i < 4; ++i) aux[0][i] = lds128(delta_s + 4 * i);
-          oks = mbar_wait(&s.bar_dp_full, cs & 1);
+          oks = mbar_wait(&s.bar_dp_full, cs & 1, a.wait_limit);
           oks = __all_sync(0xffffffffu, oks);
           if (!oks) { where = kWhereBwdDp; return false; }
           tc_fence_after_sync();
@@ -809,7 +826,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           // would push dK / dV past the tolerance: P^T and dS^T enter their products as bf16 value plus bf16 residual
           // (two products each, the residuals next to the values), and delta_i = sum_j P_ij dP_ij is taken here in
           // fp32 (all keys of these rows sit in this tile) instead of from the bf16-rounded O.
-          oks = mbar_wait(&s.bar_dp_full, cs & 1);
+          oks = mbar_wait(&s.bar_dp_full, cs & 1, a.wait_limit);
           oks = __all_sync(0xffffffffu, oks);
           if (!oks) { where = kWhereBwdDp; break; }
           tc_fence_after_sync();
@@ -863,13 +880,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             tc_fence_before_sync();
             mbar_arrive(&s.bar_p_ready);  // the dV products run under the rest of this step
             mbar_arrive(&s.bar_delta[half]);
-            oks = mbar_wait(&s.bar_delta[half], nd & 1);
+            oks = mbar_wait(&s.bar_delta[half], nd & 1, a.wait_limit);
             ++nd;
             oks = __all_sync(0xffffffffu, oks);
             if (!oks) { where = kWhereBwdDelta; break; }
             if (r < 64) delta_s[r] = (part[r] + part[64 + r]) + (part[128 + r] + part[192 + r]);
             mbar_arrive(&s.bar_delta[half]);
-            oks = mbar_wait(&s.bar_delta[half], nd & 1);
+            oks = mbar_wait(&s.bar_delta[half], nd & 1, a.wait_limit);
             ++nd;
             oks = __all_sync(0xffffffffu, oks);
             if (!oks) { where = kWhereBwdDelta; break; }
@@ -912,7 +929,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       }
       // ---- epilogue: wait for the last MMAs of the item, then write dK (scaled) and dV of this key tile
       if (oks) {
-        oks = mbar_wait(&s.bar_b_done, (gs + c.steps - 1) & 1) && mbar_wait(&s.bar_a_done, (gs + c.steps - 1) & 1);
+        oks = mbar_wait(&s.bar_b_done, (gs + c.steps - 1) & 1, a.wait_limit) && mbar_wait(&s.bar_a_done, (gs + c.steps - 1) & 1, a.wait_limit);
         oks = __all_sync(0xffffffffu, oks);
         if (!oks) where = kWhereBwdDqFull;
       }
@@ -933,6 +950,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           // Key tile 0 in the main kernel: the first-tile kernel, which ran before, left its part (q tile 0) in the
           // output; this item's sum over the q tiles 1 .. Mt-1 is added to it (one fixed order: reproducible).
           const bool add = !FIRST && c.first;
+          NSP_CHECK(!valid || (off >= 0 && off + kCols <= a.kv_elems), a.status, c.it, kWhereCheckBwdDkv, kj)
           if (valid) {
             if (a.dkv_f32) {
               float* o = static_cast<float*>(outp) + off + cc * 32;

@@ -117,6 +117,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   const uint32_t tmem = s.tmem_base;
   volatile int32_t* abort_flag = &s.abort;
   uint32_t gp = 0;  // pops so far
+  // The CTA-wide meeting points are plain barriers. Every role reaches them in bounded time: all its other waits are
+  // bounded and none of them returns before the end of the kernel. (An mbarrier with a bounded wait in their place
+  // made the register allocation of the softmax role fail.)
+  auto cta_sync = [&]() {
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+  };
 
   // ---- work decoding shared by all roles (every role runs its own copy of the loops, see the backward kernel)
   FwdRound rd;
@@ -151,9 +159,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   };
   auto next_pop = [&]() -> bool {
     if (tid == 0 && !fetched_ahead) fetch_pop(s.pop[gp & 1]);
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
+    cta_sync();
     pp = &s.pop[gp & 1];
     it0 = pp->it0;
     ++gp;
@@ -168,11 +174,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     return true;
   };
   // end of a round: every warp has finished with the Q tiles, the K/V rings and the TMEM accumulators
-  auto round_end = [&]() {
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-  };
+  auto round_end = [&]() { cta_sync(); };
 
   if (wg == 4) {
     fwd_setmaxnreg_dec<kFwdRegsAux>();
@@ -199,7 +201,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             for (int j = 0; j < n_kv; ++j) {
               if (*abort_flag) break;
               uint32_t st = kn & 1;
-              if (!mbar_wait(&s.bar_k_empty[st], ((kn >> 1) & 1) ^ 1)) {
+              if (!mbar_wait(&s.bar_k_empty[st], ((kn >> 1) & 1) ^ 1, a.wait_limit)) {
                 report_timeout(a.status, it0, kWhereFwdLoad, j);
                 *abort_flag = 1;
                 break;
@@ -209,11 +211,17 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.k[st][hf], mk, &s.bar_k_full[st], 64 * hf, g, tok0 + j * kBN);
               ++kn;
               st = vn & 1;
-              if (!mbar_wait(&s.bar_v_empty[st], ((vn >> 1) & 1) ^ 1)) {
+              if (!mbar_wait(&s.bar_v_empty[st], ((vn >> 1) & 1) ^ 1, a.wait_limit)) {
                 report_timeout(a.status, it0, kWhereFwdLoad, 100000 + j);
                 *abort_flag = 1;
                 break;
               }
+#ifdef NSP_CHECKED
+              if (a.withhold && vn == 0) {  // failure-detection test: this V tile never arrives
+                ++vn;
+                continue;
+              }
+#endif
               mbar_expect_tx(&s.bar_v_full[st], kTileBytes);
 #pragma unroll
               for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.v[st][hf], mv, &s.bar_v_full[st], 64 * hf, g, tok0 + j * kBN);
@@ -264,7 +272,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                            (j > 0 || kk > 0));
               if (leader) umma_commit(&s.bar_pv_done[x]);
             };
-            bool ok = mbar_wait(&s.bar_q, qn & 1);
+            bool ok = mbar_wait(&s.bar_q, qn & 1, a.wait_limit);
             ++qn;
             if (!ok) where = kWhereFwdLoad;
             uint32_t kst = 0;
@@ -272,7 +280,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               if (*abort_flag) break;
               if (j == 0) {
                 kst = kn & 1;
-                if (!mbar_wait(&s.bar_k_full[kst], (kn >> 1) & 1)) { ok = false; where = kWhereFwdLoad; break; }
+                if (!mbar_wait(&s.bar_k_full[kst], (kn >> 1) & 1, a.wait_limit)) { ok = false; where = kWhereFwdLoad; break; }
                 tc_fence_after_sync();
                 issue_s(0, kst);
                 if (joint) issue_s(1, kst);
@@ -281,19 +289,19 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               }
               const uint32_t vst = vn & 1;
               const bool more = j + 1 < n_kv;
-              if (!mbar_wait(&s.bar_p_ready[0], pn[0] & 1)) { ok = false; where = kWhereFwdS; break; }
+              if (!mbar_wait(&s.bar_p_ready[0], pn[0] & 1, a.wait_limit)) { ok = false; where = kWhereFwdS; break; }
               ++pn[0];
-              if (!mbar_wait(&s.bar_v_full[vst], (vn >> 1) & 1)) { ok = false; where = kWhereFwdLoad; break; }
+              if (!mbar_wait(&s.bar_v_full[vst], (vn >> 1) & 1, a.wait_limit)) { ok = false; where = kWhereFwdLoad; break; }
               tc_fence_after_sync();
               issue_pv(0, vst, j);
               if (more) {  // S_A of the next key tile runs while softmax B is still working
                 kst = kn & 1;
-                if (!mbar_wait(&s.bar_k_full[kst], (kn >> 1) & 1)) { ok = false; where = kWhereFwdLoad; break; }
+                if (!mbar_wait(&s.bar_k_full[kst], (kn >> 1) & 1, a.wait_limit)) { ok = false; where = kWhereFwdLoad; break; }
                 tc_fence_after_sync();
                 issue_s(0, kst);
               }
               if (joint) {
-                if (!mbar_wait(&s.bar_p_ready[1], pn[1] & 1)) { ok = false; where = kWhereFwdS; break; }
+                if (!mbar_wait(&s.bar_p_ready[1], pn[1] & 1, a.wait_limit)) { ok = false; where = kWhereFwdS; break; }
                 ++pn[1];
                 tc_fence_after_sync();
                 issue_pv(1, vst, j);
@@ -350,7 +358,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           int where = 0;
           for (int j = 0; j < n_kv; ++j) {
             if (*abort_flag) { ok = false; break; }
-            ok = mbar_wait(&s.bar_s_full[x], sn & 1);
+            ok = mbar_wait(&s.bar_s_full[x], sn & 1, a.wait_limit);
             ++sn;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { where = kWhereFwdS; break; }
@@ -384,13 +392,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                   mx = max3f(mx, __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
               my_slot[0] = mx;
               mbar_arrive(pair_bar);
-              ok = mbar_wait(pair_bar, xn & 1);
+              ok = mbar_wait(pair_bar, xn & 1, a.wait_limit);
               ++xn;
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) { where = kWhereFwdPair; break; }
               m_ref = fmaxf(mx, partner_slot[0]) * a.scale_log2;
             } else if (pending) {
-              ok = mbar_wait(pair_bar, xn & 1);
+              ok = mbar_wait(pair_bar, xn & 1, a.wait_limit);
               ++xn;
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) { where = kWhereFwdPair; break; }
@@ -427,7 +435,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             // maximum; the previous PV product of this half must have completed first (the next one is not
             // issued before p_ready).
             if (j > 0 && __any_sync(0xffffffffu, need)) {
-              ok = mbar_wait(&s.bar_pv_done[x], (pvn + j - 1) & 1);
+              ok = mbar_wait(&s.bar_pv_done[x], (pvn + j - 1) & 1, a.wait_limit);
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) { where = kWhereFwdO; break; }
               tc_fence_after_sync();
@@ -455,7 +463,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             }
           }
           if (ok) {
-            ok = mbar_wait(&s.bar_pv_done[x], (pvn + n_kv - 1) & 1);
+            ok = mbar_wait(&s.bar_pv_done[x], (pvn + n_kv - 1) & 1, a.wait_limit);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) where = kWhereFwdO;
           }
@@ -491,7 +499,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             my_slot[256] = l;
             my_slot[384] = part;
             mbar_arrive(pair_bar);
-            ok = mbar_wait(pair_bar, xn & 1);
+            ok = mbar_wait(pair_bar, xn & 1, a.wait_limit);
             ++xn;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) where = kWhereFwdPair;
@@ -499,8 +507,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               l += partner_slot[256];
               part += partner_slot[384];
               const int64_t at = sg.lse_off + static_cast<int64_t>(h) * sg.len + row;
-              a.lse[at] = (m_ref + log2f(l)) * 0.6931471805599453f;
-              a.delta[at] = part / l;
+              NSP_CHECK(at >= 0 && at < a.lse_elems, a.status, it0, kWhereCheckFwdLse, row) {
+                a.lse[at] = (m_ref + log2f(l)) * 0.6931471805599453f;
+                a.delta[at] = part / l;
+              }
             }
             if (!ok && lane == 0) {
               report_timeout(a.status, it0, where, 0);
@@ -512,7 +522,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           if (ok) {  // row sum = sum of the two half rows
             my_slot[256] = l;
             mbar_arrive(pair_bar);
-            ok = mbar_wait(pair_bar, xn & 1);
+            ok = mbar_wait(pair_bar, xn & 1, a.wait_limit);
             ++xn;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) where = kWhereFwdPair;
@@ -536,12 +546,16 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                   w.y = pack_bf16x2(__uint_as_float(orow[8 * e + 2]) * inv_l, __uint_as_float(orow[8 * e + 3]) * inv_l);
                   w.z = pack_bf16x2(__uint_as_float(orow[8 * e + 4]) * inv_l, __uint_as_float(orow[8 * e + 5]) * inv_l);
                   w.w = pack_bf16x2(__uint_as_float(orow[8 * e + 6]) * inv_l, __uint_as_float(orow[8 * e + 7]) * inv_l);
+                  NSP_CHECK(optr + c * 32 + e * 8 + 8 <= a.o + a.q_elems && optr >= a.o, a.status, it0, kWhereCheckFwdO, row)
                   *reinterpret_cast<uint4*>(optr + c * 32 + e * 8) = w;
                 }
               }
             }
-            if (valid && ch == 0)
-              a.lse[sg.lse_off + static_cast<int64_t>(h) * sg.len + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
+            if (valid && ch == 0) {
+              const int64_t at = sg.lse_off + static_cast<int64_t>(h) * sg.len + row;
+              NSP_CHECK(at >= 0 && at < a.lse_elems, a.status, it0, kWhereCheckFwdLse, row)
+              a.lse[at] = (m_ref + log2f(l)) * 0.6931471805599453f;
+            }
           } else if (where != 0 && lane == 0) {
             report_timeout(a.status, it0, where, 0);
             *abort_flag = 1;
@@ -552,8 +566,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     }
   }
 
-  tc_fence_before_sync();
-  __syncthreads();
+  cta_sync();  // after a timeout the stragglers are not waited for for ever
   if (warp == 0) tmem_dealloc(s.tmem_base, kFwdTmemCols);
 }
 

@@ -73,6 +73,11 @@ enum DeviceWhere : int32_t {
   kWhereBwdItemBarrier = 25,
   kWhereBwdTmemBase = 26,
   kWhereBwdTurn = 27,  // deterministic dQ: the key tiles before this one did not finish their additions
+  kWhereCheckFwdO = 40,    // checked build: an index outside the tensor (O, LSE / delta, dQ, dK / dV, LSE read)
+  kWhereCheckFwdLse = 41,
+  kWhereCheckBwdDq = 42,
+  kWhereCheckBwdDkv = 43,
+  kWhereCheckBwdLse = 44,
   kWhereSelfTest = 90,
 };
 
@@ -99,6 +104,17 @@ __device__ __forceinline__ void report_timeout(StatusWord st, int32_t item, int3
   report_status_raw(st.dev, st.host, NSP_ERR_DEVICE_TIMEOUT, item, where, aux);
 }
 
+// Index checks of the checked build (-DNSP_CHECKED, libnsp_checked.so): `NSP_CHECK(cond, ...) access;` performs the
+// access only if cond holds and otherwise records NSP_ERR_DEVICE_ASSERT; in the regular build it is the bare access.
+#ifdef NSP_CHECKED
+#define NSP_CHECK(cond, st, item, where, aux)                                       \
+  if (!(cond)) {                                                                    \
+    report_status(st, NSP_ERR_DEVICE_ASSERT, item, where, static_cast<int32_t>(aux)); \
+  } else
+#else
+#define NSP_CHECK(cond, st, item, where, aux)
+#endif
+
 struct FwdArgs {
   const SegInfo* seg;
   const nsp_tile_t* items;
@@ -108,6 +124,9 @@ struct FwdArgs {
   __nv_bfloat16* o;
   float* lse;
   float scale_log2;  // softmax_scale * log2(e)
+  long long wait_limit;  // SM clocks a device-side wait may take before it gives up
+  int32_t withhold;      // checked build only: 1 = the producer leaves out one V load (failure-detection test)
+  int64_t q_elems, lse_elems;  // tensor sizes (checked build)
   // Recomputation inside the backward pass (all three null in a plain forward): only items of segments with
   // seg_mask[seg] != 0 run, and instead of O the kernel writes delta = rowsum(dO o O) next to the LSE.
   const uint8_t* seg_mask;
@@ -132,6 +151,8 @@ struct BwdArgs {
   int32_t dkv_f32;
   float scale;
   float scale_log2;
+  long long wait_limit;  // SM clocks a device-side wait may take before it gives up
+  int64_t q_elems, kv_elems, lse_elems;  // tensor sizes (checked build)
   int32_t* front;    // [n_items / kFrontBlock + 1] arrival counters, zeroed before the launch (see next_item)
 };
 

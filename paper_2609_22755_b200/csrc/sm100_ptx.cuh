@@ -44,12 +44,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, ui
       : "memory");
   return ok != 0;
 }
-// Bounded wait: tests until the phase completes or about two seconds of SM clock have passed.
-// Returns false on expiry; the caller records it in the status word and unwinds.
-#ifndef NSP_WAIT_CYCLES
-#define NSP_WAIT_CYCLES 4000000000ll
-#endif
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit = NSP_WAIT_CYCLES) {
+// Bounded wait: tests until the phase completes or `limit` SM clocks have passed (the plan's wait limit; about two
+// seconds by default). Returns false on expiry; the caller records it in the status record and unwinds.
+#define NSP_WAIT_CYCLES_DEFAULT 4000000000ll
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit) {
   const long long t0 = clock64();
 #pragma unroll 1
   for (;;) {  // one test site only: the hot loops are instruction-cache sensitive
@@ -57,7 +55,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long l
     if (clock64() - t0 > limit) return false;
   }
 }
-
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -22,12 +22,22 @@ def B():
 
 def test_header_symbols_are_exported(B):
     header = (ROOT / "include" / "nsp.h").read_text()
+    # what the header declares only for the checked build belongs to libnsp_checked.so
+    checked_part = "".join(re.findall(r"#ifdef NSP_CHECKED(.*?)#endif", header, flags=re.S))
+    header = re.sub(r"#ifdef NSP_CHECKED.*?#endif", "", header, flags=re.S)
     declared = set(re.findall(r"\b(nsp_[a-z0-9_]+)\s*\(", header))
     assert {"nsp_plan_tiles", "nsp_attn_fwd", "nsp_attn_bwd"} <= declared
     lib = ctypes.CDLL(str(B.LIB_PATH))
     for name in sorted(declared):
         assert hasattr(lib, name), f"{name} is declared in include/nsp.h but not exported"
     assert declared == set(B.EXPORTS)
+    declared_checked = set(re.findall(r"\b(nsp_[a-z0-9_]+)\s*\(", checked_part))
+    assert declared_checked == set(B.CHECKED_EXPORTS)
+    checked = ctypes.CDLL(str(B.LIB_PATH.parent / "libnsp_checked.so"))
+    for name in sorted(declared | declared_checked):
+        assert hasattr(checked, name), f"{name} is missing from the checked build"
+    for name in declared_checked:
+        assert not hasattr(lib, name), f"{name} must not be in the regular library"
 
 
 def test_status_strings(B):
