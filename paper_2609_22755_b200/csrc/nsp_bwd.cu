@@ -407,10 +407,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               }
               if (leader) umma_commit(&s.bar_a_done);       // S^T and dV of the step
               if (leader) umma_commit(&s.bar_do_empty[0]);  // this thread is done with the dO buffer
-              if constexpr (fold) {
-                // the softmax warps read P^T back from R0 while they form dS^T: S^T of the next step waits for them
-                if (!mbar_wait(&s.bar_ds_ready, cs & 1, a.wait_limit)) { where = kWhereBwdDsReady; return false; }
-              }
               if (vt + 1 < steps && !issue_s()) return false;
               return true;
             };
@@ -830,17 +826,20 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           oks = __all_sync(0xffffffffu, oks);
           if (!oks) { where = kWhereBwdDp; break; }
           tc_fence_after_sync();
+          uint32_t pkk[4][16];
           {
             // Sweep 1: P^T (value and residual over the S^T columns just read: packed columns [16ch, 16ch + 8) and
-            // [16ch + 8, 16ch + 16)) and the partial sums of delta.
+            // [16ch + 8, 16ch + 16)) and the partial sums of delta. The packed values stay in registers for sweep 2
+            // (both sweeps fully unrolled), so R0 is free for the next S^T as soon as the dV products have run.
             float* part = reinterpret_cast<float*>(s.ds[half]);  // [4 quadrants][64 columns]; free until dS is written
             // Column sums over the 32 key rows of a warp by a butterfly: at every level a lane keeps the half of
             // the columns its lane bit selects and adds the partner's partial sums of that half (16 shuffles for
             // 16 columns); after the last level lane 2c (and 2c + 1) holds column c = lane / 2.
             const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4, b1 = lane & 2;
-#pragma unroll 1
+#pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
-              uint32_t sv[16], dpv[16], pk[16];
+              uint32_t sv[16], dpv[16];
+              uint32_t* const pk = pkk[ch];
               float4 l4[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) l4[i] = lds128(lse_s + ch * 16 + 4 * i);
@@ -891,16 +890,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             oks = __all_sync(0xffffffffu, oks);
             if (!oks) { where = kWhereBwdDelta; break; }
           }
-          // Sweep 2: dS^T = P^T o (dP^T - delta), value and residual; P^T (value + residual = P to 2^-17) is read back
-          // from R0, which the next S^T does not overwrite before bar_ds_ready.
+          // Sweep 2: dS^T = P^T o (dP^T - delta), value and residual (P = value + residual to 2^-17)
           uint8_t* const ds_row_lo = ds_row + 2 * kHalfTileBytes;
-#pragma unroll 1
+#pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
-            uint32_t pk[16], dpv[16], dsp[8], dsl[8];
+            uint32_t dpv[16], dsp[8], dsl[8];
+            const uint32_t* const pk = pkk[ch];
             float4 e4[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) e4[i] = lds128(delta_s + ch * 16 + 4 * i);
-            tmem_ld16(tS + ch * 16, pk);
             tmem_ld16(tDP + ch * 16, dpv);
             tmem_wait_ld();
 #pragma unroll
