@@ -249,6 +249,8 @@ def rank_workload(config: int, uniform: int, rank: int):
         return W.custom([uniform] * n, 32, 4, seed=1000 * rank, name=f"uniform_{n}x{uniform}_32q4kv")
     if config == 0:
         return W.profile_case()
+    if config == 7:
+        return W.profile_case_large_head()
     return W.config(config, seed=(config - 1) + 1000 * rank)
 
 
@@ -277,7 +279,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4,
                     help="benchmark configuration 1..5 (default 4: the nested-plan shard); 6 = the mixed-degree "
-                         "full-tree shard; 0 = the scaled-down nested case used for profiler captures")
+                         "full-tree shard; 0 and 7 = the scaled-down nested and large-head cases used for profiler captures")
     ap.add_argument("--uniform", type=int, default=0, metavar="L",
                     help="instead of --config: 131,072 tokens at 32q/4kv in segments of L tokens each (short-segment "
                          "studies; not a bench value)")
@@ -355,14 +357,21 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
-    for _ in range(args.steps):
+    # Per-kernel device times come from CUDA events the library records around each of its kernels on the launching
+    # stream. Reading them waits for the step, which is free when a step takes hundreds of milliseconds; short steps
+    # (the other configurations) are interrupted as little as possible: there only the first and the last step of the
+    # timed region are read.
+    read_every = False
+    for i in range(args.steps):
         eng.step_device()
-        # per-kernel device times of this step (CUDA events recorded by the library on the launching stream)
-        k_fwd.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_FWD))
-        k_pre.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_PRE))
-        k_bwd.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_MAIN))
-        k_post.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_POST))
-        k_first.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_FIRST))
+        if i == 0 or i == args.steps - 1 or read_every:
+            k_fwd.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_FWD))
+            k_pre.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_PRE))
+            k_bwd.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_MAIN))
+            k_post.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_POST))
+            k_first.append(B.nsp_plan_kernel_ms(eng.plan, B.KERNEL_BWD_FIRST))
+            if i == 0:
+                read_every = k_fwd[0] + k_bwd[0] > 50.0
     e1.record()
     barrier()
     launches = B.launch_count() - launches0

@@ -162,10 +162,10 @@ def plan_tiles(cu, hq, hkv, bm=128, bn=128, pass_=0):
 
 
 def recompute_mark(lengths, hq, level, budget_bytes, head_dim=128):
-    """Save / recompute marking of one GPU's segments (paper Sec. 4.2.2 "Tree-Level Recomputation"): walk the tree
-    from the upper levels toward the leaves, add up the bytes of the attention-output slices that are saved, and
-    once the budget is reached mark everything that is left for recomputation; inside the level where the cut
-    falls, the samples that cost more to recompute are saved first.
+    """Save / recompute marking of one GPU's segments (paper Sec. 4.2.2 "Tree-Level Recomputation"). The segments are
+    visited level by level starting at the root; the bytes of attention output that saving a segment keeps alive are
+    added up; the first segment that would exceed the budget ends the walk, and it and everything after it is
+    recomputed. Inside a level the order is by recomputation cost, most expensive first.
 
     lengths, hq, level: one entry per segment (level: larger = closer to the root). A saved segment keeps its O
     slice (2 bytes per element) and its LSE (4 bytes per row) alive; its recomputation cost is hq * L(L+1)/2.

@@ -168,6 +168,15 @@ def profile_case(seed: int = 3) -> Workload:
                "one 65,536-token segment (4q/1kv) + degree-1 tail (32q/4kv) filling 8,192 tokens")
 
 
+def profile_case_large_head(seed: int = 4) -> Workload:
+    """The large-head shard at one eighth of its size, for profiler captures: one 16,384-token segment at degree 4
+    (16q/1kv) plus a degree-1 tail (64q/4kv) filling 16,384 tokens. About 1.9 GB on the device; the q tiles of the long
+    group (16 heads) still exceed L2, which is what makes this shape's backward pass DRAM-heavy."""
+    short = lognormal_lengths(seed, 16384, 4096, 1.0, 64, 65536)
+    return _mk("large_head_profile_case_16k", [16384] + short, [16] + [64] * len(short), [1] + [4] * len(short), seed,
+               "one 16,384-token segment (16q/1kv) + degree-1 tail (64q/4kv) filling 16,384 tokens")
+
+
 def ragged(seed: int = 11) -> Workload:
     """Lengths that are not multiples of 16 or of any tile, a 1-token and a zero-length segment, three runs."""
     lengths = [1, 17, 0, 127, 129, 255, 1000, 3, 384]
