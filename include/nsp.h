@@ -295,7 +295,8 @@ enum {
   NSP_KERNEL_BWD_MAIN = 2,
   NSP_KERNEL_BWD_POST = 3,
   NSP_KERNEL_BWD_FIRST = 4, /* the backward kernel for the first 128 tokens of every segment */
-  NSP_KERNEL_COUNT = 5
+  NSP_KERNEL_FWD_FIRST = 5, /* the forward kernel for the first 128 tokens of every segment */
+  NSP_KERNEL_COUNT = 6
 };
 
 /* Measurement aid (the paper's cost model is fed by offline profiles of the compute phase, Sec. 4.1.2): when

@@ -35,7 +35,7 @@ EXPORTS = [
 CHECKED_EXPORTS = ["nsp_checked_withhold_load"]  # libnsp_checked.so only
 NSP_COST_BUCKETS = 16
 NSP_STATIC_WS_BYTES = 32 * 1024 * 1024
-KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST, KERNEL_BWD_FIRST = 0, 1, 2, 3, 4
+KERNEL_FWD, KERNEL_BWD_PRE, KERNEL_BWD_MAIN, KERNEL_BWD_POST, KERNEL_BWD_FIRST, KERNEL_FWD_FIRST = 0, 1, 2, 3, 4, 5
 
 import os
 

@@ -33,6 +33,8 @@ struct nsp_plan {
   nsp_tile_t* d_bwd_exec = nullptr;  // the backward items in the order the kernel walks them (see build_bwd_exec_order)
   nsp_tile_t* d_bwd_first = nullptr;  // one item per (segment, kv head): the first-tile kernel's list
   int64_t n_first = 0;
+  int64_t n_fwd_main = 0;             // forward items that visit at least two key tiles: a prefix of d_fwd (the
+                                      // cost-1 tail = q tile 0 of every segment runs in the first-tile forward kernel)
   bool deterministic = false;         // plan option: dQ tiles added in key-tile order
   int32_t max_len = 0;                // longest segment: no preprocess / main / postprocess launch when <= 128
   int32_t* d_front = nullptr;        // [n_bwd / kFrontBlock + 1] start-alignment counters of the backward kernel
@@ -294,6 +296,9 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     for (const nsp_tile_t& t : bwd_exec)
       if (t.tile == 0) bwd_first.push_back(nsp_tile_t{t.seg, t.head, 0, p->seg[t.seg].hq / p->seg[t.seg].hkv});
     p->n_first = static_cast<int64_t>(bwd_first.size());
+    p->n_fwd_main = nf;
+    for (const SegInfo& sg : p->seg)
+      if (sg.len > 0) p->n_fwd_main -= sg.hq;
     for (const SegInfo& sg : p->seg) p->max_len = std::max(p->max_len, sg.len);
   } catch (...) {
     delete p;
@@ -327,7 +332,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
   A(reinterpret_cast<void**>(&p->d_bwd_exec), sizeof(nsp_tile_t) * nb);
   A(reinterpret_cast<void**>(&p->d_bwd_first), sizeof(nsp_tile_t) * p->n_first);
   A(reinterpret_cast<void**>(&p->d_front), sizeof(int32_t) * (nb / kFrontBlock + 1));
-  A(reinterpret_cast<void**>(&p->d_counters), 4 * sizeof(int32_t));  // [0] forward, [1] backward main, [2] first-tile
+  A(reinterpret_cast<void**>(&p->d_counters), 4 * sizeof(int32_t));  // [0] forward, [1] backward main, [2] first-tile backward, [3] first-tile forward
   A(reinterpret_cast<void**>(&p->d_status), 4 * sizeof(int32_t));
   if (okc) {
     void* hp = nullptr;
@@ -435,11 +440,9 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
       return NSP_ERR_CUDA;
   }
   if (cudaMemsetAsync(plan->d_counters, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
+  if (cudaMemsetAsync(plan->d_counters + 3, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
   FwdArgs a;
   a.seg = plan->d_seg;
-  a.items = plan->d_fwd;
-  a.n_items = static_cast<int32_t>(plan->n_fwd);
-  a.counter = plan->d_counters;
   a.status = status_word(plan);
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
@@ -452,6 +455,17 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.d_o = nullptr;
   a.delta = nullptr;
   NSP_LOGF("fwd plan %p stream %p scale %g", static_cast<const void*>(plan), stream, softmax_scale);
+  // q tile 0 of every segment (the cost-1 tail of the list): one item per (segment, kv head)
+  a.items = plan->d_bwd_first;
+  a.n_items = static_cast<int32_t>(plan->n_first);
+  a.counter = plan->d_counters + 3;
+  prof_mark(plan, NSP_KERNEL_FWD_FIRST, 0, st);
+  if (!plan->withhold && launch_fwd_first(maps, a, plan->head_dim, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
+  prof_mark(plan, NSP_KERNEL_FWD_FIRST, 1, st);
+  // everything else: the list's prefix (with the test switch of the checked build: the whole list, general kernel)
+  a.items = plan->d_fwd;
+  a.n_items = static_cast<int32_t>(plan->withhold ? plan->n_fwd : plan->n_fwd_main);
+  a.counter = plan->d_counters;
   prof_mark(plan, NSP_KERNEL_FWD, 0, st);
   if (launch_fwd(maps, a, plan->head_dim, plan->num_sms, st) != cudaSuccess) return NSP_ERR_CUDA;
   prof_mark(plan, NSP_KERNEL_FWD, 1, st);

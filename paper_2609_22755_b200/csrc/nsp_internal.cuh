@@ -163,6 +163,8 @@ cudaError_t launch_plan_build(const SegInfo* d_seg, int n_seg, int bm, int bn, n
                               cudaStream_t st);
 size_t plan_sort_tmp_bytes(int64_t max_items);
 cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int head_dim, int num_sms, cudaStream_t st);
+// q tile 0 of every segment: items (segment, kv head); args.items / n_items / counter are that list's
+cudaError_t launch_fwd_first(const FwdMaps& maps, const FwdArgs& args, int head_dim, int num_sms, cudaStream_t st);
 // The backward launches, in the order they run: preprocess (delta and zeroed accumulator rows for tokens 128.. of
 // every segment), first-tile kernel (q tile 0 of every segment: its dQ rows, and its part of dK / dV), main kernel,
 // postprocess (tokens 128..). seg_skip (may be null): segments whose delta is left alone; lse_in / lse_out (may be
