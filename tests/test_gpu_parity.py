@@ -193,6 +193,36 @@ def test_backward_with_recomputation(env, case, which):
             assert torch.equal(getattr(eng, name), getattr(run, name))
 
 
+def test_host_to_host_step_equals_the_device_step(env):
+    """The end-to-end call (pinned host tensors in and out, copies on a second stream under the kernels) returns what
+    the device-resident step leaves in the device buffers: O, LSE, dK, dV bit for bit, dQ (bf16, from the fp32
+    accumulator) within one rounding of the fp32 sum. Two steps in a row, to cover the reuse of the buffers."""
+    torch, W = env["torch"], env["W"]
+    from paper_2609_22755_b200.api import NspAttention
+
+    w = W.custom([1536, 700, 300, 129, 64], [4, 4, 8, 2, 2], [1, 1, 2, 2, 1], seed=13, name="host_step")
+    host = {k: v.pin_memory() for k, v in W.make_tensors(w).items()}
+    eng = NspAttention(w)
+    eng.load(host)
+    eng.step_device()
+    torch.cuda.synchronize()
+    want = {n: getattr(eng, n).cpu() for n in ("o", "lse", "dq", "dk", "dv")}
+    for n in ("q", "k", "v", "do", "o", "lse", "dq", "dk", "dv"):
+        getattr(eng, n).zero_()
+    out = eng.alloc_host_outputs()
+    for _ in range(2):
+        for t in out.values():
+            t.zero_()
+        h2d, d2h = eng.step_host(host, out)
+        torch.cuda.synchronize()
+        assert eng.status()[0] == 0
+        assert h2d == sum(host[n].numel() * host[n].element_size() for n in ("q", "k", "v", "do"))
+        assert d2h == sum(t.numel() * t.element_size() for t in out.values())
+        for n in ("o", "lse", "dk", "dv"):
+            assert torch.equal(out[n], want[n]), n
+        assert torch.allclose(out["dq"].float(), want["dq"].float(), rtol=2 ** -7, atol=1e-6)
+
+
 def test_routed_shards_run_through_the_kernels(env):
     """Planner output instead of a hand-made shard: a scaled-down long-tailed batch is routed over eight GPUs (cost
     table from the shipped measured coefficients, Algorithm 1), and the shards of the first GPU and of the GPU with
