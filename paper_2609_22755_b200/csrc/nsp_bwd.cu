@@ -752,8 +752,21 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
                    a.scale_log2, -l4.x, -l4.y);
               fma2(x2, x3, __uint_as_float(sv[ch >> 1][x + 2]), __uint_as_float(sv[ch >> 1][x + 3]), a.scale_log2,
                    a.scale_log2, -l4.z, -l4.w);
-              pp[ch >> 1][(x >> 1) + 0] = pack_bf16x2(ex2f(x0), ex2f(x1));
-              pp[ch >> 1][(x >> 1) + 1] = pack_bf16x2(ex2f(x2), ex2f(x3));
+              float p0, p1, p2, p3;
+              if (((2 * i) & 3) < NSP_EMU_BWD) {
+                ex2_poly2(p0, p1, x0, x1);
+              } else {
+                p0 = ex2f(x0);
+                p1 = ex2f(x1);
+              }
+              if (((2 * i + 1) & 3) < NSP_EMU_BWD) {
+                ex2_poly2(p2, p3, x2, x3);
+              } else {
+                p2 = ex2f(x2);
+                p3 = ex2f(x3);
+              }
+              pp[ch >> 1][(x >> 1) + 0] = pack_bf16x2(p0, p1);
+              pp[ch >> 1][(x >> 1) + 1] = pack_bf16x2(p2, p3);
             }
             if constexpr (decltype(diag_tag)::value) {
               // diagonal tile: a key sees only the queries at or after it. Element e of this chunk (query column

@@ -423,7 +423,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 mx_tile = max3f(mx_tile, __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
                 fma2(x0, x1, __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]), a.scale_log2, a.scale_log2, neg_m,
                      neg_m);
-                const float p0 = ex2f(x0), p1 = ex2f(x1);
+                float p0, p1;
+                if (((e >> 1) & 3) < NSP_EMU_FWD) {
+                  ex2_poly2(p0, p1, x0, x1);
+                } else {
+                  p0 = ex2f(x0);
+                  p1 = ex2f(x1);
+                }
                 add2(sum0, sum1, sum0, sum1, p0, p1);
                 pk[c * 16 + (e >> 1)] = pack_bf16x2(p0, p1);
               }
