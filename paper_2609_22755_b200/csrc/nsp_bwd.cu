@@ -18,9 +18,9 @@
 // Roles:  warps 0-7  softmax / dS (key row = TMEM lane, two column halves)
 //         warps 8-15 dQ: TMEM -> fp32 accumulator in global memory (lane quadrant x 64-column half)
 //         warp 16    TMA producer (K, V once per item; Q two-stage ring, dO single buffer)
-//         warp 17    MMA issuer A (single thread): dV(t), S^T(t+1)
+//         warp 17    MMA issuer A (whole warp runs the waits, the elected lane issues): dV(t), S^T(t+1)
 //         warp 18    LSE / delta loader (two-stage ring in shared memory)
-//         warp 19    MMA issuer B (single thread): dK(t), dQ^T(t), dP^T(t+1)
+//         warp 19    MMA issuer B (likewise): dQ^T(t), dK(t), dP^T(t+1)
 // The softmax warps hand over P^T first (p_ready) and dS^T second (ds_ready), so dV(t) and S^T(t+1) run under
 // the dS phase of step t, and dK(t), dQ^T(t), dP^T(t+1) under the exp2 phase of step t+1.
 // dQ is produced TRANSPOSED (head dimension on the TMEM lanes): a warp of the dQ warpgroups then holds 32
@@ -336,11 +336,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       }
     } else if (warp == 17 || warp == 19) {
       // ================================================================ MMA issuers
-      // Two issuing threads share the step: thread A (warp 17) owns R0 and dV: dV(t), S^T(t+1); thread B
-      // (warp 19) owns R1 and dK: dK(t), dQ^T(t), dP^T(t+1). Each has its own chain of waits, so the bookkeeping
-      // of one (a single thread on a busy sub-partition runs at a dozen clocks per instruction) hides behind
-      // the MMAs of the other. Each thread signals completion on barriers of its own (a tcgen05.commit covers
-      // only the issuing thread's MMAs); whoever depends on both waits for both.
+      // Two issuing warps share the step: warp 17 (A) owns R0 and dV: dV(t), S^T(t+1); warp 19 (B) owns R1 and
+      // dK: dQ^T(t), dK(t), dP^T(t+1). Each has its own chain of waits, so the bookkeeping of one hides behind
+      // the MMAs of the other. All 32 lanes run the waits and the address arithmetic (convergent code); the lane
+      // elect.sync picks issues the MMAs and the commits. Each issuer signals completion on barriers of its own
+      // (a tcgen05.commit covers only the issuing thread's MMAs); whoever depends on both waits for both.
       const bool is_a = warp == 17;
       QRing qr;
       while (next_item()) {
