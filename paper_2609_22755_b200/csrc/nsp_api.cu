@@ -89,6 +89,25 @@ bool encode_run_map(CUtensorMap* out, const void* base, int64_t elem_off, int64_
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 [tokens, heads, head_dim] output of one run, boxes of 32 columns x 128 rows (128 bytes per row, 128-byte swizzle)
+bool encode_run_map_f32(CUtensorMap* out, void* base, int64_t elem_off, int64_t tokens, int heads, int head_dim) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return false;
+  if (tokens <= 0) {
+    std::memset(out, 0, sizeof(*out));
+    return true;
+  }
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(head_dim), static_cast<cuuint64_t>(heads),
+                              static_cast<cuuint64_t>(tokens)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(head_dim) * 4, static_cast<cuuint64_t>(heads) * head_dim * 4};
+  const cuuint32_t box[3] = {32, 1, 128};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  void* ptr = static_cast<char*>(base) + elem_off * 4;
+  return enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Order in which the backward kernel walks its work items (nsp_plan_get, pass 2). The published work list (pass 1)
 // is sorted by cost alone; walked in that order, the CTAs that run at the same time hold key tiles of MANY (segment,
 // kv head) groups, a q tile's fp32 dQ accumulator rows are touched by a few CTAs now and by the others much later,
@@ -436,7 +455,8 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
     const RunInfo& run = plan->runs[r];
     if (!encode_run_map(&maps.q[r], q, run.q_off, run.tokens, run.hq, plan->head_dim) ||
         !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv, plan->head_dim) ||
-        !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv, plan->head_dim))
+        !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv, plan->head_dim) ||
+        !encode_run_map(&maps.o[r], o, run.q_off, run.tokens, run.hq, plan->head_dim))
       return NSP_ERR_CUDA;
   }
   if (cudaMemsetAsync(plan->d_counters, 0, sizeof(int32_t), st) != cudaSuccess) return NSP_ERR_CUDA;
@@ -520,6 +540,9 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
         !encode_run_map(&maps.d_o[r], d_o, run.q_off, run.tokens, run.hq, plan->head_dim) ||
         !encode_run_map(&maps.k[r], k, run.kv_off, run.tokens, run.hkv, plan->head_dim) ||
         !encode_run_map(&maps.v[r], v, run.kv_off, run.tokens, run.hkv, plan->head_dim))
+      return NSP_ERR_CUDA;
+    if (dkv_dtype == NSP_F32 && (!encode_run_map_f32(&maps.dk[r], dk, run.kv_off, run.tokens, run.hkv, plan->head_dim) ||
+                                 !encode_run_map_f32(&maps.dv[r], dv, run.kv_off, run.tokens, run.hkv, plan->head_dim)))
       return NSP_ERR_CUDA;
     if (recompute) fmaps.q[r] = maps.q[r], fmaps.k[r] = maps.k[r], fmaps.v[r] = maps.v[r];
   }

@@ -29,6 +29,8 @@
 // bandwidth (MMA operand reads, TMA fills, dS^T) is a scarce resource of this kernel.
 // dK and dV accumulate in TMEM over the whole item in a fixed order (q tiles descending, heads ascending inside
 // a tile), so the reduction over the query heads of a group is deterministic.
+// At the end of an item a full fp32 tile of each is staged in the (then idle) operand buffers and written by TMA tile
+// stores; bf16 outputs and ragged tiles are stored row by row from the threads.
 // For the first q tile of a segment (rows 0..127, where P is O(1)) the step runs twice, once with the bf16
 // value of P and dS and once with the bf16 residual (hi + lo), and delta is recomputed in fp32 as
 // sum_j P_ij dP_ij instead of taking it from the bf16-rounded O; this keeps dK/dV/dQ inside the 2e-2 tolerance.
@@ -56,7 +58,8 @@ constexpr int kFrontMinGroup = 8;             // so do items of groups with fewe
 constexpr long long kFrontWaitClk = 1500000;  // ~0.9 ms: upper bound of the start alignment (also: 1/16 of the item)
 constexpr int kQStages = 2;                   // Q ring (three stages measured 3 % slower on the nested shard)
 
-// A decoded work item: written by thread 0, read by every role after the CTA-wide barrier of next_item().
+// A decoded work item: written by one thread (thread 0, or the producer's lane 0 one item ahead), read by every role
+// after the CTA-wide barrier of next_item().
 struct ItemCtx {
   int64_t q_off, kv_off, lse_off;  // element offsets of the segment
   int32_t it;                      // position in the work list (>= n_items: no more work)
@@ -96,6 +99,7 @@ struct BwdSmem {
   uint64_t bar_p_ready;   // 256 softmax threads: P^T of the step is in R0
   uint64_t bar_ds_ready;  // 256 softmax threads: dS^T of the step is in shared memory
   uint64_t bar_delta[2];  // 128 softmax threads of one column half: partial / final sums of the exact delta
+  uint64_t bar_out;       // 256 softmax threads: the item's dK and dV tiles are staged for the tile stores
   uint32_t tmem_base;
   int32_t abort;
 };
@@ -194,6 +198,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     mbar_init(&s.bar_dq_empty, 256);
     mbar_init(&s.bar_delta[0], 128);
     mbar_init(&s.bar_delta[1], 128);
+    mbar_init(&s.bar_out, 256);
     s.abort = 0;
     fence_mbar_init();
   }
@@ -222,54 +227,63 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   // Every role runs its own copy of the item loop (so that its register budget, set by setmaxnreg at the top of
   // the role, governs the whole loop); the loops meet at the CTA-wide barrier inside next_item().
   const ItemCtx* cx = nullptr;
+  // One thread pops the next item and decodes it into a slot of s.ctx: the atomic, the dependent loads and (for long
+  // items of large groups) the start alignment take ~4,000 clocks and more. After a short item the TMA producer's
+  // lane 0 has done it ahead, into the other slot, while the item's last steps and its epilogue ran: it is the one
+  // thread with nothing left to do then (4,400 -> ~1,000 clocks per item boundary; 4 % of a backward pass over
+  // 512-token segments). Both sides derive "ahead" from the finished item's step count, so no flag is needed; the
+  // barrier below publishes the slot either way.
+  constexpr int kAheadMaxSteps = 64;
+  auto fetch_item = [&](ItemCtx& x) {
+    for (;;) {
+      const int idx = atomicAdd(a.counter, 1);
+      x.it = idx;
+      if (idx >= a.n_items) break;
+      const nsp_tile_t item = a.items[idx];
+      const SegInfo sg = a.seg[item.seg];
+      x.q_off = sg.q_off, x.kv_off = sg.kv_off, x.lse_off = sg.lse_off;
+      x.len = sg.len, x.hq = sg.hq, x.hkv = sg.hkv, x.run = sg.run, x.tok0 = sg.tok_in_run;
+      x.g = item.head, x.n = item.tile;
+      x.G = sg.hq / sg.hkv;
+      x.turn_off = sg.turn_off, x.mt = (sg.len + kBM - 1) / kBM;
+      x.first = (item.tile == 0);
+      if constexpr (FIRST) {
+        x.m0 = 0;
+        x.per_head = 1;  // q tile 0 only
+        x.steps = x.G;
+        break;
+      }
+      x.m0 = item.tile + x.first;                        // q tile 0 belongs to the first-tile kernel
+      x.per_head = (sg.len + kBM - 1) / kBM - x.m0;      // q tiles max(n, 1) .. Mt-1 (bm == bn)
+      x.steps = x.G * x.per_head;
+      // Start alignment. kFrontBlock consecutive items are neighbouring key tiles of one (segment, kv head) and
+      // walk the same (q tile, head) sequence from the segment's last q tile down. CTAs that start them at the
+      // same moment stay on the same q tile for the whole item and find its Q, dO and dQ-accumulator tiles in
+      // L2; left alone they start one q tile apart (items end G steps apart), and 148 CTAs on 148 different q
+      // tiles need 148 * G * 128 KB of L2: more than there is from G = 8 on (measured at G = 16: 900 GB of DRAM
+      // traffic for tensors of 15 GB). So the CTA of a long item of such a group waits here, for at most
+      // kFrontWaitClk, until the other items of its block have been popped as well (the CTAs that pop them are
+      // the next ones to finish, G steps apart). A timeout is not an error: the CTA just starts.
+      {
+        const int blk = idx / kFrontBlock;
+        const int rest = a.n_items - blk * kFrontBlock;
+        const int expect = rest < kFrontBlock ? rest : kFrontBlock;
+        atomicAdd(a.front + blk, 1);
+        if (x.steps >= kFrontMinSteps && x.G >= kFrontMinGroup) {
+          const long long t0 = clock64();
+          const long long own = static_cast<long long>(x.steps) * 340;  // about 1/16 of what the item takes
+          const long long limit = own < kFrontWaitClk ? own : kFrontWaitClk;
+          while (*reinterpret_cast<volatile int32_t*>(a.front + blk) < expect && clock64() - t0 < limit)
+            __nanosleep(200);
+        }
+      }
+      if (x.steps > 0) break;  // the only key tile of a one-tile segment has nothing left to do here
+    }
+  };
   auto next_item = [&]() -> bool {
     ItemCtx& x = s.ctx[gi & 1];
-    if (tid == 0) {
-      for (;;) {
-        const int idx = atomicAdd(a.counter, 1);
-        x.it = idx;
-        if (idx >= a.n_items) break;
-        const nsp_tile_t item = a.items[idx];
-        const SegInfo sg = a.seg[item.seg];
-        x.q_off = sg.q_off, x.kv_off = sg.kv_off, x.lse_off = sg.lse_off;
-        x.len = sg.len, x.hq = sg.hq, x.hkv = sg.hkv, x.run = sg.run, x.tok0 = sg.tok_in_run;
-        x.g = item.head, x.n = item.tile;
-        x.G = sg.hq / sg.hkv;
-        x.turn_off = sg.turn_off, x.mt = (sg.len + kBM - 1) / kBM;
-        x.first = (item.tile == 0);
-        if constexpr (FIRST) {
-          x.m0 = 0;
-          x.per_head = 1;  // q tile 0 only
-          x.steps = x.G;
-          break;
-        }
-        x.m0 = item.tile + x.first;                        // q tile 0 belongs to the first-tile kernel
-        x.per_head = (sg.len + kBM - 1) / kBM - x.m0;      // q tiles max(n, 1) .. Mt-1 (bm == bn)
-        x.steps = x.G * x.per_head;
-        // Start alignment. kFrontBlock consecutive items are neighbouring key tiles of one (segment, kv head) and
-        // walk the same (q tile, head) sequence from the segment's last q tile down. CTAs that start them at the
-        // same moment stay on the same q tile for the whole item and find its Q, dO and dQ-accumulator tiles in
-        // L2; left alone they start one q tile apart (items end G steps apart), and 148 CTAs on 148 different q
-        // tiles need 148 * G * 128 KB of L2: more than there is from G = 8 on (measured at G = 16: 900 GB of DRAM
-        // traffic for tensors of 15 GB). So the CTA of a long item of such a group waits here, for at most
-        // kFrontWaitClk, until the other items of its block have been popped as well (the CTAs that pop them are
-        // the next ones to finish, G steps apart). A timeout is not an error: the CTA just starts.
-        {
-          const int blk = idx / kFrontBlock;
-          const int rest = a.n_items - blk * kFrontBlock;
-          const int expect = rest < kFrontBlock ? rest : kFrontBlock;
-          atomicAdd(a.front + blk, 1);
-          if (x.steps >= kFrontMinSteps && x.G >= kFrontMinGroup) {
-            const long long t0 = clock64();
-            const long long own = static_cast<long long>(x.steps) * 340;  // about 1/16 of what the item takes
-            const long long limit = own < kFrontWaitClk ? own : kFrontWaitClk;
-            while (*reinterpret_cast<volatile int32_t*>(a.front + blk) < expect && clock64() - t0 < limit)
-              __nanosleep(200);
-          }
-        }
-        if (x.steps > 0) break;  // the only key tile of a one-tile segment has nothing left to do here
-      }
-    }
+    const bool ahead = gi > 0 && cx->it < a.n_items && cx->steps <= kAheadMaxSteps;  // cx: the item just finished
+    if (tid == 0 && !ahead) fetch_item(x);
     tc_fence_before_sync();
     // Every role gets here in bounded time: all its other waits are bounded, and none of them returns before the end
     // of the kernel. (An mbarrier with a bounded wait in this place made the register allocation of the softmax role
@@ -331,6 +345,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
 #pragma unroll
             for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.d_o[hf], mdo, &s.bar_do_full, 64 * hf, h, c.tok0 + m * kBM);
           }
+          if (c.steps <= kAheadMaxSteps) fetch_item(s.ctx[(gi + 1) & 1]);  // see next_item(): the same rule on both sides
         }
         item_done();
       }
@@ -950,6 +965,53 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         const bool valid = kj < c.len;
         constexpr int kCols = D / 2;  // this thread's columns of a dK / dV row
         const int64_t off = c.kv_off + (static_cast<int64_t>(kj) * c.hkv + c.g) * kHeadDim + half * kCols;
+        // Key tile 0 in the main kernel: the first-tile kernel, which ran before, left its part (q tile 0) in the
+        // output; this item's sum over the q tiles 1 .. Mt-1 is added to it (one fixed order: reproducible).
+        const bool add = !FIRST && c.first;
+        if (a.dkv_f32 && (c.n + 1) * kBN <= c.len) {
+          // ---- fp32 outputs, full key tile: staged in shared memory (every operand buffer is free now: dK over K
+          // and V, dV over the Q ring), swizzled as sub-tiles of 32 columns, and written by TMA tile stores (added,
+          // for key tile 0). Stored row by row from the threads (a row per lane, 16 bytes per store, half a sector
+          // each) the two tiles took 12,000-13,000 clocks per item.
+          constexpr uint32_t kSubBytes = 128 * 32 * 4;
+#pragma unroll 1
+          for (int part = 0; part < 2 * (kCols / 32); ++part) {  // (dK, dV) x 32-column chunks
+            const int which = part / (kCols / 32), cc = part % (kCols / 32);
+            const float mul = which == 0 ? a.scale : 1.f;
+            uint32_t v[32];
+            tmem_ld32(tDK + which * 128 + lane_off + half * kCols + cc * 32, v);
+            tmem_wait_ld();
+            uint8_t* const sub = (which == 0 ? &s.k[0][0] : &s.q[0][0][0]) + (half * (kCols / 32) + cc) * kSubBytes + r * 128;
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+              *reinterpret_cast<float4*>(sub + ((x ^ (r & 7)) * 16)) =
+                  make_float4(__uint_as_float(v[4 * x]) * mul, __uint_as_float(v[4 * x + 1]) * mul,
+                              __uint_as_float(v[4 * x + 2]) * mul, __uint_as_float(v[4 * x + 3]) * mul);
+            }
+          }
+          fence_proxy_async_smem();
+          const uint64_t staged = mbar_arrive_token(&s.bar_out);
+          if (tid == 0) {
+            if (mbar_wait_token(&s.bar_out, staged, a.wait_limit)) {
+              const int tok = c.tok0 + c.n * kBN;
+#pragma unroll 1
+              for (int i = 0; i < D / 32; ++i) {
+                if (add) {
+                  tma_reduce_add_3d(&maps.dk[c.run], &s.k[0][0] + i * kSubBytes, 32 * i, c.g, tok);
+                  tma_reduce_add_3d(&maps.dv[c.run], &s.q[0][0][0] + i * kSubBytes, 32 * i, c.g, tok);
+                } else {
+                  tma_store_3d(&maps.dk[c.run], &s.k[0][0] + i * kSubBytes, 32 * i, c.g, tok);
+                  tma_store_3d(&maps.dv[c.run], &s.q[0][0][0] + i * kSubBytes, 32 * i, c.g, tok);
+                }
+              }
+              tma_store_commit();
+              tma_store_wait_read();  // before the barrier of next_item(): the producer refills these buffers after it
+            } else {
+              report_timeout(a.status, c.it, kWhereBwdDqFull, 1);
+              *abort_flag = 1;
+            }
+          }
+        } else {
 #pragma unroll 1
         for (int part = 0; part < 2 * (kCols / 32); ++part) {  // (dK, dV) x 32-column chunks
           const int which = part / (kCols / 32), cc = part % (kCols / 32);
@@ -958,9 +1020,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           uint32_t v[32];
           tmem_ld32(tDK + which * 128 + lane_off + half * kCols + cc * 32, v);
           tmem_wait_ld();
-          // Key tile 0 in the main kernel: the first-tile kernel, which ran before, left its part (q tile 0) in the
-          // output; this item's sum over the q tiles 1 .. Mt-1 is added to it (one fixed order: reproducible).
-          const bool add = !FIRST && c.first;
           NSP_CHECK(!valid || (off >= 0 && off + kCols <= a.kv_elems), a.status, c.it, kWhereCheckBwdDkv, kj)
           if (valid) {
             if (a.dkv_f32) {
@@ -998,6 +1057,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               }
             }
           }
+        }
         }
       } else if (where != 0 && lane == 0) {
         report_timeout(a.status, c.it, where, 0);

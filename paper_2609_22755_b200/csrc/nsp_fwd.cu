@@ -11,8 +11,9 @@
 // Issue order of the single MMA thread: PV_A(j), S_A(j+1), PV_B(j), S_B(j+1): S of the next key tile is already
 // running while the other half's softmax is still working. TMEM: S_A, S_B, O_A, O_B = 4 x 128 columns.
 // Roles: warps 0-7 softmax of A, warps 8-15 softmax of B (two threads per query row, 64 score columns each), warp 16
-// TMA producer (Q pair, two-stage K and V rings), warp 17 MMA issuer; register budgets are set per warpgroup with
-// setmaxnreg.
+// TMA producer (Q pair, two-stage K and V rings; it also starts the coming round's first tiles under the running
+// round's tail), warp 17 MMA issuer, warp 18 lane 0 pops the work list one pop ahead; register budgets are set per
+// warpgroup with setmaxnreg. A full O tile leaves through shared memory as a TMA tile store.
 // O stays in TMEM for the whole item and is rescaled in place only when the running maximum grows by more than
 // 2^8 (the stale reference maximum is exact in the final normalisation because the same reference is used for
 // the row sum). Only the diagonal tile is masked; tiles above the diagonal are never visited.
@@ -28,12 +29,13 @@ constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;  // one [128 rows x 64 cols] b
 constexpr uint32_t kFwdTmemCols = 512;  // S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512)
 constexpr int kFwdRegsSoftmax = 104, kFwdRegsAux = 64;  // 4*104 + 64 = 480 = 5 * 96, the launch-time allocation
 
-// One pop of the work list, decoded by thread 0 into shared memory (two slots: the next pop is fetched while the
-// current one runs).
+// One pop of the work list, decoded by one thread of a spare warp into shared memory (two slots: the next pop is
+// fetched while the current one runs).
 struct FwdPop {
   SegInfo sa, sb;  // segments of items a and b
   nsp_tile_t a, b;
-  int32_t it0, joint, n_rounds, pad_;
+  int32_t it0, joint, n_rounds;
+  int32_t kt_base;  // key tiles of all earlier pops of this CTA (the K / V ring stage of tile t is t & 1)
 };
 
 // D = head dimension (128 or 64): a Q / K / V tile is D / 64 sub-tiles of 64 columns.
@@ -51,6 +53,9 @@ struct FwdSmem {
                              // half-row dot product of O and dO (3, recomputation only)
                              // (slot 2) handed to the partner thread
   uint64_t bar_pv_done[2];  // [A/B] O_x += P_x V has completed
+  uint64_t bar_q_free;      // the last S products of the round have completed: the Q tiles may be overwritten
+  uint64_t bar_o_staged[2];  // [A/B] 256 softmax threads: the tile's O rows are in the staging buffer
+  uint64_t bar_pop_ready[2];  // [slot] the pop fetched ahead is in its slot
   uint32_t tmem_base;
   FwdPop pop[2];
   int32_t abort;
@@ -103,6 +108,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       for (int qd = 0; qd < 4; ++qd) mbar_init(&s.bar_pair[i][qd], 64);
       mbar_init(&s.bar_pv_done[i], 1);
     }
+    mbar_init(&s.bar_q_free, 1);
+    mbar_init(&s.bar_o_staged[0], 256);
+    mbar_init(&s.bar_o_staged[1], 256);
+    mbar_init(&s.bar_pop_ready[0], 1);
+    mbar_init(&s.bar_pop_ready[1], 1);
     s.abort = 0;
     fence_mbar_init();
   }
@@ -130,11 +140,17 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   FwdRound rd;
   int n_rounds = 0, it0 = 0;
   const FwdPop* pp = nullptr;
-  // Thread 0 only. The atomic on the cursor and the dependent loads of the items and their segments take about as
-  // long as a whole single-tile item, so after a short item they are done one pop ahead (after a long one the
-  // cursor is read when the item ends, which keeps the work list's balance at the end of the launch).
+  // One thread only, lane 0 of a spare warp of the auxiliary warpgroup. The atomic on the cursor and the dependent
+  // loads of the items and their segments take ~4,000 clocks, so after a short item they are done one pop ahead (after
+  // a long one the cursor is read when the item ends, which keeps the work list's balance at the end of the launch) —
+  // and by a thread nobody waits for: when thread 0, a softmax thread, did it, its warp came that much later to the
+  // first score tile of every round (17 % of a round at 512-token segments).
+  constexpr int kFetchTid = 18 * 32;
   bool fetched_ahead = false;
-  auto fetch_pop = [&](FwdPop& p) {
+  uint32_t kt_total = 0;  // fetching thread: key tiles of the pops fetched so far
+  constexpr int kFetchAheadCost = 128;  // items up to this many key tiles have their successor fetched while they run
+  auto fetch_pop = [&](int slot) {
+    FwdPop& p = s.pop[slot];
     for (;;) {
       const int it = atomicAdd(a.counter, 2);
       p.it0 = it;
@@ -154,11 +170,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       const int G = sa.hq / sa.hkv;
       p.joint = have_b && ib.seg == ia.seg && ib.tile == ia.tile && (ia.head / G == ib.head / G);
       p.n_rounds = p.joint ? 1 : (have_b ? 2 : 1);
+      p.kt_base = static_cast<int32_t>(kt_total);
+      kt_total += static_cast<uint32_t>(ia.cost + (p.n_rounds == 2 ? ib.cost : 0));
       break;
     }
+    mbar_arrive(&s.bar_pop_ready[slot]);  // phase gp / 2 of the slot: the producer may read it before the next barrier
   };
   auto next_pop = [&]() -> bool {
-    if (tid == 0 && !fetched_ahead) fetch_pop(s.pop[gp & 1]);
+    if (tid == kFetchTid && !fetched_ahead) fetch_pop(gp & 1);
     cta_sync();
     pp = &s.pop[gp & 1];
     it0 = pp->it0;
@@ -167,20 +186,28 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     rd.a = pp->a, rd.b = pp->b, rd.joint = pp->joint;
     n_rounds = pp->n_rounds;
     // the other slot held the previous pop: every role left it before it came to the barrier above
-    if (tid == 0) {
-      fetched_ahead = rd.a.cost <= 8;
-      if (fetched_ahead) fetch_pop(s.pop[gp & 1]);
+    if (tid == kFetchTid) {
+      fetched_ahead = rd.a.cost <= kFetchAheadCost;
+      if (fetched_ahead) fetch_pop(gp & 1);
     }
     return true;
   };
-  // end of a round: every warp has finished with the Q tiles, the K/V rings and the TMEM accumulators
-  auto round_end = [&]() { cta_sync(); };
+  // end of a round: every warp has finished with the Q tiles, the K/V rings and the TMEM accumulators. After the last
+  // round of a pop the barrier of next_pop() is that meeting point.
+  auto round_end = [&](int r) {
+    if (r + 1 < n_rounds) cta_sync();
+  };
 
   if (wg == 4) {
     fwd_setmaxnreg_dec<kFwdRegsAux>();
     if (warp == 16) {
       // ================================================================ TMA producer
-      uint32_t kn = 0, vn = 0;
+      // Besides the loads of the running round it starts those of the coming one (the Q tiles and the first K / V
+      // tile) as soon as the last S products of the running round have left the Q tiles, i.e. under the last softmax,
+      // the last PV products and the epilogue. Short items pay for it otherwise: ~3,800 clocks from the start of a
+      // round to its first score tile, a sixth of a round at 512-token segments.
+      uint32_t kn = 0, vn = 0, rn = 0;
+      bool pre = false;  // lane 0: Q and key tile 0 of the running round were started during the previous one
       while (next_pop()) {
         for (int r = 0; r < n_rounds; ++r) {
           if (lane == 0 && !*abort_flag) {
@@ -191,14 +218,16 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             const CUtensorMap* mq = &maps.q[sg.run];
             const CUtensorMap* mk = &maps.k[sg.run];
             const CUtensorMap* mv = &maps.v[sg.run];
-            mbar_expect_tx(&s.bar_q, rd.joint ? 2 * kTileBytes : kTileBytes);
+            if (!pre) {
+              mbar_expect_tx(&s.bar_q, rd.joint ? 2 * kTileBytes : kTileBytes);
 #pragma unroll
-            for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[0][hf], mq, &s.bar_q, 64 * hf, ia.head, tok0 + q_row0);
-            if (rd.joint) {
+              for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[0][hf], mq, &s.bar_q, 64 * hf, ia.head, tok0 + q_row0);
+              if (rd.joint) {
 #pragma unroll
-              for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[1][hf], mq, &s.bar_q, 64 * hf, rd.b.head, tok0 + q_row0);
+                for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[1][hf], mq, &s.bar_q, 64 * hf, rd.b.head, tok0 + q_row0);
+              }
             }
-            for (int j = 0; j < n_kv; ++j) {
+            for (int j = pre ? 1 : 0; j < n_kv; ++j) {
               if (*abort_flag) break;
               uint32_t st = kn & 1;
               if (!mbar_wait(&s.bar_k_empty[st], ((kn >> 1) & 1) ^ 1, a.wait_limit)) {
@@ -227,8 +256,49 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.v[st][hf], mv, &s.bar_v_full[st], 64 * hf, g, tok0 + j * kBN);
               ++vn;
             }
+            pre = false;
+            // ---- the coming round (the second item of this pop, or the first round of the pop fetched ahead): its Q
+            // tiles and its first K / V tile, once the last S products of this round have left the Q tiles. Kept apart
+            // from the loop above, whose code the long items live in (sharing its body through a lambda cost them 0.6 %).
+            const FwdPop* nx = nullptr;
+            int second = 0;
+            if (r + 1 < n_rounds) {
+              nx = pp, second = 1;
+            } else if (n_kv <= kFetchAheadCost && mbar_wait(&s.bar_pop_ready[gp & 1], (gp >> 1) & 1, a.wait_limit)) {
+              if (s.pop[gp & 1].it0 < a.n_items) nx = &s.pop[gp & 1];
+            }
+            if (nx != nullptr && !*abort_flag && mbar_wait(&s.bar_q_free, rn & 1, a.wait_limit)) {
+              const nsp_tile_t* na = second ? &nx->b : &nx->a;
+              const SegInfo* ns = second ? &nx->sb : &nx->sa;
+              const int joint = second ? 0 : nx->joint;
+              const int ng = na->head / (ns->hq / ns->hkv), ntok = ns->tok_in_run;
+              mbar_expect_tx(&s.bar_q, joint ? 2 * kTileBytes : kTileBytes);
+#pragma unroll
+              for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[0][hf], &maps.q[ns->run], &s.bar_q, 64 * hf, na->head, ntok + na->tile * kBM);
+              if (joint) {
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[1][hf], &maps.q[ns->run], &s.bar_q, 64 * hf, nx->b.head, ntok + na->tile * kBM);
+              }
+              const uint32_t kst = kn & 1, vst = vn & 1;
+              if (mbar_wait(&s.bar_k_empty[kst], ((kn >> 1) & 1) ^ 1, a.wait_limit) &&
+                  mbar_wait(&s.bar_v_empty[vst], ((vn >> 1) & 1) ^ 1, a.wait_limit)) {
+                mbar_expect_tx(&s.bar_k_full[kst], kTileBytes);
+                mbar_expect_tx(&s.bar_v_full[vst], kTileBytes);
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf) {
+                  tma_load_3d(s.k[kst][hf], &maps.k[ns->run], &s.bar_k_full[kst], 64 * hf, ng, ntok);
+                  tma_load_3d(s.v[vst][hf], &maps.v[ns->run], &s.bar_v_full[vst], 64 * hf, ng, ntok);
+                }
+                ++kn, ++vn;
+                pre = true;
+              } else {
+                report_timeout(a.status, it0, kWhereFwdLoad, 200000);
+                *abort_flag = 1;
+              }
+            }
           }
-          round_end();
+          ++rn;
+          round_end(r);
         }
       }
     } else if (warp == 17) {
@@ -289,6 +359,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               }
               const uint32_t vst = vn & 1;
               const bool more = j + 1 < n_kv;
+              if (!more && leader) umma_commit(&s.bar_q_free);  // every S product of the round has been issued
               if (!mbar_wait(&s.bar_p_ready[0], pn[0] & 1, a.wait_limit)) { ok = false; where = kWhereFwdS; break; }
               ++pn[0];
               if (!mbar_wait(&s.bar_v_full[vst], (vn >> 1) & 1, a.wait_limit)) { ok = false; where = kWhereFwdLoad; break; }
@@ -319,12 +390,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               *abort_flag = 1;
             }
           }
-          round_end();
+          round_end(r);
         }
       }
     } else {
       while (next_pop())
-        for (int r = 0; r < n_rounds; ++r) round_end();  // spare warps: only keep the CTA-wide barrier count
+        for (int r = 0; r < n_rounds; ++r) round_end(r);  // spare warps: only keep the CTA-wide barrier count
     }
   } else {
     // ================================================================ softmax of item x (A: warps 0-7, B: warps 8-15)
@@ -522,7 +593,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               report_timeout(a.status, it0, where, 0);
               *abort_flag = 1;
             }
-            round_end();
+            round_end(r);
             continue;
           }
           if (ok) {  // row sum = sum of the two half rows
@@ -538,6 +609,50 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             l += partner_slot[256];
             tc_fence_after_sync();
             const float inv_l = 1.f / l;
+            if (q_row0 + kBM <= sg.len) {
+              // ---- a full tile goes out as a TMA tile store. The rows are staged, swizzled like an operand tile, in
+              // the ring stage of the round's last key tile: K's for item A, V's for item B. Both are free: the last
+              // PV product of this half has completed, and the tensor pipe runs one thread's products in order, so
+              // the last S and PV products of the other half, which read the same stages, have completed as well; the
+              // tiles the producer has already started for the coming round sit in the other stage. Written row by
+              // row from the threads (each lane another row, 8 KB apart) the same tile cost 3,900 clocks per round:
+              // the store path takes one 32-byte sector per clock, and every 16-byte store was half a sector.
+              const int kt = pp->kt_base + rd.a.cost + (r == 1 ? rd.b.cost : 0);  // key tiles up to the end of this round
+              uint8_t* const stage = (x == 0 ? s.k : s.v)[(kt - 1) & 1][0];
+              uint8_t* const srow = stage + (D == 128 ? ch : 0) * kHalfTileBytes + rl * 128;
+              constexpr int kChunk0 = 0;
+#pragma unroll
+              for (int c = 0; c < kOCols / 32; ++c) {
+                uint32_t orow[32];
+                tmem_ld32(tO + lane_off + ch * kOCols + c * 32, orow);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  uint4 w;
+                  w.x = pack_bf16x2(__uint_as_float(orow[8 * e + 0]) * inv_l, __uint_as_float(orow[8 * e + 1]) * inv_l);
+                  w.y = pack_bf16x2(__uint_as_float(orow[8 * e + 2]) * inv_l, __uint_as_float(orow[8 * e + 3]) * inv_l);
+                  w.z = pack_bf16x2(__uint_as_float(orow[8 * e + 4]) * inv_l, __uint_as_float(orow[8 * e + 5]) * inv_l);
+                  w.w = pack_bf16x2(__uint_as_float(orow[8 * e + 6]) * inv_l, __uint_as_float(orow[8 * e + 7]) * inv_l);
+                  const int chunk = kChunk0 + (D == 128 ? 0 : ch * 4) + c * 4 + e;  // 16-byte chunk of the 128-byte row
+                  *reinterpret_cast<uint4*>(srow + ((chunk ^ (rl & 7)) * 16)) = w;
+                }
+              }
+              fence_proxy_async_smem();
+              const uint64_t staged = mbar_arrive_token(&s.bar_o_staged[x]);
+              if (ch == 0 && rl == 0) {  // one thread of the tile: wait for all rows, store, wait for the reads
+                if (mbar_wait_token(&s.bar_o_staged[x], staged, a.wait_limit)) {
+#pragma unroll
+                  for (int hf = 0; hf < kHalves; ++hf)
+                    tma_store_3d(&maps.o[sg.run], stage + hf * kHalfTileBytes, 64 * hf, h, sg.tok_in_run + q_row0);
+                  tma_store_commit();
+                  tma_store_wait_read();
+                } else {
+                  report_timeout(a.status, it0, kWhereFwdO, 1);
+                  *abort_flag = 1;
+                }
+              }
+            } else {
+            // ---- ragged last tile of a segment: the valid rows only, straight from the threads
             __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim + ch * kOCols;
 #pragma unroll
             for (int c = 0; c < kOCols / 32; ++c) {
@@ -557,6 +672,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 }
               }
             }
+            }
             if (valid && ch == 0) {
               const int64_t at = sg.lse_off + static_cast<int64_t>(h) * sg.len + row;
               NSP_CHECK(at >= 0 && at < a.lse_elems, a.status, it0, kWhereCheckFwdLse, row)
@@ -567,7 +683,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             *abort_flag = 1;
           }
         }
-        round_end();
+        round_end(r);
       }
     }
   }

@@ -36,9 +36,11 @@ struct RunInfo {
 // Tensor maps of every run, passed by value as a __grid_constant__ kernel parameter.
 struct FwdMaps {
   CUtensorMap q[NSP_MAX_RUNS], k[NSP_MAX_RUNS], v[NSP_MAX_RUNS];
+  CUtensorMap o[NSP_MAX_RUNS];  // output tiles of the general forward kernel (stores); same geometry as q
 };
 struct BwdMaps {
   CUtensorMap q[NSP_MAX_RUNS], d_o[NSP_MAX_RUNS], k[NSP_MAX_RUNS], v[NSP_MAX_RUNS];
+  CUtensorMap dk[NSP_MAX_RUNS], dv[NSP_MAX_RUNS];  // fp32 dK / dV outputs (tile stores of 32 columns x 128 rows); unset for bf16 outputs
 };
 
 // Device status record {code, item, where, aux}; the first writer wins (atomicCAS on the code in device memory) and
