@@ -620,7 +620,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
               const int kt = pp->kt_base + rd.a.cost + (r == 1 ? rd.b.cost : 0);  // key tiles up to the end of this round
               uint8_t* const stage = (x == 0 ? s.k : s.v)[(kt - 1) & 1][0];
               uint8_t* const srow = stage + (D == 128 ? ch : 0) * kHalfTileBytes + rl * 128;
-              constexpr int kChunk0 = 0;
 #pragma unroll
               for (int c = 0; c < kOCols / 32; ++c) {
                 uint32_t orow[32];
@@ -633,7 +632,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                   w.y = pack_bf16x2(__uint_as_float(orow[8 * e + 2]) * inv_l, __uint_as_float(orow[8 * e + 3]) * inv_l);
                   w.z = pack_bf16x2(__uint_as_float(orow[8 * e + 4]) * inv_l, __uint_as_float(orow[8 * e + 5]) * inv_l);
                   w.w = pack_bf16x2(__uint_as_float(orow[8 * e + 6]) * inv_l, __uint_as_float(orow[8 * e + 7]) * inv_l);
-                  const int chunk = kChunk0 + (D == 128 ? 0 : ch * 4) + c * 4 + e;  // 16-byte chunk of the 128-byte row
+                  const int chunk = (D == 128 ? 0 : ch * 4) + c * 4 + e;  // 16-byte chunk of the 128-byte row
                   *reinterpret_cast<uint4*>(srow + ((chunk ^ (rl & 7)) * 16)) = w;
                 }
               }
@@ -652,26 +651,26 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                 }
               }
             } else {
-            // ---- ragged last tile of a segment: the valid rows only, straight from the threads
-            __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim + ch * kOCols;
-#pragma unroll
-            for (int c = 0; c < kOCols / 32; ++c) {
-              uint32_t orow[32];
-              tmem_ld32(tO + lane_off + ch * kOCols + c * 32, orow);
-              tmem_wait_ld();
-              if (valid) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  uint4 w;
-                  w.x = pack_bf16x2(__uint_as_float(orow[8 * e + 0]) * inv_l, __uint_as_float(orow[8 * e + 1]) * inv_l);
-                  w.y = pack_bf16x2(__uint_as_float(orow[8 * e + 2]) * inv_l, __uint_as_float(orow[8 * e + 3]) * inv_l);
-                  w.z = pack_bf16x2(__uint_as_float(orow[8 * e + 4]) * inv_l, __uint_as_float(orow[8 * e + 5]) * inv_l);
-                  w.w = pack_bf16x2(__uint_as_float(orow[8 * e + 6]) * inv_l, __uint_as_float(orow[8 * e + 7]) * inv_l);
-                  NSP_CHECK(optr + c * 32 + e * 8 + 8 <= a.o + a.q_elems && optr >= a.o, a.status, it0, kWhereCheckFwdO, row)
-                  *reinterpret_cast<uint4*>(optr + c * 32 + e * 8) = w;
+              // ---- ragged last tile of a segment: the valid rows only, straight from the threads
+              __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim + ch * kOCols;
+  #pragma unroll
+              for (int c = 0; c < kOCols / 32; ++c) {
+                uint32_t orow[32];
+                tmem_ld32(tO + lane_off + ch * kOCols + c * 32, orow);
+                tmem_wait_ld();
+                if (valid) {
+  #pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    uint4 w;
+                    w.x = pack_bf16x2(__uint_as_float(orow[8 * e + 0]) * inv_l, __uint_as_float(orow[8 * e + 1]) * inv_l);
+                    w.y = pack_bf16x2(__uint_as_float(orow[8 * e + 2]) * inv_l, __uint_as_float(orow[8 * e + 3]) * inv_l);
+                    w.z = pack_bf16x2(__uint_as_float(orow[8 * e + 4]) * inv_l, __uint_as_float(orow[8 * e + 5]) * inv_l);
+                    w.w = pack_bf16x2(__uint_as_float(orow[8 * e + 6]) * inv_l, __uint_as_float(orow[8 * e + 7]) * inv_l);
+                    NSP_CHECK(optr + c * 32 + e * 8 + 8 <= a.o + a.q_elems && optr >= a.o, a.status, it0, kWhereCheckFwdO, row)
+                    *reinterpret_cast<uint4*>(optr + c * 32 + e * 8) = w;
+                  }
                 }
               }
-            }
             }
             if (valid && ch == 0) {
               const int64_t at = sg.lse_off + static_cast<int64_t>(h) * sg.len + row;
