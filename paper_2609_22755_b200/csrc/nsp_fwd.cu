@@ -653,13 +653,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
             } else {
               // ---- ragged last tile of a segment: the valid rows only, straight from the threads
               __nv_bfloat16* optr = a.o + sg.q_off + (static_cast<int64_t>(row) * sg.hq + h) * kHeadDim + ch * kOCols;
-  #pragma unroll
+#pragma unroll
               for (int c = 0; c < kOCols / 32; ++c) {
                 uint32_t orow[32];
                 tmem_ld32(tO + lane_off + ch * kOCols + c * 32, orow);
                 tmem_wait_ld();
                 if (valid) {
-  #pragma unroll
+#pragma unroll
                   for (int e = 0; e < 4; ++e) {
                     uint4 w;
                     w.x = pack_bf16x2(__uint_as_float(orow[8 * e + 0]) * inv_l, __uint_as_float(orow[8 * e + 1]) * inv_l);

@@ -27,6 +27,7 @@ constexpr int kThreads = 640;
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;
 constexpr uint32_t kTmemCols = 512;  // S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512)
 constexpr int kRegsSoftmax = 104, kRegsAux = 64;
+constexpr int kPopThread = 18 * 32;  // lane 0 of the first store warp pops: its item starts with a long wait anyway
 
 struct FirstCtx {
   int64_t q_off, lse_off;
@@ -40,11 +41,13 @@ struct FwdFirstSmem {
   uint8_t v[D / 64][kHalfTileBytes];
   uint8_t q[2][2][D / 64][kHalfTileBytes];  // [stage][A/B][64-column half]
   uint64_t bar_kv, bar_kv_free;
-  uint64_t bar_q_full[2], bar_q_empty[2];
+  uint64_t bar_q_full[2];
+  uint64_t bar_q_empty[2][2];  // [stage][A/B] the slot's O tile has left (or was never staged): the slot may be reloaded
   uint64_t bar_s_full[2];   // [A/B]
   uint64_t bar_p_ready[2];  // [A/B] 256 softmax threads: P_x written
   uint64_t bar_pv_done[2];  // [A/B] O_x complete
   uint64_t bar_o_free[2];   // [A/B] 256 softmax threads: O_x read out of TMEM
+  uint64_t bar_o_staged[2];  // [A/B] 256 softmax threads: the bf16 O tile is in shared memory (or went out row by row)
   uint64_t bar_pair[2][4];  // [A/B][lane quadrant] the two threads of every row have published their half-row value
   float xchg[2][2][2][128];  // [A/B][column half][slot: maximum, sum][row]
   FirstCtx ctx[2];
@@ -83,7 +86,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
     mbar_init(&s.bar_kv_free, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s.bar_q_full[i], 1);
-      mbar_init(&s.bar_q_empty[i], 1);
+      mbar_init(&s.bar_q_empty[i][0], 1);
+      mbar_init(&s.bar_q_empty[i][1], 1);
+      mbar_init(&s.bar_o_staged[i], 256);
       mbar_init(&s.bar_s_full[i], 1);
       mbar_init(&s.bar_p_ready[i], 256);
       mbar_init(&s.bar_pv_done[i], 1);
@@ -118,14 +123,14 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
     }
   };
   auto next_item = [&]() -> bool {
-    if (tid == 0 && gi == 0) fetch(s.ctx[0]);
+    if (tid == kPopThread && gi == 0) fetch(s.ctx[0]);
     // Every role reaches this barrier in bounded time: all its other waits are bounded and none returns early.
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     c = s.ctx[gi & 1];
     const bool more = c.it < a.n_items && !*abort_flag;
-    if (tid == 0 && more) fetch(s.ctx[(gi + 1) & 1]);  // the other slot held the item every role has left
+    if (tid == kPopThread && more) fetch(s.ctx[(gi + 1) & 1]);  // the other slot held the item every role has left
     return more;
   };
 
@@ -133,7 +138,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
     ff_setmaxnreg_dec<kRegsAux>();
     if (warp == 16) {
       // ================================================================ TMA producer
-      uint32_t R = 0;  // rounds issued so far
+      uint32_t R = 0;            // rounds issued so far
+      uint32_t use = 0;          // bit 2*stage + half: parity of the loads issued so far into that slot
       while (next_item()) {
         if (lane == 0) {
           const CUtensorMap* mq = &maps.q[c.run];
@@ -149,10 +155,12 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
           for (int r = 0; ok && r < c.rounds; ++r) {
             if (*abort_flag) break;
             const uint32_t st = (R + r) & 1;
-            ok = mbar_wait(&s.bar_q_empty[st], (((R + r) >> 1) & 1) ^ 1, a.wait_limit);
-            if (!ok) break;
             const int hA = c.g * c.G + 2 * r;
             const bool joint = 2 * r + 1 < c.G;
+            ok = mbar_wait(&s.bar_q_empty[st][0], ((use >> (2 * st)) & 1) ^ 1, a.wait_limit) &&
+                 (!joint || mbar_wait(&s.bar_q_empty[st][1], ((use >> (2 * st + 1)) & 1) ^ 1, a.wait_limit));
+            if (!ok) break;
+            use ^= (joint ? 3u : 1u) << (2 * st);
             mbar_expect_tx(&s.bar_q_full[st], joint ? 2 * kTileBytes : kTileBytes);
 #pragma unroll
             for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(s.q[st][0][hf], mq, &s.bar_q_full[st], 64 * hf, hA, c.tok0);
@@ -202,7 +210,6 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
             }
             if (leader) umma_commit(&s.bar_s_full[x]);
           }
-          if (leader) umma_commit(&s.bar_q_empty[st]);
           for (int x = 0; x < halves; ++x) {
             if (!mbar_wait(&s.bar_p_ready[x], n[x] & 1, a.wait_limit)) { ok = false; where = kWhereFwdS; break; }
             if (!mbar_wait(&s.bar_o_free[x], (n[x] & 1) ^ 1, a.wait_limit)) { ok = false; where = kWhereFwdO; break; }
@@ -224,7 +231,38 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
         ++gi;
       }
     } else {
-      while (next_item()) ++gi;  // spare warps: only keep the CTA-wide barrier count
+      // ================================================================ store warps (18: half A, 19: half B)
+      // A full O tile is staged by the softmax threads in the Q slot it came from (dead once S has run), swizzled
+      // like an operand tile, and leaves as a TMA tile store; the slot goes back to the producer when the store has
+      // read it. Lane 0 of warp 18 also pops the work items (next_item).
+      const int x = warp - 18;
+      uint32_t R = 0, nx = 0;
+      while (next_item()) {
+        for (int r = 0; r < c.rounds; ++r) {
+          if (x == 1 && 2 * r + 1 >= c.G) break;
+          if (*abort_flag) break;
+          if (lane == 0) {
+            const uint32_t st = (R + r) & 1;
+            if (mbar_wait(&s.bar_o_staged[x], nx & 1, a.wait_limit)) {
+              if (c.len >= kBM) {
+                const int h = c.g * c.G + 2 * r + x;
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf) tma_store_3d(&maps.o[c.run], s.q[st][x][hf], 64 * hf, h, c.tok0);
+                tma_store_commit();
+                tma_store_wait_read();
+              }
+              mbar_arrive(&s.bar_q_empty[st][x]);
+            } else {
+              report_timeout(a.status, c.it, kWhereFwdO, 2 + x);
+              *abort_flag = 1;
+            }
+          }
+          ++nx;
+        }
+        __syncwarp();
+        R += static_cast<uint32_t>(c.rounds);
+        ++gi;
+      }
     }
   } else {
     // ================================================================ softmax of half x (A: warps 0-7, B: warps 8-15)
@@ -237,6 +275,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
     const uint32_t tS = tmem + 128 * x, tO = tmem + 256 + 128 * x;
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
     uint32_t nx = 0;  // rounds in which this half took part
+    uint32_t R = 0;   // rounds of the items finished so far (the Q slot of round r is stage (R + r) & 1)
     uint32_t xn = 0;  // completed phases of this row pair's exchange barrier
     float* my_slot = &s.xchg[x][ch][0][rl];  // slot k is my_slot[128 * k]
     const float* partner_slot = &s.xchg[x][ch ^ 1][0][rl];
@@ -313,7 +352,25 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
         tmem_wait_ld();
         tc_fence_before_sync();
         mbar_arrive(&s.bar_o_free[x]);  // the next round's PV may overwrite O_x
-        if (valid) {
+        if (c.len >= kBM) {
+          // a full tile: the rows go to the Q slot of this round and half, swizzled like an operand tile (written from
+          // the threads, a row per lane 8 KB apart and 16 bytes per store, every store is half a sector of the
+          // store path: 4,096 clocks per pair of tiles)
+          uint8_t* const srow = s.q[(R + r) & 1][x][D == 128 ? ch : 0] + rl * 128;
+#pragma unroll
+          for (int cc = 0; cc < kOCols / 32; ++cc)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              uint4 w;
+              w.x = pack_bf16x2(__uint_as_float(orow[cc][8 * e + 0]) * inv_l, __uint_as_float(orow[cc][8 * e + 1]) * inv_l);
+              w.y = pack_bf16x2(__uint_as_float(orow[cc][8 * e + 2]) * inv_l, __uint_as_float(orow[cc][8 * e + 3]) * inv_l);
+              w.z = pack_bf16x2(__uint_as_float(orow[cc][8 * e + 4]) * inv_l, __uint_as_float(orow[cc][8 * e + 5]) * inv_l);
+              w.w = pack_bf16x2(__uint_as_float(orow[cc][8 * e + 6]) * inv_l, __uint_as_float(orow[cc][8 * e + 7]) * inv_l);
+              const int chunk = (D == 128 ? 0 : ch * 4) + cc * 4 + e;  // 16-byte chunk of the 128-byte row
+              *reinterpret_cast<uint4*>(srow + ((chunk ^ (rl & 7)) * 16)) = w;
+            }
+          fence_proxy_async_smem();
+        } else if (valid) {
 #pragma unroll
           for (int cc = 0; cc < kOCols / 32; ++cc)
 #pragma unroll
@@ -326,6 +383,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
               NSP_CHECK(optr + cc * 32 + e * 8 + 8 <= a.o + a.q_elems && optr >= a.o, a.status, c.it, kWhereCheckFwdO, rl)
               *reinterpret_cast<uint4*>(optr + cc * 32 + e * 8) = w;
             }
+        }
+        mbar_arrive(&s.bar_o_staged[x]);  // the store warp sends the tile off (or just hands the slot back)
+        if (valid) {
           if (ch == 0) {
             const int64_t at = c.lse_off + static_cast<int64_t>(h) * c.len + rl;
             NSP_CHECK(at >= 0 && at < a.lse_elems, a.status, c.it, kWhereCheckFwdLse, rl)
@@ -337,6 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
         report_timeout(a.status, c.it, where, x);
         *abort_flag = 1;
       }
+      R += static_cast<uint32_t>(c.rounds);
       ++gi;
     }
   }
