@@ -162,6 +162,29 @@ int nsp_attn_bwd_static(const nsp_plan_t* plan, const void* q, const void* k, co
                         float softmax_scale, void* stream);
 
 /*
+ * One forward + backward pass with HOST buffers (paper Sec. 4.1.2: T^comp,fwd + T^comp,bwd of this GPU's chain, as a
+ * caller sees it whose tensors live in host memory): nsp_attn_fwd followed by nsp_attn_bwd on device copies that this
+ * call makes and reads back.
+ * h_q, h_do [q_elems] bf16, h_k, h_v [kv_elems] bf16: host, read. h_o [q_elems] bf16, h_lse [lse_elems] fp32, h_dq
+ * [q_elems] in dq_dtype, h_dk / h_dv [kv_elems] in dkv_dtype: host, written. Pinned (page-locked) host memory lets
+ * the copies run asynchronously; with pageable memory they still work but the call blocks while they are staged.
+ * dev_ws: device memory of at least nsp_plan_step_host_ws_bytes(plan, dq_dtype, dkv_dtype) bytes, 256-byte aligned,
+ * owned by the caller: it holds the nine device tensors and the backward workspace; contents undefined afterwards.
+ * The copies run on a second stream owned by the plan (created, with six events, at the first call on the plan: make
+ * that call outside any stream capture), ordered with events against `stream`: dO travels to the device while the
+ * forward pass runs, O and LSE travel back while the backward pass runs; exposed are the copies of Q, K, V before the
+ * forward pass and of dQ, dK, dV after the backward pass. The call returns without waiting; the host outputs are
+ * complete once `stream` has passed everything this call enqueued on it (synchronise `stream`), and the host inputs
+ * must stay unchanged until then. Two calls on the same plan must not overlap from different host threads.
+ * Errors: INVALID_ARG (null pointer, dtype), WORKSPACE (dev_ws missing, misaligned or too small), CUDA,
+ * DEVICE_TIMEOUT (sticky status), and whatever nsp_attn_fwd / nsp_attn_bwd return.
+ */
+int nsp_plan_step_host_ws_bytes(const nsp_plan_t* plan, int dq_dtype, int dkv_dtype, size_t* bytes);
+int nsp_attn_step_host(nsp_plan_t* plan, const void* h_q, const void* h_k, const void* h_v, const void* h_do, void* h_o,
+                       float* h_lse, void* h_dq, void* h_dk, void* h_dv, int dq_dtype, int dkv_dtype,
+                       float softmax_scale, void* dev_ws, size_t dev_ws_bytes, void* stream);
+
+/*
  * Tree-level recomputation (paper Sec. 4.2.2 "Tree-Level Recomputation"): the backward pass of a shard in which the
  * attention output of some segments was not kept after the forward pass.
  *

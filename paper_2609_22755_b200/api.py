@@ -2,9 +2,8 @@
 forward + backward of the local attention compute phase through the C ABI.
 
 Only marshalling lives here. ``step_device`` runs on tensors already resident on the GPU; ``step_host`` is the
-end-to-end call: it copies Q, K, V, dO from (pinned) host tensors, runs forward and backward, and copies
-O, LSE, dQ, dK, dV back to host tensors; the copies run on a second stream under the kernels where the data
-dependencies allow.
+end-to-end call (nsp_attn_step_host): Q, K, V, dO come from (pinned) host tensors and O, LSE, dQ, dK, dV go back to
+host tensors; the library makes the copies on a second stream under the kernels where the data dependencies allow.
 """
 from __future__ import annotations
 
@@ -74,45 +73,19 @@ class NspAttention:
         self.backward()
 
     def step_host(self, host_in, host_out):
-        """End to end: host tensors in, host tensors out. The copies run on a second stream, ordered with events, so
-        that dO travels to the device while the forward pass runs and O / LSE travel back while the backward pass
-        runs; what stays exposed is the copy of Q, K, V before the forward and of dQ, dK, dV after the backward.
+        """End to end: host tensors in (dict with q, k, v, do), host tensors out (dict with o, lse, dq, dk, dv), through
+        the library's host-buffer entry point nsp_attn_step_host: the copies run on the plan's second stream, so that
+        dO travels to the device while the forward pass runs and O / LSE travel back while the backward pass runs.
+        The device copies live in a workspace of this object's own (not in the tensors step_device uses).
         Returns (host-to-device bytes, device-to-host bytes). The call returns without waiting for the device."""
-        torch = self.torch
-        comp = torch.cuda.current_stream() if self.stream is None else self.stream
-        if getattr(self, "_copy_stream", None) is None:
-            self._copy_stream = torch.cuda.Stream(device=self.dev)
-        cp = self._copy_stream
-        size = lambda t: t.numel() * t.element_size()
-        cp.wait_stream(comp)  # the buffers of the previous step are free
-        with torch.cuda.stream(cp):
-            for name, dst in (("q", self.q), ("k", self.k), ("v", self.v)):
-                dst.copy_(host_in[name], non_blocking=True)
-            qkv_in = torch.cuda.Event()
-            qkv_in.record(cp)
-            self.do.copy_(host_in["do"], non_blocking=True)
-            do_in = torch.cuda.Event()
-            do_in.record(cp)
-        comp.wait_event(qkv_in)
-        self.forward()
-        fwd_done = torch.cuda.Event()
-        fwd_done.record(comp)
-        with torch.cuda.stream(cp):
-            cp.wait_event(fwd_done)
-            host_out["o"].copy_(self.o, non_blocking=True)
-            host_out["lse"].copy_(self.lse, non_blocking=True)
-        comp.wait_event(do_in)
-        self.backward()
-        bwd_done = torch.cuda.Event()
-        bwd_done.record(comp)
-        with torch.cuda.stream(cp):
-            cp.wait_event(bwd_done)
-            for name, src in (("dq", self.dq), ("dk", self.dk), ("dv", self.dv)):
-                host_out[name].copy_(src, non_blocking=True)
-        comp.wait_stream(cp)  # the step is complete on the caller's stream once the last copy is
-        h2d = sum(size(host_in[n]) for n in ("q", "k", "v", "do"))
-        d2h = sum(size(t) for t in (self.o, self.lse, self.dq, self.dk, self.dv))
-        return h2d, d2h
+        if getattr(self, "_host_ws", None) is None:
+            dq_dt = B.NSP_F32 if host_out["dq"].dtype == self.torch.float32 else B.NSP_BF16
+            dkv_dt = B.NSP_F32 if host_out["dk"].dtype == self.torch.float32 else B.NSP_BF16
+            need = B.nsp_plan_step_host_ws_bytes(self.plan, dq_dt, dkv_dt)
+            self._host_ws = self.torch.empty(max(need, 256), dtype=self.torch.uint8, device=self.dev)
+        return B.nsp_attn_step_host(self.plan, host_in["q"], host_in["k"], host_in["v"], host_in["do"], host_out["o"],
+                                    host_out["lse"], host_out["dq"], host_out["dk"], host_out["dv"], self.scale,
+                                    self._host_ws, stream=self.stream)
 
     def status(self):
         return B.nsp_device_status(self.plan)

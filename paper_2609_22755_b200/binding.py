@@ -31,6 +31,7 @@ EXPORTS = [
     "nsp_attn_bwd_static", "nsp_recompute_mark", "nsp_plan_recompute_ws_bytes", "nsp_attn_bwd_recompute",
     "nsp_cost_table", "nsp_route_sp_tree", "nsp_a2a_gather_heads", "nsp_a2a_scatter_heads",
     "nsp_selftest_wait_timeout", "nsp_a2a_gather_heads_to", "nsp_plan_set_wait_limit",
+    "nsp_plan_step_host_ws_bytes", "nsp_attn_step_host",
 ]
 CHECKED_EXPORTS = ["nsp_checked_withhold_load"]  # libnsp_checked.so only
 NSP_COST_BUCKETS = 16
@@ -99,6 +100,10 @@ def lib() -> ctypes.CDLL:
         L.nsp_a2a_gather_heads_to.argtypes = [vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
                                               ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
         L.nsp_a2a_gather_heads_to.restype = ctypes.c_int
+        L.nsp_plan_step_host_ws_bytes.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_size_t)]
+        L.nsp_plan_step_host_ws_bytes.restype = ctypes.c_int
+        L.nsp_attn_step_host.argtypes = [vp] * 10 + [ctypes.c_int, ctypes.c_int, ctypes.c_float, vp, ctypes.c_size_t, vp]
+        L.nsp_attn_step_host.restype = ctypes.c_int
         L.nsp_plan_set_wait_limit.argtypes = [vp, ctypes.c_int64]
         L.nsp_plan_set_wait_limit.restype = ctypes.c_int
         if hasattr(L, "nsp_checked_withhold_load"):
@@ -284,6 +289,43 @@ def nsp_attn_bwd(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, softmax_scale, ws
                             _stream_ptr(stream))
     if rc != NSP_OK:
         raise NspError(rc, "nsp_attn_bwd")
+
+
+def nsp_plan_step_host_ws_bytes(plan: Plan, dq_dtype=NSP_BF16, dkv_dtype=NSP_F32) -> int:
+    n = ctypes.c_size_t()
+    rc = lib().nsp_plan_step_host_ws_bytes(plan.handle, int(dq_dtype), int(dkv_dtype), ctypes.byref(n))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_plan_step_host_ws_bytes")
+    return int(n.value)
+
+
+def nsp_attn_step_host(plan: Plan, h_q, h_k, h_v, h_do, h_o, h_lse, h_dq, h_dk, h_dv, softmax_scale, dev_ws, stream=None):
+    """Forward + backward with host tensors in and out (CPU torch tensors, pinned for asynchronous copies); dev_ws is
+    a CUDA uint8 tensor of at least nsp_plan_step_host_ws_bytes. Returns (host-to-device, device-to-host) bytes."""
+    import torch
+
+    bf, f32 = (torch.bfloat16,), (torch.float32,)
+    dq_dtype = NSP_F32 if h_dq.dtype == torch.float32 else NSP_BF16
+    dkv_dtype = NSP_F32 if h_dk.dtype == torch.float32 else NSP_BF16
+    specs = [("h_q", h_q, bf, plan.q_elems), ("h_k", h_k, bf, plan.kv_elems), ("h_v", h_v, bf, plan.kv_elems),
+             ("h_do", h_do, bf, plan.q_elems), ("h_o", h_o, bf, plan.q_elems), ("h_lse", h_lse, f32, plan.lse_elems),
+             ("h_dq", h_dq, f32 + bf, plan.q_elems), ("h_dk", h_dk, f32 + bf, plan.kv_elems),
+             ("h_dv", h_dv, (h_dk.dtype,), plan.kv_elems)]
+    for name, t, dtypes, need in specs:
+        if need == 0:
+            continue
+        if not isinstance(t, torch.Tensor) or t.is_cuda or not t.is_contiguous() or t.dtype not in dtypes or t.numel() < need:
+            raise NspError(NSP_ERR_INVALID_ARG, f"nsp_attn_step_host: {name} must be a contiguous host tensor of "
+                                                f"{need} elements of {dtypes}")
+    _check_ws("nsp_attn_step_host", dev_ws)
+    ws_bytes = 0 if dev_ws is None else dev_ws.numel() * dev_ws.element_size()
+    rc = lib().nsp_attn_step_host(plan.handle, _ptr(h_q), _ptr(h_k), _ptr(h_v), _ptr(h_do), _ptr(h_o), _ptr(h_lse),
+                                  _ptr(h_dq), _ptr(h_dk), _ptr(h_dv), dq_dtype, dkv_dtype, float(softmax_scale),
+                                  _ptr(dev_ws), ws_bytes, _stream_ptr(stream))
+    if rc != NSP_OK:
+        raise NspError(rc, "nsp_attn_step_host")
+    size = lambda t: t.numel() * t.element_size()
+    return (sum(size(t) for t in (h_q, h_k, h_v, h_do)), sum(size(t) for t in (h_o, h_lse, h_dq, h_dk, h_dv)))
 
 
 def nsp_recompute_mark(cu_seqlens, hq, level, budget_bytes: int, head_dim: int = 128):

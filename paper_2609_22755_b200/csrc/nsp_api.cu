@@ -49,6 +49,9 @@ struct nsp_plan {
   bool profiling = false;
   cudaEvent_t ev[2 * NSP_KERNEL_COUNT] = {};
   bool ev_valid[NSP_KERNEL_COUNT] = {};
+  // host-to-host step (nsp_attn_step_host): a copy stream and ordering events, created at its first call
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t hev[6] = {};
 };
 
 namespace {
@@ -186,6 +189,9 @@ void free_plan(nsp_plan* p) {
   if (p->h_status) cudaFreeHost(p->h_status);
   for (cudaEvent_t e : p->ev)
     if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : p->hev)
+    if (e) cudaEventDestroy(e);
+  if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
   delete p;
 }
 
@@ -640,6 +646,99 @@ int nsp_attn_bwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
                  void* ws, size_t ws_bytes, void* stream) {
   return bwd_impl(plan, nullptr, q, k, v, o, d_o, lse, dq, dk, dv, dq_dtype, dkv_dtype, softmax_scale, ws, ws_bytes,
                   stream);
+}
+
+namespace {
+
+// Device layout of the host-to-host step's workspace: the nine packed tensors, then the backward workspace.
+struct HostStepLayout {
+  size_t q, k, v, d_o, o, lse, dq, dk, dv, bwd_ws, total;
+  size_t q_bytes, kv_bytes, lse_bytes, dq_bytes, dkv_bytes, bwd_ws_bytes;
+};
+
+bool host_step_layout(const nsp_plan_t* plan, int dq_dtype, int dkv_dtype, HostStepLayout* L) {
+  if ((dq_dtype != NSP_BF16 && dq_dtype != NSP_F32) || (dkv_dtype != NSP_BF16 && dkv_dtype != NSP_F32)) return false;
+  size_t bwd_ws = 0;
+  nsp_plan_sizes(plan, nullptr, nullptr, nullptr, nullptr, &bwd_ws);
+  L->q_bytes = static_cast<size_t>(plan->q_elems) * 2;
+  L->kv_bytes = static_cast<size_t>(plan->kv_elems) * 2;
+  L->lse_bytes = static_cast<size_t>(plan->lse_elems) * 4;
+  L->dq_bytes = static_cast<size_t>(plan->q_elems) * (dq_dtype == NSP_F32 ? 4 : 2);
+  L->dkv_bytes = static_cast<size_t>(plan->kv_elems) * (dkv_dtype == NSP_F32 ? 4 : 2);
+  L->bwd_ws_bytes = bwd_ws;
+  size_t at = 0;
+  auto take = [&](size_t bytes) {
+    const size_t here = at;
+    at += align_up(bytes > 0 ? bytes : 1, 256);
+    return here;
+  };
+  L->q = take(L->q_bytes), L->k = take(L->kv_bytes), L->v = take(L->kv_bytes), L->d_o = take(L->q_bytes);
+  L->o = take(L->q_bytes), L->lse = take(L->lse_bytes);
+  L->dq = take(L->dq_bytes), L->dk = take(L->dkv_bytes), L->dv = take(L->dkv_bytes);
+  L->bwd_ws = take(bwd_ws);
+  L->total = at;
+  return true;
+}
+
+}  // namespace
+
+int nsp_plan_step_host_ws_bytes(const nsp_plan_t* plan, int dq_dtype, int dkv_dtype, size_t* bytes) {
+  if (!plan || !bytes) return NSP_ERR_INVALID_ARG;
+  HostStepLayout L;
+  if (!host_step_layout(plan, dq_dtype, dkv_dtype, &L)) return NSP_ERR_INVALID_ARG;
+  *bytes = L.total;
+  return NSP_OK;
+}
+
+int nsp_attn_step_host(nsp_plan_t* plan, const void* h_q, const void* h_k, const void* h_v, const void* h_do, void* h_o,
+                       float* h_lse, void* h_dq, void* h_dk, void* h_dv, int dq_dtype, int dkv_dtype,
+                       float softmax_scale, void* dev_ws, size_t dev_ws_bytes, void* stream) {
+  if (!plan) return NSP_ERR_INVALID_ARG;
+  if (const int failed = plan_failed(plan)) return failed;
+  HostStepLayout L;
+  if (!host_step_layout(plan, dq_dtype, dkv_dtype, &L)) return NSP_ERR_INVALID_ARG;
+  if (plan->n_fwd == 0) return NSP_OK;
+  if (!h_q || !h_k || !h_v || !h_do || !h_o || !h_lse || !h_dq || !h_dk || !h_dv) return NSP_ERR_INVALID_ARG;
+  if (!dev_ws || (reinterpret_cast<uintptr_t>(dev_ws) & 255) != 0 || dev_ws_bytes < L.total) return NSP_ERR_WORKSPACE;
+  if (!plan->copy_stream) {
+    if (cudaStreamCreateWithFlags(&plan->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return NSP_ERR_CUDA;
+    for (cudaEvent_t& e : plan->hev)
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return NSP_ERR_CUDA;
+  }
+  cudaStream_t comp = static_cast<cudaStream_t>(stream), cp = plan->copy_stream;
+  char* base = static_cast<char*>(dev_ws);
+  enum { kFree = 0, kQkvIn, kDoIn, kFwdDone, kBwdDone, kAllOut };
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+  const cudaMemcpyKind in = cudaMemcpyHostToDevice, out = cudaMemcpyDeviceToHost;
+  NSP_LOGF("host step plan %p stream %p: %zu bytes in, %zu bytes out", static_cast<const void*>(plan), stream,
+           2 * L.q_bytes + 2 * L.kv_bytes, L.q_bytes + L.lse_bytes + L.dq_bytes + 2 * L.dkv_bytes);
+  // the device buffers are free once everything enqueued on the caller's stream so far has run
+  if (!ok(cudaEventRecord(plan->hev[kFree], comp)) || !ok(cudaStreamWaitEvent(cp, plan->hev[kFree], 0))) return NSP_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(base + L.q, h_q, L.q_bytes, in, cp)) || !ok(cudaMemcpyAsync(base + L.k, h_k, L.kv_bytes, in, cp)) ||
+      !ok(cudaMemcpyAsync(base + L.v, h_v, L.kv_bytes, in, cp)) || !ok(cudaEventRecord(plan->hev[kQkvIn], cp)))
+    return NSP_ERR_CUDA;
+  // dO travels in under the forward pass
+  if (!ok(cudaMemcpyAsync(base + L.d_o, h_do, L.q_bytes, in, cp)) || !ok(cudaEventRecord(plan->hev[kDoIn], cp)))
+    return NSP_ERR_CUDA;
+  if (!ok(cudaStreamWaitEvent(comp, plan->hev[kQkvIn], 0))) return NSP_ERR_CUDA;
+  int rc = nsp_attn_fwd(plan, base + L.q, base + L.k, base + L.v, base + L.o, reinterpret_cast<float*>(base + L.lse),
+                        softmax_scale, nullptr, 0, stream);
+  if (rc != NSP_OK) return rc;
+  // O and LSE travel out under the backward pass
+  if (!ok(cudaEventRecord(plan->hev[kFwdDone], comp)) || !ok(cudaStreamWaitEvent(cp, plan->hev[kFwdDone], 0)) ||
+      !ok(cudaMemcpyAsync(h_o, base + L.o, L.q_bytes, out, cp)) || !ok(cudaMemcpyAsync(h_lse, base + L.lse, L.lse_bytes, out, cp)))
+    return NSP_ERR_CUDA;
+  if (!ok(cudaStreamWaitEvent(comp, plan->hev[kDoIn], 0))) return NSP_ERR_CUDA;
+  rc = nsp_attn_bwd(plan, base + L.q, base + L.k, base + L.v, base + L.o, base + L.d_o,
+                    reinterpret_cast<const float*>(base + L.lse), base + L.dq, base + L.dk, base + L.dv, dq_dtype, dkv_dtype,
+                    softmax_scale, base + L.bwd_ws, L.bwd_ws_bytes, stream);
+  if (rc != NSP_OK) return rc;
+  if (!ok(cudaEventRecord(plan->hev[kBwdDone], comp)) || !ok(cudaStreamWaitEvent(cp, plan->hev[kBwdDone], 0)) ||
+      !ok(cudaMemcpyAsync(h_dq, base + L.dq, L.dq_bytes, out, cp)) || !ok(cudaMemcpyAsync(h_dk, base + L.dk, L.dkv_bytes, out, cp)) ||
+      !ok(cudaMemcpyAsync(h_dv, base + L.dv, L.dkv_bytes, out, cp)) || !ok(cudaEventRecord(plan->hev[kAllOut], cp)) ||
+      !ok(cudaStreamWaitEvent(comp, plan->hev[kAllOut], 0)))  // the step is complete on the caller's stream
+    return NSP_ERR_CUDA;
+  return NSP_OK;
 }
 
 int nsp_plan_recompute_ws_bytes(const nsp_plan_t* plan, size_t* bytes) {

@@ -102,6 +102,10 @@ def test_null_plan_is_rejected(B):
     assert L.nsp_attn_fwd(None, None, None, None, None, None, 1.0, None, 0, None) == B.NSP_ERR_INVALID_ARG
     assert L.nsp_attn_bwd(None, None, None, None, None, None, None, None, None, None, 0, 1, 1.0, None, 0,
                           None) == B.NSP_ERR_INVALID_ARG
+    n = ctypes.c_size_t()
+    assert L.nsp_plan_step_host_ws_bytes(None, 0, 1, ctypes.byref(n)) == B.NSP_ERR_INVALID_ARG
+    assert L.nsp_attn_step_host(None, None, None, None, None, None, None, None, None, None, 0, 1, 1.0, None, 0,
+                                None) == B.NSP_ERR_INVALID_ARG
     assert L.nsp_plan_destroy(None) == B.NSP_OK
     assert L.nsp_launch_count() >= 0
 

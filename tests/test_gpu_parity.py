@@ -194,7 +194,8 @@ def test_backward_with_recomputation(env, case, which):
 
 
 def test_host_to_host_step_equals_the_device_step(env):
-    """The end-to-end call (pinned host tensors in and out, copies on a second stream under the kernels) returns what
+    """The end-to-end call (nsp_attn_step_host through the C ABI: pinned host tensors in and out, device copies in a
+    workspace of its own, the copies on the plan's second stream under the kernels) returns what
     the device-resident step leaves in the device buffers: O, LSE, dK, dV bit for bit, dQ (bf16, from the fp32
     accumulator) within one rounding of the fp32 sum. Two steps in a row, to cover the reuse of the buffers."""
     torch, W = env["torch"], env["W"]
