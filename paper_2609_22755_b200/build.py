@@ -1,6 +1,6 @@
 """Build ``libnsp.so`` (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-``python -m paper_2609_22755_b200.build`` compiles every ``csrc/*.cu`` to an object file (in parallel) and links
+``python -m paper_2609_22755_b200.build`` compiles every ``csrc/*.cu`` (and the host-only ``csrc/*.cpp``) to an object file (in parallel) and links
 them into ``paper_2609_22755_b200/libnsp.so`` with the CUDA runtime linked statically, so the library loads on a
 machine without a GPU driver (the driver entry point it needs is resolved at run time).
 """
@@ -46,7 +46,7 @@ def build_library(force: bool = False, verbose: bool = False, checked: bool = Fa
     """Build libnsp.so, or with checked=True libnsp_checked.so (kernels verify every index they compute; for tests)."""
     nvcc = _nvcc()
     lib, tag, extra = (LIB_CHECKED, "_checked", ["-DNSP_CHECKED"]) if checked else (LIB, "", [])
-    sources = sorted(CSRC.glob("*.cu"))
+    sources = sorted(CSRC.glob("*.cu")) + sorted(CSRC.glob("*.cpp"))  # the planner is host-only C++
     headers = sorted(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "nsp.h"]
     OBJ_DIR.mkdir(exist_ok=True)
 
