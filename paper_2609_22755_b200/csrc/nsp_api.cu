@@ -31,8 +31,10 @@ struct nsp_plan {
   nsp_tile_t* d_fwd = nullptr;
   nsp_tile_t* d_bwd = nullptr;
   nsp_tile_t* d_bwd_exec = nullptr;  // the backward items in the order the kernel walks them (see build_bwd_exec_order)
-  nsp_tile_t* d_bwd_first = nullptr;  // one item per (segment, kv head): the first-tile kernel's list
+  nsp_tile_t* d_bwd_first = nullptr;  // one item per (segment or pack, kv head): the first-tile kernels' list
   int64_t n_first = 0;
+  RowInfo* d_rows = nullptr;          // row tables of the packs, 128 entries each (d_seg holds the packs' entries after
+  int64_t n_packs = 0;                // the n_seg segments')
   int64_t n_fwd_main = 0;             // forward items that visit at least two key tiles: a prefix of d_fwd (the
                                       // cost-1 tail = q tile 0 of every segment runs in the first-tile forward kernel)
   bool deterministic = false;         // plan option: dQ tiles added in key-tile order
@@ -183,6 +185,7 @@ void free_plan(nsp_plan* p) {
   cudaFree(p->d_bwd);
   cudaFree(p->d_bwd_exec);
   cudaFree(p->d_bwd_first);
+  cudaFree(p->d_rows);
   cudaFree(p->d_front);
   cudaFree(p->d_counters);
   cudaFree(p->d_status);
@@ -315,11 +318,62 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
   }
 
   std::vector<nsp_tile_t> bwd_exec, bwd_first;
+  std::vector<SegInfo> pack_segs;
+  std::vector<RowInfo> pack_rows;
   try {
     bwd_exec = build_bwd_exec_order(p->seg, bm, bn);
     // the first-tile kernel's items: key tile 0 of every group, in the same group order; q heads of the group = steps
-    for (const nsp_tile_t& t : bwd_exec)
-      if (t.tile == 0) bwd_first.push_back(nsp_tile_t{t.seg, t.head, 0, p->seg[t.seg].hq / p->seg[t.seg].hkv});
+    // Segments of fewer than 128 tokens that follow one another inside a run (they are contiguous in every tensor)
+    // and together hold at most 128 tokens share one first tile: such a pack becomes an entry of its own behind the
+    // segments (len = its tokens, offsets of its first segment) with a row table, and takes its segments' places in
+    // the first-tile list.
+    std::vector<int32_t> pack_of(n_seg, -1);
+    for (int s0 = 0; s0 < n_seg;) {
+      const SegInfo& first = p->seg[s0];
+      if (first.len <= 0 || first.len >= kBM) { ++s0; continue; }
+      int s1 = s0 + 1, tokens = first.len, members = 1;
+      while (s1 < n_seg && p->seg[s1].run == first.run && p->seg[s1].len < kBM && tokens + p->seg[s1].len <= kBM) {
+        tokens += p->seg[s1].len;
+        members += p->seg[s1].len > 0;
+        ++s1;
+      }
+      if (members >= 2) {
+        SegInfo pk = first;
+        pk.len = tokens;
+        pk.rows = static_cast<int32_t>(pack_rows.size() / kBM) + 1;
+        int row = 0;
+        for (int s = s0; s < s1; ++s) {
+          const SegInfo& sg = p->seg[s];
+          if (sg.len <= 0) continue;
+          pack_of[s] = n_seg + static_cast<int32_t>(pack_segs.size());
+          RowInfo ri{};
+          ri.lse_base = sg.lse_off - row;
+          ri.len = sg.len;
+          ri.lo = static_cast<uint8_t>(row);
+          ri.hi = static_cast<uint8_t>(row + sg.len);
+          for (int i = 0; i < sg.len; ++i) pack_rows.push_back(ri);
+          row += sg.len;
+        }
+        pack_rows.resize(pack_rows.size() + (kBM - tokens), RowInfo{});
+        pack_segs.push_back(pk);
+      }
+      s0 = s1;
+    }
+    p->n_packs = static_cast<int64_t>(pack_segs.size());
+    {
+      std::vector<char> listed(pack_segs.size() * 256, 0);  // (pack, kv head) already in the list
+      for (const nsp_tile_t& t : bwd_exec) {
+        if (t.tile != 0) continue;
+        const int32_t G = p->seg[t.seg].hq / p->seg[t.seg].hkv;
+        if (pack_of[t.seg] < 0) {
+          bwd_first.push_back(nsp_tile_t{t.seg, t.head, 0, G});
+        } else {
+          char& seen = listed[static_cast<size_t>(pack_of[t.seg] - n_seg) * 256 + t.head];
+          if (!seen) bwd_first.push_back(nsp_tile_t{pack_of[t.seg], t.head, 0, G});
+          seen = 1;
+        }
+      }
+    }
     p->n_first = static_cast<int64_t>(bwd_first.size());
     p->n_fwd_main = nf;
     for (const SegInfo& sg : p->seg)
@@ -350,7 +404,8 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
   auto A = [&](void** ptr, size_t bytes) {
     if (okc && cudaMalloc(ptr, bytes ? bytes : 16) != cudaSuccess) okc = false;
   };
-  A(reinterpret_cast<void**>(&p->d_seg), sizeof(SegInfo) * n_seg);
+  A(reinterpret_cast<void**>(&p->d_seg), sizeof(SegInfo) * (n_seg + pack_segs.size()));
+  A(reinterpret_cast<void**>(&p->d_rows), sizeof(RowInfo) * pack_rows.size());
   A(reinterpret_cast<void**>(&p->d_row_base), sizeof(int64_t) * (n_seg + 1));
   A(reinterpret_cast<void**>(&p->d_fwd), sizeof(nsp_tile_t) * nf);
   A(reinterpret_cast<void**>(&p->d_bwd), sizeof(nsp_tile_t) * nb);
@@ -392,6 +447,10 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
                         st));
     }
     C(cudaMemcpyAsync(p->d_row_base, row_base.data(), sizeof(int64_t) * (n_seg + 1), cudaMemcpyHostToDevice, st));
+    if (!pack_segs.empty()) {
+      C(cudaMemcpyAsync(p->d_seg + n_seg, pack_segs.data(), sizeof(SegInfo) * pack_segs.size(), cudaMemcpyHostToDevice, st));
+      C(cudaMemcpyAsync(p->d_rows, pack_rows.data(), sizeof(RowInfo) * pack_rows.size(), cudaMemcpyHostToDevice, st));
+    }
     if (nb > 0) C(cudaMemcpyAsync(p->d_bwd_exec, bwd_exec.data(), sizeof(nsp_tile_t) * nb, cudaMemcpyHostToDevice, st));
     if (p->n_first > 0)
       C(cudaMemcpyAsync(p->d_bwd_first, bwd_first.data(), sizeof(nsp_tile_t) * p->n_first, cudaMemcpyHostToDevice, st));
@@ -478,6 +537,7 @@ int nsp_attn_fwd(const nsp_plan_t* plan, const void* q, const void* k, const voi
   a.q_elems = plan->q_elems;
   a.lse_elems = plan->lse_elems;
   a.seg_mask = nullptr;
+  a.rows = plan->d_rows;
   a.d_o = nullptr;
   a.delta = nullptr;
   NSP_LOGF("fwd plan %p stream %p scale %g", static_cast<const void*>(plan), stream, softmax_scale);
@@ -575,6 +635,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
     fa.q_elems = plan->q_elems;
     fa.lse_elems = plan->lse_elems;
     fa.seg_mask = d_mask;
+    fa.rows = plan->d_rows;
     fa.d_o = static_cast<const __nv_bfloat16*>(d_o);
     fa.delta = delta;
     prof_mark(plan, NSP_KERNEL_FWD, 0, st);
@@ -608,6 +669,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   a.dq_f32 = dq_dtype == NSP_F32;
   a.dq_turn = dq_turn;
   a.front = plan->d_front;
+  a.rows = plan->d_rows;
   a.dk = dk;
   a.dv = dv;
   a.dkv_f32 = dkv_dtype == NSP_F32;

@@ -71,6 +71,7 @@ struct ItemCtx {
   int32_t m0;                      // first (lowest) q tile of the walk
   int32_t per_head;                // steps per q head
   int32_t steps;                   // G * per_head
+  int32_t rows;                    // first-tile kernel: 0, or 1 + index of the row table of a pack of short segments
 };
 
 // FIRST: the first-tile kernel also keeps the bf16 residual of dS^T. The main kernel does without those 32 KB on
@@ -247,6 +248,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       x.G = sg.hq / sg.hkv;
       x.turn_off = sg.turn_off, x.mt = (sg.len + kBM - 1) / kBM;
       x.first = (item.tile == 0);
+      x.rows = sg.rows;
       if constexpr (FIRST) {
         x.m0 = 0;
         x.per_head = 1;  // q tile 0 only
@@ -524,9 +526,16 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             const bool valid = qi < c.len;
             float lv = INFINITY, dv_ = 0.f;
             if (valid) {
-              NSP_CHECK(base + qi >= 0 && base + qi < a.lse_elems, a.status, c.it, kWhereCheckBwdLse, qi) {
-                lv = a.lse[base + qi] * kLog2e;
-                dv_ = a.delta[base + qi];
+              int64_t at = base + qi;
+              if constexpr (FIRST) {
+                if (c.rows > 0) {  // a tile shared by several short segments: LSE is laid out per segment
+                  const RowInfo ri = a.rows[static_cast<int64_t>(c.rows - 1) * kBM + col];
+                  at = ri.lse_base + static_cast<int64_t>(h) * ri.len + col;
+                }
+              }
+              NSP_CHECK(at >= 0 && at < a.lse_elems, a.status, c.it, kWhereCheckBwdLse, qi) {
+                lv = a.lse[at] * kLog2e;
+                dv_ = a.delta[at];
               }
             }
             s.lse[st][col] = lv;
@@ -720,6 +729,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       const ItemCtx c = *cx;
       bool oks = true;
       int where = 0;
+      // first-tile kernel, a tile shared by several short segments: key row r is seen by the queries r .. r_end - 1
+      // (the rest of its own segment); a tile of one segment: every query from r on
+      int r_end = kBM;
+      if constexpr (FIRST) {
+        if (c.rows > 0) r_end = a.rows[static_cast<int64_t>(c.rows - 1) * kBM + r].hi;
+      }
       StepWalk w;
       w.reset();
 #pragma unroll 1
@@ -880,8 +895,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
                 const float lse0 = (x & 2) ? l4[x >> 2].z : l4[x >> 2].x, lse1 = (x & 2) ? l4[x >> 2].w : l4[x >> 2].y;
                 float p0 = ex2f(fmaf(__uint_as_float(sv[x + 0]), a.scale_log2, -lse0));
                 float p1 = ex2f(fmaf(__uint_as_float(sv[x + 1]), a.scale_log2, -lse1));
-                if (half * 64 + ch * 16 + x + 0 < r) p0 = 0.f;  // query index must be >= key index
-                if (half * 64 + ch * 16 + x + 1 < r) p1 = 0.f;
+                const int qc = half * 64 + ch * 16 + x;
+                if (qc + 0 < r || qc + 0 >= r_end) p0 = 0.f;  // query index must be >= key index, inside its segment
+                if (qc + 1 < r || qc + 1 >= r_end) p1 = 0.f;
                 v[x + 0] = p0 * __uint_as_float(dpv[x + 0]);
                 v[x + 1] = p1 * __uint_as_float(dpv[x + 1]);
                 const uint32_t pa = pack_bf16x2(p0, p1);

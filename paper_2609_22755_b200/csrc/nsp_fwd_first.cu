@@ -33,6 +33,7 @@ struct FirstCtx {
   int64_t q_off, lse_off;
   int32_t it;  // position in the list (>= n_items: no more work)
   int32_t len, hq, G, g, run, tok0, rounds;
+  int32_t rows;  // 0, or 1 + index of the row table of a pack of short segments (see RowInfo)
 };
 
 template <int D>
@@ -120,6 +121,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
       x.q_off = sg.q_off, x.lse_off = sg.lse_off;
       x.len = sg.len, x.hq = sg.hq, x.G = sg.hq / sg.hkv, x.g = item.head, x.run = sg.run, x.tok0 = sg.tok_in_run;
       x.rounds = (x.G + 1) / 2;
+      x.rows = sg.rows;
     }
   };
   auto next_item = [&]() -> bool {
@@ -283,6 +285,15 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
     while (next_item()) {
       bool ok = true;
       int where = 0;
+      // A tile shared by several short segments: row rl belongs to the segment that covers rows [lo, hi) of the tile and
+      // sees the keys lo .. rl; its LSE element for head h is lse_row + h * lse_len. A tile of one segment: lo = 0.
+      int lo = 0;
+      int64_t lse_row = c.lse_off + rl;
+      int lse_len = c.len;
+      if (c.rows > 0) {
+        const RowInfo ri = a.rows[static_cast<int64_t>(c.rows - 1) * kBM + rl];
+        lo = ri.lo, lse_row = ri.lse_base + rl, lse_len = ri.len;
+      }
       for (int r = 0; r < c.rounds; ++r) {
         if (x == 1 && 2 * r + 1 >= c.G) break;  // an odd group's last head runs alone, as half A
         if (*abort_flag) { ok = false; break; }
@@ -301,8 +312,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
         for (int cc = 0; cc < 2; ++cc)
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            if (ch * 64 + cc * 32 + e > rl) sr[cc][e] = __float_as_uint(-INFINITY);
-            if (ch * 64 + cc * 32 + e + 1 > rl) sr[cc][e + 1] = __float_as_uint(-INFINITY);
+            const int col = ch * 64 + cc * 32 + e;
+            if (col > rl || col < lo) sr[cc][e] = __float_as_uint(-INFINITY);
+            if (col + 1 > rl || col + 1 < lo) sr[cc][e + 1] = __float_as_uint(-INFINITY);
             mx = ff_max3(mx, __uint_as_float(sr[cc][e]), __uint_as_float(sr[cc][e + 1]));
           }
         my_slot[0] = mx;
@@ -311,7 +323,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
         ++xn;
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { where = kWhereFwdPair; break; }
-        const float m_ref = fmaxf(mx, partner_slot[0]) * a.scale_log2;  // key 0 is never masked: finite
+        const float m_ref = fmaxf(mx, partner_slot[0]) * a.scale_log2;  // a row always sees its own key: finite
         const float neg_m = -m_ref;
         float sum0 = 0.f, sum1 = 0.f;
         uint32_t pk[32];
@@ -387,7 +399,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_first_kernel(const __grid_con
         mbar_arrive(&s.bar_o_staged[x]);  // the store warp sends the tile off (or just hands the slot back)
         if (valid) {
           if (ch == 0) {
-            const int64_t at = c.lse_off + static_cast<int64_t>(h) * c.len + rl;
+            const int64_t at = lse_row + static_cast<int64_t>(h) * lse_len;
             NSP_CHECK(at >= 0 && at < a.lse_elems, a.status, c.it, kWhereCheckFwdLse, rl)
             a.lse[at] = (m_ref + log2f(l)) * 0.6931471805599453f;
           }

@@ -23,9 +23,23 @@ struct SegInfo {
   int32_t tok_in_run;  // first token of the segment, relative to the run
   int32_t run_tokens;  // tokens of the whole run (extent of its tensor maps)
   int32_t turn_off;    // index of the segment's first (q head, q tile) turn counter (deterministic dQ): + h * Mt + m
-  int32_t pad_;
+  int32_t rows;        // 0: a segment. k > 0: a pack of several short segments that share one first tile (see
+                       // RowInfo); its row table starts at entry (k - 1) * 128 and len is the pack's token count
 };
 static_assert(sizeof(SegInfo) == 56 || sizeof(SegInfo) == 64, "SegInfo layout");
+
+// First tiles shared by several segments. Consecutive segments of a run are contiguous in Q, K, V and the outputs, so
+// segments of fewer than 128 tokens that follow one another and together hold at most 128 tokens go through the
+// first-tile kernels as ONE tile: row i of the tile belongs to the segment that covers rows [lo, hi) and sees the keys
+// lo .. i of the tile. Only LSE and delta are laid out per segment ([hq, len]): lse_base + h * len + i is the element
+// of (row i, q head h). One table of 128 entries per pack; the entries past the pack's tokens are zero.
+struct RowInfo {
+  int64_t lse_base;
+  int32_t len;
+  uint8_t lo, hi;
+  uint8_t pad_[2];
+};
+static_assert(sizeof(RowInfo) == 16, "RowInfo layout");
 
 struct RunInfo {
   int64_t q_off, kv_off;  // element offsets of the run's first token
@@ -134,6 +148,7 @@ struct FwdArgs {
   const uint8_t* seg_mask;
   const __nv_bfloat16* d_o;
   float* delta;
+  const RowInfo* rows;  // row tables of the packs (first-tile kernel)
 };
 
 struct BwdArgs {
@@ -156,6 +171,7 @@ struct BwdArgs {
   long long wait_limit;  // SM clocks a device-side wait may take before it gives up
   int64_t q_elems, kv_elems, lse_elems;  // tensor sizes (checked build)
   int32_t* front;    // [n_items / kFrontBlock + 1] arrival counters, zeroed before the launch (see next_item)
+  const RowInfo* rows;  // row tables of the packs (first-tile kernel)
 };
 
 // Host-side launchers implemented next to their kernels.

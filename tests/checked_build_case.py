@@ -26,7 +26,9 @@ assert hasattr(B.lib(), "nsp_checked_withhold_load")
 
 base = W.ragged()
 cases = [W.config(1), base, W.config(4, twin=True),
-         W.custom(base.lengths.tolist(), base.hq.tolist(), base.hkv.tolist(), seed=2, head_dim=64)]
+         W.custom(base.lengths.tolist(), base.hq.tolist(), base.hkv.tolist(), seed=2, head_dim=64),
+         # short segments that share first tiles (per-row LSE addresses)
+         W.custom([5, 60, 63, 1, 127, 2, 64, 7, 0, 9, 200, 16, 16, 16], [8] * 7 + [4] * 7, [2] * 7 + [4] * 7, seed=3)]
 for w in cases:
     run = P.GpuRun(w)
     run.forward()

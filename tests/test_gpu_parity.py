@@ -59,6 +59,26 @@ def test_ragged_tails_every_element(env):
     _full_case(env, env["W"].ragged())
 
 
+@pytest.mark.parametrize("head_dim", [128, 64])
+def test_short_segments_that_share_a_first_tile(env, head_dim):
+    """Consecutive segments of fewer than 128 tokens inside a run go through the first-tile kernels as one tile
+    (block-diagonal causal mask, per-segment LSE layout). Covered: packs of exactly 128 tokens (tile stores) and ragged
+    ones, a pack of eight segments, a zero-length segment inside a pack, a 128-token and a multi-tile segment between
+    packs, odd and unit group sizes; every element of every output against the oracle, and the published lists (which
+    know nothing of packs) unchanged."""
+    W, B, oracle = env["W"], env["B"], env["oracle"]
+    lengths = [5, 60, 63, 1, 127, 2, 64, 64] + [100, 28, 128, 30, 98] + [200, 7, 0, 9, 112] + [16] * 8 + [48, 48, 48]
+    hq = [8] * 8 + [3] * 5 + [4] * 5 + [16] * 11
+    hkv = [2] * 8 + [1] * 5 + [4] * 5 + [2] * 11
+    w = W.custom(lengths, hq, hkv, seed=21, name=f"shared_first_tiles_d{head_dim}", head_dim=head_dim)
+    errs, run, res, ref = _full_case(env, w)
+    for p_ in (0, 1, 2):
+        assert np.array_equal(B.nsp_plan_get(run.plan, p_), oracle.plan_tiles(w.cu_seqlens, w.hq, w.hkv, 128, 128, p_))
+    # uniform batches of very short segments: every tile holds 128 / L whole segments
+    for L, n in ((16, 24), (48, 9)):
+        _full_case(env, W.custom([L] * n, [8] * n, [2] * n, seed=22 + L, name=f"uniform_{L}_d{head_dim}", head_dim=head_dim))
+
+
 def test_bf16_gradients_and_fp32_dq_variants(env):
     # the dtype arguments of nsp_attn_bwd: fp32 dQ meets the tolerance; bf16 dK/dV are produced and close
     # (their output rounding alone can exceed 2e-2 where |dV| > 8, so only rel-L2 is asserted for them)
