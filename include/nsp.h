@@ -79,8 +79,15 @@ typedef struct {
  * the backward pass then adds the dQ tiles of a (segment, q head, q tile) in key-tile order (a turn counter per tile,
  * taken with the library's bounded wait), so that dQ, like O, LSE, dK and dV, comes out bit for bit the same in every
  * run and for every packing order; bwd_ws_bytes grows by 4 bytes per (q head, q tile). Without the flag the tiles
- * are added in arrival order with floating-point reductions: equal up to the rounding of an fp32 sum. */
+ * are added in arrival order with floating-point reductions: equal up to the rounding of an fp32 sum.
+ * NSP_PLAN_ROUNDED_DQ reaches the same bitwise reproducibility without any waiting: every term a key tile adds to the
+ * fp32 accumulator of dQ / softmax_scale is first rounded to a multiple of 2^-12; sums of such multiples are exact in
+ * fp32 while they stay below 4096, so the order of the additions cannot change the result. The price is accuracy with
+ * an ABSOLUTE quantum (at most 2^-13 of error per key tile and element, in units of dQ / softmax_scale): meant for
+ * gradients of order one, as in training with normalised activations; should an accumulator element pass 4096 the sum
+ * is merely no longer order-independent. Ignored when NSP_PLAN_DETERMINISTIC_DQ is set as well. */
 #define NSP_PLAN_DETERMINISTIC_DQ 1
+#define NSP_PLAN_ROUNDED_DQ 2
 typedef struct {
   int32_t bm, bn, order_version, flags;
 } nsp_plan_opts;

@@ -24,6 +24,7 @@ NSP_BF16 = 0
 NSP_F32 = 1
 NSP_MAX_RUNS = 32
 NSP_PLAN_DETERMINISTIC_DQ = 1
+NSP_PLAN_ROUNDED_DQ = 2
 
 EXPORTS = [
     "nsp_plan_tiles", "nsp_plan_sizes", "nsp_plan_get", "nsp_attn_fwd", "nsp_attn_bwd", "nsp_device_status",

@@ -38,6 +38,7 @@ struct nsp_plan {
   int64_t n_fwd_main = 0;             // forward items that visit at least two key tiles: a prefix of d_fwd (the
                                       // cost-1 tail = q tile 0 of every segment runs in the first-tile forward kernel)
   bool deterministic = false;         // plan option: dQ tiles added in key-tile order
+  bool rounded_dq = false;            // plan option: dQ terms rounded to a fixed quantum (order-independent sums)
   int32_t max_len = 0;                // longest segment: no preprocess / main / postprocess launch when <= 128
   int32_t* d_front = nullptr;        // [n_bwd / kFrontBlock + 1] start-alignment counters of the backward kernel
   int32_t* d_counters = nullptr;  // [0] forward cursor, [1] backward cursor
@@ -242,7 +243,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
     if (opts->bm <= 0 || opts->bn <= 0) return NSP_ERR_INVALID_ARG;
     bm = opts->bm;
     bn = opts->bn;
-    if (opts->order_version != 1 || (opts->flags & ~NSP_PLAN_DETERMINISTIC_DQ) != 0) return NSP_ERR_UNSUPPORTED;
+    if (opts->order_version != 1 || (opts->flags & ~(NSP_PLAN_DETERMINISTIC_DQ | NSP_PLAN_ROUNDED_DQ)) != 0) return NSP_ERR_UNSUPPORTED;
   }
   if (head_dim != 128 && head_dim != 64) return NSP_ERR_UNSUPPORTED;
   if (bm != kBM || bn != kBN) return NSP_ERR_UNSUPPORTED;
@@ -253,6 +254,7 @@ int nsp_plan_tiles(const int32_t* cu_seqlens, const int32_t* hq, const int32_t* 
   p->n_seg = n_seg;
   p->head_dim = head_dim;
   p->deterministic = opts && (opts->flags & NSP_PLAN_DETERMINISTIC_DQ) != 0;
+  p->rounded_dq = opts && !p->deterministic && (opts->flags & NSP_PLAN_ROUNDED_DQ) != 0;
   p->bm = bm;
   p->bn = bn;
   std::vector<int64_t> row_base, fwd_base, bwd_base;
@@ -668,6 +670,7 @@ int bwd_impl(const nsp_plan_t* plan, const uint8_t* recompute, const void* q, co
   a.dq = dq;
   a.dq_f32 = dq_dtype == NSP_F32;
   a.dq_turn = dq_turn;
+  a.dq_rounded = plan->rounded_dq ? 1 : 0;
   a.front = plan->d_front;
   a.rows = plan->d_rows;
   a.dk = dk;

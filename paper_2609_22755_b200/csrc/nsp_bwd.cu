@@ -106,6 +106,17 @@ struct BwdSmem {
 };
 static_assert(sizeof(BwdSmem<true, 128>) <= 232448, "shared memory budget (227 KB)");
 
+// DET = 2: every term a key tile adds to the dQ accumulator is first rounded to a multiple of 2^-12 (x + 1.5 * 2^11
+// lands in [2^11, 2^12), where fp32 steps by 2^-12; taking the constant off again is exact). Sums of such multiples are
+// exact in fp32 while they stay below 2^12, so the order of the floating-point reductions no longer matters: the
+// accumulator, and with it dQ, comes out bit for bit the same in every run and for every packing, with no waiting.
+// The price is the quantum itself (2^-13 of error per term, in units of dQ / softmax_scale).
+constexpr float kDqRound = 3072.f;
+template <int DET>
+__device__ __forceinline__ float dq_term(float x) {
+  if constexpr (DET == 2) return __fadd_rn(__fadd_rn(x, kDqRound), -kDqRound);
+  return x;
+}
 __device__ __forceinline__ void red_add_f32(float* addr, float v) {
   asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
 }
@@ -160,11 +171,12 @@ struct QRing {
 // bf16-rounded O. Its dQ rows are complete (no other key tile reaches q tile 0) and are stored directly; its dK / dV
 // rows are the whole result for a one-tile segment and otherwise the part the main kernel, which runs after it, adds
 // its own sum to.
-// DET (main kernel only): the dQ tiles of the key tiles 0, 1, 2, ... of a (segment, q head, q tile) are added to the
+// DET = 2 (main kernel only): see dq_term above.
+// DET = 1 (main kernel only): the dQ tiles of the key tiles 0, 1, 2, ... of a (segment, q head, q tile) are added to the
 // accumulator in exactly that order: a dQ warp waits (bounded) until the turn counter of its q tile says that the key
 // tiles before its own are done, adds, and passes the turn on. In lock-step the CTAs of neighbouring key tiles then
 // follow one another a reduction apart instead of all adding at once.
-template <bool FIRST, bool DET, int D>
+template <bool FIRST, int DET, int D>
 __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   BwdSmem<FIRST, D>& s = *reinterpret_cast<BwdSmem<FIRST, D>*>(smem_raw);
@@ -587,7 +599,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           if (d >= D) {
             tc_fence_before_sync();
             mbar_arrive(&s.bar_dq_empty);
-            if constexpr (DET) {
+            if constexpr (DET == 1) {
               int32_t* turn = a.dq_turn + c.turn_off + h * c.mt + m;
               if (lane == 0) {
                 const long long t0 = clock64();
@@ -629,7 +641,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         }
         float* p0 = tile0 + colhalf * 64 * q_stride;
         int32_t* turn = nullptr;
-        if constexpr (DET) turn = a.dq_turn + c.turn_off + h * c.mt + m;
+        if constexpr (DET == 1) turn = a.dq_turn + c.turn_off + h * c.mt + m;
         auto wait_turn = [&]() -> bool {  // key tiles 0 .. n-1 have added their tiles (eight dQ warps each)
           bool okt = true;
           if (lane == 0) {
@@ -654,7 +666,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           tmem_wait_ld();
           tc_fence_before_sync();
           mbar_arrive(&s.bar_dq_empty);  // R1 is drained: the next dP^T may overwrite it
-          if constexpr (DET) {
+          if constexpr (DET == 1) {
             if (!wait_turn()) {
               if (lane == 0) {
                 report_timeout(a.status, c.it, kWhereBwdTurn, vt);
@@ -671,13 +683,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             float* p1 = p0 + 32 * q_stride;
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-              red_add_f32(p0, __uint_as_float(v0[e]));
-              red_add_f32(p1, __uint_as_float(v1[e]));
+              red_add_f32(p0, dq_term<DET>(__uint_as_float(v0[e])));
+              red_add_f32(p1, dq_term<DET>(__uint_as_float(v1[e])));
               p0 += q_stride;
               p1 += q_stride;
             }
           }
-          if constexpr (DET) pass_turn();
+          if constexpr (DET == 1) pass_turn();
         } else {  // ragged tail: 16 columns at a time, each row checked
           bool okt = true;
 #pragma unroll 1
@@ -689,7 +701,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
               tc_fence_before_sync();
               mbar_arrive(&s.bar_dq_empty);
             }
-            if constexpr (DET) {
+            if constexpr (DET == 1) {
               if (ch == 0) okt = wait_turn();
               if (!okt) continue;
             }
@@ -697,12 +709,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
             for (int e = 0; e < 16; ++e) {
               if (c.hq > 0 && ch * 16 + e < n_valid) {
                 NSP_CHECK(p0 >= a.dq_acc && p0 < a.dq_acc + a.q_elems, a.status, c.it, kWhereCheckBwdDq, m)
-                red_add_f32(p0, __uint_as_float(v[e]));
+                red_add_f32(p0, dq_term<DET>(__uint_as_float(v[e])));
               }
               p0 += q_stride;
             }
           }
-          if constexpr (DET) {
+          if constexpr (DET == 1) {
             if (!okt) {
               if (lane == 0) {
                 report_timeout(a.status, c.it, kWhereBwdTurn, vt);
@@ -1240,7 +1252,7 @@ cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t
 }
 
 namespace {
-template <bool FIRST, bool DET, int D>
+template <bool FIRST, int DET, int D>
 cudaError_t launch_bwd_t(const BwdMaps& maps, const BwdArgs& args, int num_sms, cudaStream_t st) {
   if (args.n_items == 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(bwd_kernel<FIRST, DET, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1255,14 +1267,16 @@ cudaError_t launch_bwd_t(const BwdMaps& maps, const BwdArgs& args, int num_sms, 
 
 cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st) {
   if (head_dim == 64)
-    return args.dq_turn ? launch_bwd_t<false, true, 64>(maps, args, num_sms, st)
-                        : launch_bwd_t<false, false, 64>(maps, args, num_sms, st);
-  return args.dq_turn ? launch_bwd_t<false, true, 128>(maps, args, num_sms, st)
-                      : launch_bwd_t<false, false, 128>(maps, args, num_sms, st);
+    return args.dq_turn    ? launch_bwd_t<false, 1, 64>(maps, args, num_sms, st)
+           : args.dq_rounded ? launch_bwd_t<false, 2, 64>(maps, args, num_sms, st)
+                             : launch_bwd_t<false, 0, 64>(maps, args, num_sms, st);
+  return args.dq_turn    ? launch_bwd_t<false, 1, 128>(maps, args, num_sms, st)
+         : args.dq_rounded ? launch_bwd_t<false, 2, 128>(maps, args, num_sms, st)
+                           : launch_bwd_t<false, 0, 128>(maps, args, num_sms, st);
 }
 cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st) {
-  return head_dim == 64 ? launch_bwd_t<true, false, 64>(maps, args, num_sms, st)
-                        : launch_bwd_t<true, false, 128>(maps, args, num_sms, st);
+  return head_dim == 64 ? launch_bwd_t<true, 0, 64>(maps, args, num_sms, st)
+                        : launch_bwd_t<true, 0, 128>(maps, args, num_sms, st);
 }
 
 cudaError_t launch_bwd_postprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,

@@ -163,6 +163,7 @@ struct BwdArgs {
   void* dq;       // first-tile kernel: rows 0..127 of every segment are stored here directly
   int32_t dq_f32;
   int32_t* dq_turn;  // deterministic dQ: one counter per (segment, q head, q tile), zeroed before the launch; else null
+  int32_t dq_rounded;  // 1: dQ terms rounded to a fixed quantum before they are added (order-independent sums)
   void* dk;
   void* dv;
   int32_t dkv_f32;
@@ -192,7 +193,7 @@ cudaError_t launch_bwd_preprocess(const SegInfo* d_seg, int n_seg, const int64_t
                                   float* dq_acc, const uint8_t* seg_skip, const float* lse_in, float* lse_out,
                                   cudaStream_t st);
 cudaError_t launch_bwd_first(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st);
-cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st);  // args.dq_turn selects the deterministic variant
+cudaError_t launch_bwd(const BwdMaps& maps, const BwdArgs& args, int head_dim, int num_sms, cudaStream_t st);  // args.dq_turn / args.dq_rounded select the reproducible variants
 cudaError_t launch_bwd_postprocess(const SegInfo* d_seg, int n_seg, const int64_t* d_row_base, int64_t total_rows,
                                    int head_dim, const float* dq_acc, void* dq, int dq_f32, float scale,
                                    cudaStream_t st);

@@ -45,7 +45,9 @@ class GpuRun:
         self.dev = torch.device(device)
         self.host = tensors if tensors is not None else W.make_tensors(w)
         self.q, self.k, self.v, self.do = (self.host[n].to(self.dev) for n in ("q", "k", "v", "do"))
-        opts = (128, 128, 1, B.NSP_PLAN_DETERMINISTIC_DQ) if deterministic else None
+        # deterministic: False, True (ordered additions) or "rounded" (terms rounded to a fixed quantum)
+        flag = B.NSP_PLAN_ROUNDED_DQ if deterministic == "rounded" else B.NSP_PLAN_DETERMINISTIC_DQ
+        opts = (128, 128, 1, flag) if deterministic else None
         self.plan = B.nsp_plan_tiles(w.cu_seqlens, w.hq, w.hkv, w.head_dim, opts=opts)
         assert self.plan.q_elems == w.q_elems() and self.plan.kv_elems == w.kv_elems()
         assert self.plan.lse_elems == w.lse_elems()

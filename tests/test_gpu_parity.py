@@ -418,13 +418,16 @@ def test_packing_order_invariance_and_reproducibility(env):
         assert np.max(np.abs(x - y) / np.maximum(np.abs(y), 1e-3)) <= 2.0 ** -7
 
 
-def test_deterministic_dq_option_is_bitwise_reproducible(env):
-    """Plan flag NSP_PLAN_DETERMINISTIC_DQ: the dQ tiles are added in key-tile order, so every output, dQ included, is
-    bit for bit the same in two runs and under a permuted packing; and it still matches the oracle."""
+@pytest.mark.parametrize("mode", [True, "rounded"])
+def test_deterministic_dq_option_is_bitwise_reproducible(env, mode):
+    """Plan flags NSP_PLAN_DETERMINISTIC_DQ (the dQ tiles are added in key-tile order) and NSP_PLAN_ROUNDED_DQ (every
+    term is rounded to a fixed quantum first, so that the fp32 sums are exact and their order is irrelevant): every
+    output, dQ included, is bit for bit the same in three runs and under a permuted packing; and it still matches the
+    oracle."""
     W, P, torch = env["W"], env["P"], env["torch"]
     lengths, hq, hkv = [3000, 130, 2048, 700, 64], [8, 8, 4, 4, 4], [2, 2, 1, 1, 1]
     w = W.custom(lengths, hq, hkv, seed=23)
-    run = P.GpuRun(w, dq_dtype="f32", deterministic=True)
+    run = P.GpuRun(w, dq_dtype="f32", deterministic=mode)
     outs = []
     for _ in range(3):
         for t in (run.dq, run.dk, run.dv):
@@ -442,7 +445,7 @@ def test_deterministic_dq_option_is_bitwise_reproducible(env):
     host = {}
     for name, off in (("q", qo), ("do", qo), ("k", kvo), ("v", kvo)):
         host[name] = torch.cat([run.host[name][off[p]:off[p + 1]] for p in perm])
-    runp = P.GpuRun(wp, tensors=host, dq_dtype="f32", deterministic=True)
+    runp = P.GpuRun(wp, tensors=host, dq_dtype="f32", deterministic=mode)
     runp.forward()
     runp.backward()
     c = runp.results()
