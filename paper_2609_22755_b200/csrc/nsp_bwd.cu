@@ -1133,17 +1133,6 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
   const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
   for (int64_t grp = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; grp < n_groups; grp += n_warps) {
     const int64_t row0 = grp * kRowsPerPass;
-    uint4 va[4], vb[4];
-#pragma unroll
-    for (int p = 0; p < 4; ++p) {
-      const int64_t row = row0 + kRowsPerLoad * p + sub;
-      if (row < total_rows) {
-        va[p] = __ldg(reinterpret_cast<const uint4*>(o + row * D) + l);
-        vb[p] = __ldg(reinterpret_cast<const uint4*>(d_o + row * D) + l);
-      } else {
-        va[p] = vb[p] = make_uint4(0u, 0u, 0u, 0u);
-      }
-    }
     // row row0 + (lane % kRowsPerPass): where its delta goes (-1: nowhere), and whether it is one of the main kernel's rows
     int64_t dst = -1;
     int mine = 0;
@@ -1164,6 +1153,21 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
         }
       }
     }
+    // O and dO are read only for the rows whose delta is wanted: with short segments the first 128 tokens, which the
+    // first-tile kernel serves, are a large part of the batch (half of it at 256-token segments)
+    uint4 va[4], vb[4];
+    int64_t dst_p[4];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      const int64_t row = row0 + kRowsPerLoad * p + sub;
+      dst_p[p] = __shfl_sync(0xffffffffu, dst, kRowsPerLoad * p + sub);
+      if (dst_p[p] >= 0) {
+        va[p] = __ldg(reinterpret_cast<const uint4*>(o + row * D) + l);
+        vb[p] = __ldg(reinterpret_cast<const uint4*>(d_o + row * D) + l);
+      } else {
+        va[p] = vb[p] = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
       const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&va[p]);
@@ -1177,9 +1181,8 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const SegInfo* __re
       }
 #pragma unroll
       for (int sft = kLanesPerRow / 2; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
-      const int64_t dst_p = __shfl_sync(0xffffffffu, dst, kRowsPerLoad * p + sub);
       const int mine_p = __shfl_sync(0xffffffffu, mine, kRowsPerLoad * p + sub);
-      if (l == 0 && dst_p >= 0) delta[dst_p] = acc;
+      if (l == 0 && dst_p[p] >= 0) delta[dst_p[p]] = acc;
       if (mine_p) {
         float4* z = reinterpret_cast<float4*>(dq_acc + (row0 + kRowsPerLoad * p + sub) * D) + 2 * l;
         z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
