@@ -659,7 +659,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           __syncwarp();
           if (lane == 0) atomicAdd(turn, 1);
         };
-        if (n_valid >= 64) {  // interior tile: no row checks
+        {
+          // One drain for interior and ragged tiles: every reduction under its row's predicate (rows past the segment
+          // end are skipped: their dS^T columns are zero, and they may lie outside the buffer). Every item starts on
+          // the segment's last q tile, once per q head, so a ragged tile must not cost more than an interior one: as a
+          // rolled loop of 16-column loads with a wait each, R1 was handed back late and such a step took twice as long
+          // (batches of 500-, 1,000- and 2,000-token segments ran 10-18 % slower per flop than 512 / 1,024 / 2,048).
           uint32_t v0[32], v1[32];
           tmem_ld32(tR1 + lane_off + colhalf * 64, v0);
           tmem_ld32(tR1 + lane_off + colhalf * 64 + 32, v1);
@@ -678,52 +683,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           // The reductions sit in a conditional region on purpose (the condition always holds): as straight-line
           // code the compiler computes all 64 row addresses ahead of the TMEM loads, runs out of the 80 registers
           // this role has and spills inside the loop (measured: the whole kernel 25 % slower).
-          NSP_CHECK(p0 >= a.dq_acc && p0 + 63 * q_stride < a.dq_acc + a.q_elems, a.status, c.it, kWhereCheckBwdDq, m)
+          NSP_CHECK(n_valid <= 0 || (p0 >= a.dq_acc && p0 + (min(n_valid, 64) - 1) * q_stride < a.dq_acc + a.q_elems), a.status,
+                    c.it, kWhereCheckBwdDq, m)
           if (c.hq > 0) {
             float* p1 = p0 + 32 * q_stride;
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-              red_add_f32(p0, dq_term<DET>(__uint_as_float(v0[e])));
-              red_add_f32(p1, dq_term<DET>(__uint_as_float(v1[e])));
+              if (e < n_valid) red_add_f32(p0, dq_term<DET>(__uint_as_float(v0[e])));
+              if (e + 32 < n_valid) red_add_f32(p1, dq_term<DET>(__uint_as_float(v1[e])));
               p0 += q_stride;
               p1 += q_stride;
             }
           }
           if constexpr (DET == 1) pass_turn();
-        } else {  // ragged tail: 16 columns at a time, each row checked
-          bool okt = true;
-#pragma unroll 1
-          for (int ch = 0; ch < 4; ++ch) {
-            uint32_t v[16];
-            tmem_ld16(tR1 + lane_off + colhalf * 64 + ch * 16, v);
-            tmem_wait_ld();
-            if (ch == 3) {
-              tc_fence_before_sync();
-              mbar_arrive(&s.bar_dq_empty);
-            }
-            if constexpr (DET == 1) {
-              if (ch == 0) okt = wait_turn();
-              if (!okt) continue;
-            }
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              if (c.hq > 0 && ch * 16 + e < n_valid) {
-                NSP_CHECK(p0 >= a.dq_acc && p0 < a.dq_acc + a.q_elems, a.status, c.it, kWhereCheckBwdDq, m)
-                red_add_f32(p0, dq_term<DET>(__uint_as_float(v[e])));
-              }
-              p0 += q_stride;
-            }
-          }
-          if constexpr (DET == 1) {
-            if (!okt) {
-              if (lane == 0) {
-                report_timeout(a.status, c.it, kWhereBwdTurn, vt);
-                *abort_flag = 1;
-              }
-              break;
-            }
-            pass_turn();
-          }
         }
       }
       item_done();
