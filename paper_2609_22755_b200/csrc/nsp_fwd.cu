@@ -83,7 +83,9 @@ struct FwdRound {
   nsp_tile_t a, b;
   int joint;
 };
-template <int D>
+// RECOMP: the instantiation the recomputing backward pass launches (marked segments only; LSE and delta instead of O).
+// The plain forward pass carries none of that code: the long items are sensitive to the size of the kernel.
+template <int D, bool RECOMP>
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   FwdSmem<D>& s = *reinterpret_cast<FwdSmem<D>*>(smem_raw);
@@ -158,7 +160,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       bool have_b = it + 1 < a.n_items;
       nsp_tile_t ia = a.items[it];
       nsp_tile_t ib = have_b ? a.items[it + 1] : ia;
-      if (a.seg_mask != nullptr) {  // recomputation: only the marked segments
+      if (RECOMP && a.seg_mask != nullptr) {  // recomputation: only the marked segments
         const bool fa = a.seg_mask[ia.seg] != 0, fb = have_b && a.seg_mask[ib.seg] != 0;
         if (!fa && !fb) continue;
         if (!fa) ia = ib;
@@ -547,7 +549,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           pvn += n_kv;
           const int row = q_row0 + rl;
           const bool valid = row < sg.len;
-          if (ok && a.delta != nullptr) {
+          if (RECOMP && ok && a.delta != nullptr) {
             // ---- epilogue of a recomputation: LSE and delta = <dO, O> of the row, O itself is not written.
             // The half-row dot product is taken with the unnormalised O and handed over together with the half-row
             // sum.
@@ -694,14 +696,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
 }  // namespace
 
 namespace {
-template <int D>
+template <int D, bool RECOMP>
 cudaError_t launch_fwd_t(const FwdMaps& maps, const FwdArgs& args, int num_sms, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(fwd_kernel<D, RECOMP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(sizeof(FwdSmem<D>)));
   if (e != cudaSuccess) return e;
   const int pops = (args.n_items + 1) / 2;
   const int grid = pops < num_sms ? pops : num_sms;
-  fwd_kernel<D><<<grid, kFwdThreads, sizeof(FwdSmem<D>), st>>>(maps, args);
+  fwd_kernel<D, RECOMP><<<grid, kFwdThreads, sizeof(FwdSmem<D>), st>>>(maps, args);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -709,7 +711,10 @@ cudaError_t launch_fwd_t(const FwdMaps& maps, const FwdArgs& args, int num_sms, 
 
 cudaError_t launch_fwd(const FwdMaps& maps, const FwdArgs& args, int head_dim, int num_sms, cudaStream_t st) {
   if (args.n_items == 0) return cudaSuccess;
-  return head_dim == 64 ? launch_fwd_t<64>(maps, args, num_sms, st) : launch_fwd_t<128>(maps, args, num_sms, st);
+  const bool recomp = args.delta != nullptr || args.seg_mask != nullptr;
+  if (head_dim == 64)
+    return recomp ? launch_fwd_t<64, true>(maps, args, num_sms, st) : launch_fwd_t<64, false>(maps, args, num_sms, st);
+  return recomp ? launch_fwd_t<128, true>(maps, args, num_sms, st) : launch_fwd_t<128, false>(maps, args, num_sms, st);
 }
 
 }  // namespace nsp
