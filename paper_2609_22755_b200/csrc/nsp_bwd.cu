@@ -51,8 +51,15 @@ constexpr int kBwdThreads = 640;  // 8 softmax warps, 8 dQ warps, one auxiliary 
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
-// setmaxnreg redistributes the launch-time allocation (96 per thread): 256*136 + 256*80 + 128*48 = 640*96
-constexpr int kRegsSoftmax = 136, kRegsReduce = 80, kRegsAux = 48;
+// setmaxnreg redistributes the launch-time allocation (96 per thread, 640 threads): softmax x2 / dQ x2 / auxiliary.
+// Main kernel 120 / 96 / 48: the dQ role holds 64 accumulator values, 64 row pointers' worth of arithmetic and the
+// turn logic, and with 80 registers it spilled inside its drain (cfg4 backward 400 ms; 88: 392 ms; 96: 389 ms, the
+// most a warpgroup can keep without an increase of its own), while the softmax role fits 120. First-tile kernel
+// 136 / 80 / 48: there the softmax role carries the packed P of a whole tile across two sweeps and the dQ role only
+// stores. 256 * (120 + 96) + 128 * 48 = 256 * (136 + 80) + 128 * 48 = 640 * 96.
+template <bool FIRST> constexpr int kRegsSoftmax = FIRST ? 136 : 120;
+template <bool FIRST> constexpr int kRegsReduce = FIRST ? 80 : 96;
+constexpr int kRegsAux = 48;
 constexpr int kFrontMinSteps = 2048;          // items shorter than this start at once
 constexpr int kFrontMinGroup = 8;             // so do items of groups with fewer q heads per kv head
 constexpr long long kFrontWaitClk = 1500000;  // ~0.9 ms: upper bound of the start alignment (also: 1/16 of the item)
@@ -560,7 +567,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     }
   } else if (wg >= 2) {
     // ================================================================ dQ^T: R1 -> global fp32 accumulator
-    setmaxnreg_dec<kRegsReduce>();
+    setmaxnreg_dec<kRegsReduce<FIRST>>();
     const int quad = warp & 3, colhalf = wg - 2;  // this warp drains query columns [64*colhalf, 64*colhalf + 64)
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
     const int d = quad * 32 + lane;  // head-dimension index = TMEM lane
@@ -702,7 +709,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     }
   } else {
     // ================================================================ softmax / dS (key row r, 64 query columns)
-    setmaxnreg_inc<kRegsSoftmax>();
+    setmaxnreg_inc<kRegsSoftmax<FIRST>>();
     const int quad = warp & 3, half = wg;
     const int r = quad * 32 + lane;
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
