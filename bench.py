@@ -305,7 +305,8 @@ def main():
     # and the CUDA runtime's threads, the same oracle sample ran half as fast.
     cpu = None
     if world == 1 and rank == 0 and not args.no_cpu_baseline:
-        cmd = [sys.executable, str(Path(__file__).resolve()), "--impl", "reference", "--steps", "1", "--warmup", "0",
+        # one untimed pass first: on the GPU hosts the first pass of a fresh process takes twice as long as every later one
+        cmd = [sys.executable, str(Path(__file__).resolve()), "--impl", "reference", "--steps", "1", "--warmup", "1",
                "--config", str(args.config)] + (["--uniform", str(args.uniform)] if args.uniform else [])
         r = subprocess.run(cmd, capture_output=True, text=True)
         try:
