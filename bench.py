@@ -300,12 +300,11 @@ def main():
     if not args.profile_mode:
         args.warmup = max(args.warmup, 3)
 
-    # The CPU baseline is timed first, in a process of its own that never touches CUDA (it is the reference arm of
-    # this script run for one step): timed inside this process after the GPU work, next to 3.5 GB of pinned memory
-    # and the CUDA runtime's threads, the same oracle sample ran half as fast.
+    # The CPU baseline is timed first, in a process of its own that never touches CUDA: it is the reference arm of
+    # this script run for one untimed and one timed step, so the two arms report the same figure.
     cpu = None
     if world == 1 and rank == 0 and not args.no_cpu_baseline:
-        # one untimed pass first: on the GPU hosts the first pass of a fresh process takes twice as long as every later one
+        # the untimed pass matters: on the GPU hosts the first pass of a fresh process takes twice as long as the later ones
         cmd = [sys.executable, str(Path(__file__).resolve()), "--impl", "reference", "--steps", "1", "--warmup", "1",
                "--config", str(args.config)] + (["--uniform", str(args.uniform)] if args.uniform else [])
         r = subprocess.run(cmd, capture_output=True, text=True)
