@@ -120,7 +120,7 @@ def peaks_in_run(torch):
     return {"bf16_tflops": tflops, "hbm_gbs": gbs, "how": "torch.matmul bf16 8192^3 best of 10; copy of 2^30 bf16 best of 10"}
 
 
-def short_segment_roofline(torch, B, peaks, lengths=(128, 512), iters=5):
+def short_segment_roofline(torch, B, peaks, lengths=(32, 128, 512), iters=5):
     """The HBM-bound class: uniform batches of 131,072 tokens at 32q/4kv in segments of L tokens; achieved algorithmic
     bytes per second of the forward launch and of the backward launches against the measured copy bandwidth."""
     out = {}
@@ -164,7 +164,8 @@ def short_segment_roofline(torch, B, peaks, lengths=(128, 512), iters=5):
         del q, do, k, v, o, dq, lse, dk, dv, ws
         torch.cuda.empty_cache()
     return {"bound": "hbm", "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_kind": f"hbm_gbs of {peaks['source']}",
-            "note": "bwd = memset + preprocess + main + postprocess", **out}
+            "note": "bwd = all launches of the backward pass (first-tile kernel; preprocess, main and postprocess where a "
+                    "segment has more than one tile); at L = 32 four segments share a tile", **out}
 
 
 class ClockSampler:
